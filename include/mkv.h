@@ -1,0 +1,156 @@
+/*
+ * mkv.h -- C ABI of the MorphKV decode + update hot path for NVIDIA B200 (sm_100a).
+ *
+ * MorphKV ("Dialogue Without Limits: Constant-Sized KV Caches for Extended Responses in
+ * LLMs", arXiv 2503.00979) keeps, for every layer and KV head, a cache of C selected
+ * distant tokens plus the R most recent tokens.  One *unit* is a (layer, batch row, KV head)
+ * triple serving G = n_q_heads / n_kv_heads grouped query heads; units share nothing
+ * ("Handling Multiple Heads").  Each decode step does, per unit:
+ *
+ *   attend   Eq. 1: soft-max attention of the new query over the cached tokens and itself;
+ *   score    Eq. 4-6 + Algorithm 1: every cached token outside the recent window gets
+ *            F[k] = sum_r or max_r of S_r[k], S_r[k] = sum over the GQA group of the weight
+ *            window token r assigned to k when r was generated;
+ *   select   Algorithm 1 / Eq. 7: keep the C largest F (ties: the lower position is kept);
+ *   update   Eq. 7 + the "lightweight KV cache extension" of the Implementation paragraph:
+ *            the evicted slot receives the new token's K/V, and the new query with its
+ *            soft-max statistics replaces the oldest row of the recent-query ring.
+ *
+ * Conventions
+ *   - Every `const void*` / `void*` tensor argument is a DEVICE pointer unless the name of
+ *     the function ends in `_host`.  Tensors are contiguous, row-major, in the context's
+ *     dtype (bf16 or f32).  The library applies no positional encoding: q and k are used
+ *     as given.
+ *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = the default stream).  Calls
+ *     enqueue work on it and return without synchronising unless stated otherwise.
+ *   - No call throws or aborts across this boundary.  Every call returns an `mkv_status`;
+ *     `mkv_last_error` gives the text of the last failure of a context.
+ *   - There is no CPU fallback: without a CUDA device every compute call returns MKV_CUDA.
+ *   - Input buffers are borrowed until the enqueued work has completed.
+ */
+#ifndef MKV_H
+#define MKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum mkv_status {
+    MKV_OK = 0,
+    MKV_INVALID_ARG = 1,    /* a parameter or pointer is out of range / NULL               */
+    MKV_BAD_STATE = 2,      /* call order violated (e.g. decode before prefill)            */
+    MKV_OOM = 3,            /* workspace too small or device allocation failed             */
+    MKV_CUDA = 4,           /* a CUDA runtime call failed (text in mkv_last_error)         */
+    MKV_UNSUPPORTED = 5,    /* valid request this build has no kernel for                  */
+    MKV_DEVICE_TIMEOUT = 6  /* a bounded device-side wait gave up; state is undefined      */
+} mkv_status;
+
+typedef enum mkv_fusion { MKV_FUSION_SUM = 0, MKV_FUSION_MAX = 1 } mkv_fusion;   /* Eq. 5, Eq. 6 */
+typedef enum mkv_dtype { MKV_DTYPE_BF16 = 0, MKV_DTYPE_F32 = 1 } mkv_dtype;
+/* which decode kernel to use: AUTO picks the tensor-core kernel when the shape allows it */
+typedef enum mkv_kernel { MKV_KERNEL_AUTO = 0, MKV_KERNEL_SIMT = 1, MKV_KERNEL_TC = 2 } mkv_kernel;
+
+typedef struct mkv_ctx mkv_ctx;
+
+typedef struct mkv_params {
+    int layers, batch, n_q_heads, n_kv_heads, head_dim;
+    int C;                  /* distant tokens retained per unit (Eq. 3)                    */
+    int R;                  /* recent window (H1)                                           */
+    mkv_fusion fusion;
+    mkv_dtype dtype;
+    int evict_interval;     /* run the policy every T-th step (coarse-grained eviction
+                               appendix); 0 or 1 = every step                              */
+    mkv_kernel kernel;
+    int splits;             /* CTAs cooperating on one unit's cache; 0 = choose            */
+    void *workspace;        /* device memory owned by the caller, 256-byte aligned, or NULL
+                               to let the library allocate it with cudaMalloc              */
+    size_t workspace_bytes;
+} mkv_params;
+
+/* What one layer of the cache looks like.  Slot order inside a unit is unspecified: the
+ * retained set of unit (b, h) is { pos[b][h][i] : i < count }. */
+typedef struct mkv_view {
+    void *K, *V;            /* [batch][n_kv_heads][capacity][head_dim], context dtype      */
+    int32_t *pos;           /* [batch][n_kv_heads][capacity] absolute position, -1 = free  */
+    float *F;               /* [batch][n_kv_heads][capacity] fused score of each slot at the
+                               last selection (-1 for slots inside the recent window)      */
+    int32_t *evicted_pos;   /* [batch][n_kv_heads] position evicted by the last step, -1 = none */
+    void *ring_q;           /* [batch][n_kv_heads][R][G][head_dim] recent queries; the query of
+                               position p sits in ring row p % R                            */
+    float *ring_c;          /* [batch][n_kv_heads][R][G] log2-domain soft-max normaliser of a
+                               ring row: weight(k) = exp2(q.k * log2(e)/sqrt(d) - ring_c);
+                               +inf marks an empty row                                     */
+    int32_t count;          /* tokens cached per unit (the same for every unit)            */
+    int32_t capacity;       /* slots per unit: C + R + evict_interval - 1                  */
+    int64_t next_pos;       /* absolute position of the next token to decode               */
+} mkv_view;
+
+/* Fills *p with defaults: bf16, every-step eviction, automatic kernel and split choice,
+ * library-owned workspace.  The caller then sets the shape fields. */
+void mkv_default_params(mkv_params *p);
+
+/* Bytes of device workspace a context with these parameters needs (0 if they are invalid). */
+size_t mkv_workspace_bytes(const mkv_params *p);
+
+/* Problem statement of the paper (Eq. 2-3): a cache of C + R entries per KV head.
+ * bf16, every-step eviction, library-owned workspace.  Validates: all sizes >= 1,
+ * n_q_heads % n_kv_heads == 0 with a group of at most 16, head_dim in {64, 128}.
+ * No kernel is launched. */
+mkv_status mkv_create(mkv_ctx **out, int layers, int batch, int n_q_heads, int n_kv_heads,
+                      int head_dim, int C, int R, mkv_fusion fusion);
+
+/* Same with every option spelled out.  If p->workspace is non-NULL the context lives in
+ * that caller-owned memory (at least mkv_workspace_bytes(p) bytes) and never allocates
+ * device memory for its state. */
+mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p);
+
+/* Releases the context (and its workspace if the library allocated it).  NULL is allowed. */
+void mkv_destroy(mkv_ctx *ctx);
+
+/* Prompt phase (the paper gives no procedure; this applies Algorithm 1 once with the whole
+ * prompt as G_i): k, v [layers][batch][n_kv_heads][prompt_len][head_dim]; q_window
+ * [layers][batch][n_q_heads][min(R, prompt_len)][head_dim] = the queries of the last prompt
+ * positions, oldest first.  If prompt_len <= C + R everything is kept; otherwise the window
+ * rows are scored causally over all prompt keys and the top C older tokens are kept.
+ * Allocates temporary device scratch; synchronises the stream before returning. */
+mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
+                       int prompt_len, void *stream);
+
+/* One decode step for every unit (Eq. 1, Eq. 4-7, Algorithm 1): q, out
+ * [layers][batch][n_q_heads][head_dim]; k_new, v_new [layers][batch][n_kv_heads][head_dim].
+ * Asynchronous; launches a fixed kernel sequence with no host-side dependence on the step
+ * index, so a sequence of calls can be recorded into a CUDA graph. */
+mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                           void *out, void *stream);
+
+/* n_steps consecutive decode steps; every tensor has a leading [n_steps] dimension. */
+mkv_status mkv_decode_steps(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                            void *out, int n_steps, void *stream);
+
+/* One decode step with HOST buffers (pinned memory recommended): copies q, k_new, v_new to
+ * the device, runs the step, copies `out` back, all on `stream`; does not synchronise. */
+mkv_status mkv_decode_step_host(mkv_ctx *ctx, const void *q_host, const void *k_new_host,
+                                const void *v_new_host, void *out_host, void *stream);
+
+/* Device pointers into one layer of the cache.  Valid until the context is destroyed;
+ * contents change with every decode step.  Reading them needs a stream synchronisation. */
+mkv_status mkv_cache_view(mkv_ctx *ctx, int layer, mkv_view *view);
+
+/* Waits for `stream` and reports device-side errors (MKV_DEVICE_TIMEOUT) recorded so far. */
+mkv_status mkv_sync(mkv_ctx *ctx, void *stream);
+
+/* Text of the last failure on this context ("" if none).  Never NULL. */
+const char *mkv_last_error(const mkv_ctx *ctx);
+
+/* Counters for reporting: kernels launched by this context so far, and the name of the
+ * decode kernel in use ("simt" or "tc"). */
+uint64_t mkv_launch_count(const mkv_ctx *ctx);
+const char *mkv_kernel_name(const mkv_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MKV_H */

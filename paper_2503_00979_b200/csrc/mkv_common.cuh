@@ -1,0 +1,229 @@
+// Shared device-side definitions of the MorphKV decode path: argument blocks, element
+// helpers and the per-unit epilogue that merges split partials, selects the eviction and
+// appends the new token (Eq. 1 merge, Eq. 4-7, Algorithm 1 of the paper).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mkv {
+
+constexpr int kMaxGroup = 16;     // largest supported GQA group size
+constexpr int kFusionSum = 0;
+constexpr int kFusionMax = 1;
+
+// Device-resident step state.  Kernels read it at entry; the last CTA of a launch to finish
+// advances it, so consecutive launches need no host-side step index.
+struct DevState {
+    long long t;          // absolute position of the token being decoded
+    int n;                // tokens cached per unit before this step
+    int steps;            // decode steps completed
+    int err;              // sticky device-side error code (0 = none)
+    unsigned int done;    // CTAs of the current launch that have finished
+    int pad;
+};
+
+enum DevError { kErrNone = 0, kErrBarrierTimeout = 1 };
+
+// Everything a decode kernel needs.  Passed by value as a __grid_constant__.
+struct DecodeArgs {
+    void *K, *V;               // [U][cap][D]
+    int *pos;                  // [U][cap]
+    void *ring_q;              // [U][R][G][D]
+    float *ring_c;             // [U][R][G]
+    const void *q, *k_new, *v_new;
+    void *out;
+    float *s_new;              // [U][G][cap]   scaled log2-domain logits of the new query
+    float *F;                  // [U][cap]      fused score (partial, then final)
+    float *part_ml;            // [U][splits][G][2]  (max, denominator) of each split
+    float *part_o;             // [U][splits][G][D]  un-normalised split outputs
+    int *ticket;               // [U]
+    int *evicted_pos;          // [U]
+    DevState *st;
+    int U, G, R, C, cap, splits, fusion, T;
+    float scale2;              // log2(e) / sqrt(D)
+};
+
+__device__ __forceinline__ float ldf(const float *p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float *p, float v) { *p = v; }
+__device__ __forceinline__ void stf(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float fuse(int fusion, float a, float b)
+{
+    return fusion == kFusionSum ? a + b : fmaxf(a, b);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Ordering key of a candidate: larger key = better.  Fused scores are non-negative floats,
+// whose bit patterns order like the values; among equal scores the LOWER position gets the
+// larger key, so it is the one kept.  All keys of a unit are distinct.
+__host__ __device__ __forceinline__ unsigned long long rank_key(unsigned int F_bits, int pos)
+{
+    return ((unsigned long long)F_bits << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)pos);
+}
+
+// How a unit's n cached tokens are divided among `splits` CTAs: contiguous ranges whose
+// length is a multiple of `tile`.  Returns the per-split length; *active = splits with work.
+__host__ __device__ inline int split_len(int n, int splits, int tile, int *active)
+{
+    const int tiles = (n + tile - 1) / tile;
+    const int per = ((tiles + splits - 1) / splits) * tile;
+    *active = per > 0 ? (n + per - 1) / per : 0;
+    return per;
+}
+
+// True when this step must evict: after the new token joins, the tokens outside the window
+// of min(R, t+1) recent ones exceed C (Eq. 7 keeps the cache at C + R).
+__host__ __device__ inline bool step_evicts(long long t, int n, int R, int C)
+{
+    const long long win = (t + 1 < (long long)R) ? t + 1 : (long long)R;
+    return (long long)n + 1 - win > (long long)C;
+}
+
+constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32;
+
+// Per-unit epilogue, run by the whole CTA that finished a unit last.  Data written by other
+// CTAs is read with ld.global.cg so that no stale L1 line can be used.  `sm` needs
+// kFinalizeSmemFloats floats of shared memory, 8-byte aligned.
+template <typename T, int D>
+__device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, int active, bool evict, float *sm)
+{
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const int G = a.G;
+    float *s_self = sm, *mfin = sm + kMaxGroup, *lfin = sm + 2 * kMaxGroup, *cnew = sm + 3 * kMaxGroup;
+    unsigned long long *red_key = reinterpret_cast<unsigned long long *>(sm + 4 * kMaxGroup);  // [32]
+    int *red_slot = reinterpret_cast<int *>(sm + 4 * kMaxGroup + 64);                          // [32]
+
+    const T *q = static_cast<const T *>(a.q) + (size_t)u * G * D;
+    const T *kn = static_cast<const T *>(a.k_new) + (size_t)u * D;
+    const T *vn = static_cast<const T *>(a.v_new) + (size_t)u * D;
+    const float *pml = a.part_ml + (size_t)u * a.splits * G * 2;
+    const float *po = a.part_o + (size_t)u * a.splits * G * D;
+
+    // the new token attends to itself (self-inclusive Eq. 1): one more logit per head
+    for (int g = warp; g < G; g += nwarp) {
+        float acc = 0.f;
+        for (int i = lane; i < D; i += 32) acc += ldf(q + g * D + i) * ldf(kn + i);
+        acc = warp_sum(acc);
+        if (lane == 0) s_self[g] = acc * a.scale2;
+    }
+    __syncthreads();
+    if (tid < G) {
+        float m = s_self[tid];
+        for (int sp = 0; sp < active; ++sp) m = fmaxf(m, __ldcg(pml + (sp * G + tid) * 2));
+        float l = exp2f(s_self[tid] - m);
+        for (int sp = 0; sp < active; ++sp)
+            l += __ldcg(pml + (sp * G + tid) * 2 + 1) * exp2f(__ldcg(pml + (sp * G + tid) * 2) - m);
+        mfin[tid] = m;
+        lfin[tid] = l;
+        cnew[tid] = m + log2f(l);
+    }
+    __syncthreads();
+    T *out = static_cast<T *>(a.out) + (size_t)u * G * D;
+    for (int idx = tid; idx < G * D; idx += nthr) {
+        const int g = idx / D, dd = idx % D;
+        const float m = mfin[g];
+        float o = exp2f(s_self[g] - m) * ldf(vn + dd);
+        for (int sp = 0; sp < active; ++sp)
+            o += __ldcg(po + (sp * G + g) * D + dd) * exp2f(__ldcg(pml + (sp * G + g) * 2) - m);
+        stf(out + idx, o / lfin[g]);
+    }
+
+    // Algorithm 1 / Eq. 7: add the new row's term to the fused scores, evict the minimum
+    int *pos = a.pos + (size_t)u * a.cap;
+    float *F = a.F + (size_t)u * a.cap;
+    int e_slot = n, e_pos = -1;
+    if (evict) {
+        const float *sn = a.s_new + (size_t)u * G * a.cap;
+        const long long thr = t - a.R;
+        unsigned long long best = ~0ull;
+        int bslot = -1;
+        for (int k = tid; k < n; k += nthr) {
+            const int p = pos[k];
+            if ((long long)p <= thr) {
+                float s = 0.f;
+                for (int g = 0; g < G; ++g) s += exp2f(__ldcg(sn + (size_t)g * a.cap + k) - cnew[g]);
+                const float f = fuse(a.fusion, __ldcg(F + k), s);
+                F[k] = f;
+                const unsigned long long key = rank_key(__float_as_uint(f), p);
+                if (key < best) { best = key; bslot = k; }
+            } else {
+                F[k] = -1.f;   // window slot: not a candidate
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+            const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+            if (ok < best) { best = ok; bslot = os; }
+        }
+        if (lane == 0) { red_key[warp] = best; red_slot[warp] = bslot; }
+        __syncthreads();
+        if (warp == 0) {
+            best = lane < nwarp ? red_key[lane] : ~0ull;
+            bslot = lane < nwarp ? red_slot[lane] : -1;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+                const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+                if (ok < best) { best = ok; bslot = os; }
+            }
+            if (lane == 0) red_slot[0] = bslot;
+        }
+        __syncthreads();
+        e_slot = red_slot[0];
+        e_pos = pos[e_slot];
+        __syncthreads();
+    }
+
+    // Eq. 7 update: the freed (or next free) slot takes the new token; the ring row of the
+    // token that left the window takes the new query and its soft-max normaliser
+    T *Kd = static_cast<T *>(a.K) + ((size_t)u * a.cap + e_slot) * D;
+    T *Vd = static_cast<T *>(a.V) + ((size_t)u * a.cap + e_slot) * D;
+    for (int i = tid; i < D; i += nthr) { Kd[i] = kn[i]; Vd[i] = vn[i]; }
+    const int rs = (int)(t % a.R);
+    T *rq = static_cast<T *>(a.ring_q) + ((size_t)u * a.R + rs) * G * D;
+    for (int i = tid; i < G * D; i += nthr) rq[i] = q[i];
+    if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
+    if (tid == 0) {
+        pos[e_slot] = (int)t;
+        a.evicted_pos[u] = e_pos;
+        a.ticket[u] = 0;
+    }
+}
+
+// Last action of every CTA of a decode launch: the CTA that finishes last advances the
+// device-resident step state.  Must be called by all CTAs, after all their other work,
+// so that no CTA can still be about to read the state when it changes.
+__device__ __forceinline__ void finish_cta(const DecodeArgs &a, long long t, int n, bool evict)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int total = gridDim.x * gridDim.y * gridDim.z;
+        if (atomicAdd(&a.st->done, 1u) == total - 1) {
+            a.st->t = t + 1;
+            a.st->n = evict ? n : n + 1;
+            a.st->steps += 1;
+            a.st->done = 0;
+            __threadfence();
+        }
+    }
+}
+
+}  // namespace mkv

@@ -1,0 +1,18 @@
+// Host-callable launchers of the MorphKV kernels (internal to the library).
+#pragma once
+
+#include "mkv_common.cuh"
+
+namespace mkv {
+
+// CUDA-core decode step (any supported shape).  `a.splits` CTAs per unit.
+cudaError_t launch_decode_simt(const DecodeArgs &a, bool f32, int D, cudaStream_t stream);
+int simt_default_splits(int U, int cap);
+
+// Prompt phase: fills the arena (K, V, pos, ring) and the step state from a prompt of P
+// tokens.  `a` supplies the arena pointers and shape; q/k_new/v_new/out are ignored.
+// Allocates and frees its own temporary scratch.  *launches is advanced per kernel launched.
+cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
+                        int P, cudaStream_t stream, unsigned long long *launches);
+
+}  // namespace mkv
