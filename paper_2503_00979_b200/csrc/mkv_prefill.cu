@@ -1,0 +1,328 @@
+// Prompt phase of MorphKV (set-up, not part of the per-token hot path).
+//
+// The paper states no prefill procedure; this is one application of Algorithm 1 with the
+// whole prompt as the cache G_i: the last Rw = min(R, P) prompt tokens are the window, each
+// window row's attention profile is its causal soft-max over all prompt keys (Eq. 1), every
+// older prompt token gets the fused score of Eq. 4-6 (group sum first), and the C best are
+// kept beside the window (Eq. 7).  The selection is a block-wide radix select over
+// (score, position) keys, so ties keep the lower position deterministically.
+#include "mkv_common.cuh"
+#include "mkv_kernels.h"
+
+namespace mkv {
+
+namespace {
+
+constexpr int kPT = 256;    // threads per CTA
+constexpr int kPK = 32;     // keys per tile
+constexpr int kPR = 64;     // window rows per sub-block
+
+__device__ __forceinline__ void ld4(const float *p, float (&o)[4])
+{
+    const float4 v = *reinterpret_cast<const float4 *>(p);
+    o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+}
+__device__ __forceinline__ void ld4(const __nv_bfloat16 *p, float (&o)[4])
+{
+    const uint2 v = *reinterpret_cast<const uint2 *>(p);
+    o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+    o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+
+__global__ void init_arena_kernel(DecodeArgs a)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t ncap = (size_t)a.U * a.cap;
+    if (i < ncap) { a.pos[i] = -1; a.F[i] = 0.f; }
+    if (i < (size_t)a.U * a.R * a.G) a.ring_c[i] = INFINITY;   // empty ring row: weight 0
+    if (i < (size_t)a.U) { a.ticket[i] = 0; a.evicted_pos[i] = -1; }
+}
+
+__global__ void set_state_kernel(DevState *st, long long t, int n)
+{
+    st->t = t; st->n = n; st->steps = 0; st->err = 0; st->done = 0; st->pad = 0;
+}
+
+// S[ub][row = i*G + g][j] = log2-domain logit of window row (i, g) against prompt key j,
+// -inf where j lies after the row's own position (causal mask).
+template <typename T, int D>
+__global__ void __launch_bounds__(kPT) prefill_logits_kernel(const T *__restrict__ k, const T *__restrict__ qwin,
+                                                             float *__restrict__ S, int ub0, int P, int Rw, int G,
+                                                             float scale2)
+{
+    extern __shared__ __align__(16) float psm[];
+    float *Ks = psm, *Qs = psm + kPK * (D + 4), *Ssm = Qs + kPR * (D + 4);
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int u = ub0 + blockIdx.y, kt = blockIdx.x * kPK;
+    const int rows = Rw * G;
+    constexpr int KS = D + 4, C4 = D / 4;
+    const T *Ku = k + (size_t)u * P * D;
+    for (int idx = tid; idx < kPK * C4; idx += kPT) {
+        const int key = idx / C4, c4 = idx % C4;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (kt + key < P) ld4(Ku + (size_t)(kt + key) * D + c4 * 4, v);
+        *reinterpret_cast<float4 *>(Ks + key * KS + c4 * 4) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    for (int r0 = 0; r0 < rows; r0 += kPR) {
+        const int nr = min(kPR, rows - r0);
+        __syncthreads();
+        for (int idx = tid; idx < nr * C4; idx += kPT) {
+            const int rl = idx / C4, c4 = idx % C4;
+            const int row = r0 + rl, i = row / G, g = row % G;
+            float v[4];
+            ld4(qwin + (((size_t)u * G + g) * Rw + i) * D + c4 * 4, v);
+            *reinterpret_cast<float4 *>(Qs + rl * KS + c4 * 4) = make_float4(v[0], v[1], v[2], v[3]);
+        }
+        __syncthreads();
+        float acc[2][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { acc[0][i] = 0.f; acc[1][i] = 0.f; }
+        const float *ka = Ks + ty * KS, *kb = Ks + (ty + 16) * KS;
+        const float *qr[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) qr[i] = Qs + ((tx + 16 * i) < nr ? (tx + 16 * i) : 0) * KS;
+#pragma unroll 4
+        for (int dd = 0; dd < D; dd += 4) {
+            const float4 x = *reinterpret_cast<const float4 *>(ka + dd);
+            const float4 y = *reinterpret_cast<const float4 *>(kb + dd);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 qv = *reinterpret_cast<const float4 *>(qr[i] + dd);
+                acc[0][i] += x.x * qv.x + x.y * qv.y + x.z * qv.z + x.w * qv.w;
+                acc[1][i] += y.x * qv.x + y.y * qv.y + y.z * qv.z + y.w * qv.w;
+            }
+        }
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) Ssm[(ty + 16 * kk) * (kPR + 1) + tx + 16 * i] = acc[kk][i] * scale2;
+        __syncthreads();
+        for (int idx = tid; idx < nr * kPK; idx += kPT) {
+            const int rl = idx / kPK, key = idx % kPK;
+            const int j = kt + key;
+            if (j >= P) continue;
+            const int row = r0 + rl;
+            const int rpos = P - Rw + row / G;           // absolute position of the window row
+            S[((size_t)blockIdx.y * rows + row) * P + j] = (j <= rpos) ? Ssm[key * (kPR + 1) + rl] : -INFINITY;
+        }
+    }
+}
+
+// c = max + log2(sum exp2(s - max)) of one window row; stored in the ring row p % R.
+__global__ void __launch_bounds__(kPT) prefill_rowstats_kernel(const float *__restrict__ S, float *__restrict__ ring_c,
+                                                               int ub0, int P, int Rw, int G, int R)
+{
+    __shared__ float red[kPT / 32];
+    __shared__ float bc;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row = blockIdx.x, u = ub0 + blockIdx.y;
+    const float *s = S + ((size_t)blockIdx.y * Rw * G + row) * P;
+    float m = -INFINITY;
+    for (int j = tid; j < P; j += kPT) m = fmaxf(m, s[j]);
+    m = warp_max(m);
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (tid == 0) { float x = red[0]; for (int w = 1; w < kPT / 32; ++w) x = fmaxf(x, red[w]); bc = x; }
+    __syncthreads();
+    m = bc;
+    float l = 0.f;
+    for (int j = tid; j < P; j += kPT) l += exp2f(s[j] - m);
+    l = warp_sum(l);
+    __syncthreads();
+    if (lane == 0) red[warp] = l;
+    __syncthreads();
+    if (tid == 0) {
+        float x = 0.f;
+        for (int w = 0; w < kPT / 32; ++w) x += red[w];
+        const int i = row / G, g = row % G;
+        const int rslot = (P - Rw + i) % R;
+        ring_c[((size_t)u * R + rslot) * G + g] = m + log2f(x);
+    }
+}
+
+// Eq. 4-6 with Algorithm 1's group sum: F[j] for every older prompt token j < P - Rw.
+__global__ void __launch_bounds__(kPT) prefill_fuse_kernel(const float *__restrict__ S, const float *__restrict__ ring_c,
+                                                           float *__restrict__ Fp, int ub0, int P, int Rw, int G, int R,
+                                                           int fusion)
+{
+    extern __shared__ float cs[];   // [Rw * G]
+    const int u = ub0 + blockIdx.y, rows = Rw * G;
+    for (int row = threadIdx.x; row < rows; row += kPT) {
+        const int rslot = (P - Rw + row / G) % R;
+        cs[row] = ring_c[((size_t)u * R + rslot) * G + row % G];
+    }
+    __syncthreads();
+    const int j = blockIdx.x * kPT + threadIdx.x;
+    if (j >= P - Rw) return;
+    const float *s = S + (size_t)blockIdx.y * rows * P + j;
+    float F = 0.f;
+    for (int i = 0; i < Rw; ++i) {
+        float Sr = 0.f;
+        for (int g = 0; g < G; ++g) Sr += exp2f(s[(size_t)(i * G + g) * P] - cs[i * G + g]);
+        F = fuse(fusion, F, Sr);
+    }
+    Fp[(size_t)blockIdx.y * P + j] = F;
+}
+
+// Top-C of the M = P - Rw older tokens by (F descending, position ascending): an 8-pass
+// radix select finds the C-th best 64-bit rank key, then an order-preserving compaction
+// lists the kept positions, followed by the window positions.
+__global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__restrict__ Fp, int *__restrict__ pos, int ub0,
+                                                             int P, int Rw, int C, int cap)
+{
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long prefix_s;
+    __shared__ int remaining_s;
+    __shared__ int wtot[kPT / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int u = ub0 + blockIdx.x, M = P - Rw;
+    const float *F = Fp + (size_t)blockIdx.x * P;
+    int *upos = pos + (size_t)u * cap;
+    unsigned long long prefix = 0;
+    int remaining = C;
+    for (int pass = 7; pass >= 0; --pass) {
+        for (int i = tid; i < 256; i += kPT) hist[i] = 0;
+        __syncthreads();
+        const int shift = 8 * pass;
+        for (int j = tid; j < M; j += kPT) {
+            const unsigned long long key = rank_key(__float_as_uint(F[j]), j);
+            if (pass == 7 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int acc = 0, b = 255;
+            for (; b > 0; --b) {
+                if (acc + (int)hist[b] >= remaining) break;
+                acc += (int)hist[b];
+            }
+            remaining_s = remaining - acc;
+            prefix_s = (prefix << 8) | (unsigned long long)b;
+        }
+        __syncthreads();
+        prefix = prefix_s;
+        remaining = remaining_s;
+        __syncthreads();
+    }
+    int base = 0;
+    for (int c0 = 0; c0 < M; c0 += kPT) {
+        const int j = c0 + tid;
+        const bool keep = j < M && rank_key(__float_as_uint(F[j]), j) >= prefix;
+        const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) wtot[warp] = __popc(bal);
+        __syncthreads();
+        int off = base;
+        for (int w = 0; w < warp; ++w) off += wtot[w];
+        if (keep) upos[off + __popc(bal & ((1u << lane) - 1u))] = j;
+        for (int w = 0; w < kPT / 32; ++w) base += wtot[w];
+        __syncthreads();
+    }
+    for (int i = tid; i < Rw; i += kPT) upos[C + i] = M + i;
+}
+
+__global__ void prefill_identity_pos_kernel(int *pos, int U, int n, int cap)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)U * n) return;
+    pos[(i / n) * cap + (i % n)] = (int)(i % n);
+}
+
+// K/V rows of the kept prompt positions into the arena, 16 bytes per thread.
+template <typename T, int D>
+__global__ void prefill_gather_kernel(const T *__restrict__ k, const T *__restrict__ v, DecodeArgs a, int P, int n)
+{
+    constexpr int CH = D * sizeof(T) / 16;
+    const int u = blockIdx.x;
+    const int idx = blockIdx.y * blockDim.x + threadIdx.x;
+    if (idx >= n * CH) return;
+    const int slot = idx / CH, c = idx % CH;
+    const int p = a.pos[(size_t)u * a.cap + slot];
+    const uint4 *ks = reinterpret_cast<const uint4 *>(k + ((size_t)u * P + p) * D) + c;
+    const uint4 *vs = reinterpret_cast<const uint4 *>(v + ((size_t)u * P + p) * D) + c;
+    reinterpret_cast<uint4 *>(static_cast<T *>(a.K) + ((size_t)u * a.cap + slot) * D)[c] = *ks;
+    reinterpret_cast<uint4 *>(static_cast<T *>(a.V) + ((size_t)u * a.cap + slot) * D)[c] = *vs;
+}
+
+// window queries into their ring rows (row p % R)
+template <typename T, int D>
+__global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, int P, int Rw)
+{
+    const int u = blockIdx.x, G = a.G;
+    T *rq = static_cast<T *>(a.ring_q) + (size_t)u * a.R * G * D;
+    for (int idx = threadIdx.x; idx < Rw * G * D; idx += blockDim.x) {
+        const int dd = idx % D, g = (idx / D) % G, i = idx / (D * G);
+        const int rslot = (P - Rw + i) % a.R;
+        rq[((size_t)rslot * G + g) * D + dd] = qwin[(((size_t)u * G + g) * Rw + i) * D + dd];
+    }
+}
+
+template <typename T, int D>
+cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
+                          unsigned long long *launches)
+{
+    const int U = a.U, G = a.G, R = a.R, C = a.C;
+    const int Rw = P < R ? P : R, rows = Rw * G;
+    const bool select = P - Rw > C;
+    const int n = select ? C + Rw : P;
+    if (n > a.cap) return cudaErrorInvalidValue;
+
+    const size_t per_unit = ((size_t)rows * P + P) * sizeof(float);
+    size_t ub = ((size_t)1 << 30) / per_unit;
+    if (ub < 1) ub = 1;
+    if (ub > (size_t)U) ub = U;
+    if (ub > 65535) ub = 65535;
+    float *S = nullptr;
+    cudaError_t e = cudaMalloc(&S, ub * per_unit);
+    if (e != cudaSuccess) return e;
+    float *Fp = S + ub * (size_t)rows * P;
+
+    const size_t logits_smem = (size_t)(kPK * (D + 4) + kPR * (D + 4) + kPK * (kPR + 1)) * sizeof(float);
+    e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
+    if (e != cudaSuccess) { cudaFree(S); return e; }
+    const size_t init_n = max((size_t)U * a.cap, (size_t)U * R * G);
+    init_arena_kernel<<<(unsigned)((init_n + 255) / 256), 256, 0, stream>>>(a);
+    ++*launches;
+    for (int ub0 = 0; ub0 < U; ub0 += (int)ub) {
+        const int nb = min((int)ub, U - ub0);
+        prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw, G,
+                                                                                             a.scale2);
+        prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, G, R);
+        *launches += 2;
+        if (select) {
+            prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
+                S, a.ring_c, Fp, ub0, P, Rw, G, R, a.fusion);
+            prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
+            *launches += 2;
+        }
+    }
+    if (!select) {
+        prefill_identity_pos_kernel<<<(unsigned)(((size_t)U * n + 255) / 256), 256, 0, stream>>>(a.pos, U, n, a.cap);
+        ++*launches;
+    }
+    constexpr int CH = D * sizeof(T) / 16;
+    prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
+    prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
+    set_state_kernel<<<1, 1, 0, stream>>>(a.st, (long long)P, n);
+    *launches += 3;
+    e = cudaGetLastError();
+    const cudaError_t e2 = cudaStreamSynchronize(stream);
+    cudaFree(S);
+    return e != cudaSuccess ? e : e2;
+}
+
+}  // namespace
+
+cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
+                        cudaStream_t stream, unsigned long long *launches)
+{
+    if (f32) {
+        auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
+        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches)
+                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches);
+    }
+    auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
+         qq = static_cast<const __nv_bfloat16 *>(q_window);
+    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches)
+                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches);
+}
+
+}  // namespace mkv

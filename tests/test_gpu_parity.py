@@ -1,0 +1,163 @@
+"""Parity of the CUDA decode path (called through the C ABI) with the CPU oracle, step by step."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2503_00979_b200 import binding, synth
+from tests.parity import run_parity
+
+pytestmark = pytest.mark.gpu
+
+SMALL = synth.Workload("small", 2, 2, 8, 2, 128, "bf16", 300, 96, 200, 16, "sum", 777)
+
+
+def _report(rep):
+    print(f"\n[parity] kernel={rep.kernel} steps={rep.steps} unit_steps={rep.unit_steps} max_out_err={rep.max_out_err:.3e} "
+          f"evictions={rep.evictions} near_tie_resyncs={rep.near_tie_resyncs} max_F_rel_err={rep.max_F_rel_err:.3e} "
+          f"(F compared {rep.F_compared}) prefill_dropped={rep.prefill_dropped}")
+
+
+@pytest.mark.parametrize("seed_off", [0, 100, 200])
+def test_config0_every_unit_every_step(seed_off):
+    w = synth.WORKLOADS["c0"]
+    rep = run_parity(w.replace(seed=w.seed + seed_off), steps=w.steps, n_units=w.units, chunk=128)
+    _report(rep)
+    assert rep.unit_steps == (w.units - rep.prefill_dropped) * w.steps and rep.evictions > 0
+    assert rep.near_tie_resyncs <= 0.01 * rep.evictions + 2
+
+
+@pytest.mark.parametrize("fusion", ["sum", "max"])
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("bf16", 64), ("f32", 128), ("f32", 64)])
+def test_small_shapes_simt(fusion, dtype, d):
+    w = SMALL.replace(fusion=fusion, dtype=dtype, head_dim=d)
+    rep = run_parity(w, steps=w.steps, n_units=8, kernel="simt")
+    _report(rep)
+    assert rep.evictions > 0 and rep.F_compared > 0
+
+
+@pytest.mark.parametrize("G,R,C,P", [(1, 8, 100, 150), (7, 12, 90, 133), (4, 32, 2000 - 1, 2100), (16, 4, 33, 80),
+                                     (2, 1, 50, 70), (4, 40, 217, 250)])
+def test_group_sizes_windows_and_ragged_tails(G, R, C, P):
+    # G = 1 is MHA, G = 7 the Qwen ratio; cache sizes that are no multiple of any tile
+    w = SMALL.replace(layers=1, batch=2, n_q_heads=2 * G, n_kv_heads=2, R=R, C=C, prompt_len=P, steps=48, fusion="max")
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel="simt")
+    _report(rep)
+    assert rep.evictions > 0
+
+
+@pytest.mark.parametrize("splits", [1, 2, 5])
+def test_split_counts_give_the_same_answer(splits):
+    w = SMALL.replace(layers=1, C=500, prompt_len=700, steps=40)
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel="simt", splits=splits)
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_no_eviction_regime_is_full_attention():
+    # C + R >= P + S: the oracle equals plain causal attention here (pinned on the CPU side)
+    w = SMALL.replace(C=400, R=16, prompt_len=100, steps=64)
+    rep = run_parity(w, steps=w.steps, n_units=8)
+    _report(rep)
+    assert rep.evictions == 0
+
+
+def test_fill_phase_then_eviction_starts():
+    w = SMALL.replace(C=120, R=16, prompt_len=100, steps=80)      # fills 36 steps, then evicts
+    rep = run_parity(w, steps=w.steps, n_units=8)
+    _report(rep)
+    assert rep.evictions == 8 * (80 - 36)
+
+
+def test_prompt_shorter_than_the_window():
+    w = SMALL.replace(C=20, R=16, prompt_len=5, steps=60, layers=1)
+    rep = run_parity(w, steps=w.steps, n_units=4)
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_single_token_prompt():
+    w = SMALL.replace(C=6, R=3, prompt_len=1, steps=30, layers=1)
+    rep = run_parity(w, steps=w.steps, n_units=4)
+    _report(rep)
+
+
+def test_attention_sink_workload():
+    w = synth.WORKLOADS["c2"].replace(layers=1, batch=2, prompt_len=600, C=256, steps=64)
+    rep = run_parity(w, steps=w.steps, n_units=8)
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_decode_steps_call_and_host_call():
+    w = SMALL.replace(layers=1, steps=32)
+    rep = run_parity(w, steps=w.steps, n_units=4, use_steps_call=True)
+    _report(rep)
+    rep = run_parity(w, steps=w.steps, n_units=4, host_call_every=3)
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_state_order_and_argument_errors():
+    mk = binding.MorphKV(1, 1, 8, 2, 64, 16, 4, "sum", "f32")
+    q = torch.zeros(1, 1, 8, 64, device="cuda")
+    kv = torch.zeros(1, 1, 2, 64, device="cuda")
+    assert binding.mkv_decode_step(mk.ctx, q, kv, kv, q) == binding.BAD_STATE
+    assert "prefill" in binding.mkv_last_error(mk.ctx)
+    assert binding.mkv_prefill(mk.ctx, None, None, None, 4) == binding.INVALID_ARG
+    k = torch.randn(1, 1, 2, 5, 64, device="cuda")
+    qw = torch.randn(1, 1, 8, 4, 64, device="cuda")
+    assert binding.mkv_prefill(mk.ctx, k, k, qw, 0) == binding.INVALID_ARG
+    mk.prefill(k, k, qw)
+    assert binding.mkv_prefill(mk.ctx, k, k, qw, 5) == binding.BAD_STATE
+    assert binding.mkv_decode_step(mk.ctx, q, kv, None, q) == binding.INVALID_ARG
+    st, v = binding.mkv_cache_view(mk.ctx, 3)
+    assert st == binding.INVALID_ARG
+    mk.decode_step(q, kv, kv)
+    mk.sync()
+    assert mk.view(0)["count"] == 6 and mk.view(0)["next_pos"] == 6 and mk.launch_count > 0
+    mk.close()
+
+
+def test_workspace_too_small_is_oom():
+    p = binding.mkv_default_params()
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 8, 2, 64, 16, 4
+    buf = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    p.workspace, p.workspace_bytes = (buf.data_ptr() + 255) & ~255, 1024
+    st, h = binding.mkv_create_ex(p)
+    assert st == binding.OOM and h is None
+    p.workspace = ((buf.data_ptr() + 255) & ~255) + 8       # misaligned
+    st, h = binding.mkv_create_ex(p)
+    assert st == binding.INVALID_ARG
+
+
+def test_slot_permutation_does_not_change_results():
+    # physical slot order is free: swapping two cached rows (K, V, pos together) changes nothing
+    w = SMALL.replace(layers=1, batch=1, steps=8)
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    k, v = st.kv(np.arange(w.prompt_len))
+    qw = st.q(np.arange(w.prompt_len - w.R, w.prompt_len))
+    outs = []
+    for swap in (False, True):
+        mk = binding.MorphKV(1, 1, 8, 2, 128, w.C, w.R, w.fusion, "bf16")
+        mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+        mk.sync()
+        if swap:
+            vw = mk.view(0)
+            perm = torch.randperm(vw["count"], device=dev)
+            for name in ("K", "V", "pos"):
+                t = vw[name]
+                t[:, :, :vw["count"]] = t[:, :, :vw["count"]][:, :, perm].clone()
+        res = []
+        for i in range(w.steps):
+            p = [w.prompt_len + i]
+            kk, vv = st.kv(p)
+            o = mk.decode_step(st.q(p)[:, :, :, 0].bfloat16().contiguous(), kk[:, :, :, 0].bfloat16().contiguous(),
+                               vv[:, :, :, 0].bfloat16().contiguous())
+            res.append(o.float())
+        mk.sync()
+        vw = mk.view(0)
+        outs.append((torch.stack(res), torch.sort(vw["pos"][0, :, :vw["count"]], dim=-1).values.clone()))
+        mk.close()
+    assert torch.equal(outs[0][1], outs[1][1])
+    assert (outs[0][0] - outs[1][0]).abs().max() < 2e-2
