@@ -1,0 +1,307 @@
+#!/usr/bin/env python
+"""Benchmark of the MorphKV decode + update hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1] [--impl ours|reference]
+
+A *step* is one decode step (attend, score, select, update) of every unit of the workload.
+The default workload is the Llama-3.1-8B-shaped attention stack (32 layers, 32/8 heads,
+d = 128, bf16, batch 1, 4096-token prompt, C = 2000, R = 32, max fusion) in steady state:
+the cache is full after the prompt, so every timed step evicts one token per unit.
+
+With N > 1 (under torchrun) every rank runs its own replica of the workload on its own GPU
+with a different seed: units share nothing, so there is no collective on the data path.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_00979_b200 import synth  # noqa: E402
+
+METRIC, UNIT = "decode_tokens_per_s", "tokens/s"
+
+
+def algorithmic_bytes_per_step(w: synth.Workload, n: int) -> int:
+    """K and V of the n cached tokens read once plus the R*G recent queries, per unit."""
+    e = 2 if w.dtype == "bf16" else 4
+    return w.units * (2 * n * w.head_dim * e + w.R * w.group * w.head_dim * e)
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, an earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_throughput(w: synth.Workload, n_units: int, steps: int, warm: int = 2):
+    """Times the CPU oracle as it stands on `n_units` units (one thread each) for `steps` steady-state
+    decode steps.  Returns (unit-steps per second, threads used, description of the sample)."""
+    from oracle import morphkv_oracle as ora
+    ora.build()
+    G, d, P = w.group, w.head_dim, w.prompt_len
+    Rw = min(w.R, P)
+    st = synth.Stream(w, "cpu")
+    units = [(i % w.layers, (i // w.layers) % w.batch, (i // (w.layers * w.batch)) % w.n_kv_heads) for i in range(n_units)]
+    pos = np.arange(P, P + warm + steps)
+    work = []
+    for (l, b, h) in units:
+        k, v = st.kv(np.arange(P), [l], [b], [h])
+        qw = st.q(np.arange(P - Rw, P), [l], [b], [h])
+        u = ora.Unit(G, d, w.C, w.R, w.fusion)
+        u.prefill(k[0, 0, 0].double().numpy(), v[0, 0, 0].double().numpy(), qw[0, 0].double().numpy())
+        kk, vv = st.kv(pos, [l], [b], [h])
+        qq = st.q(pos, [l], [b], [h])
+        work.append((u, qq[0, 0].double().numpy(), kk[0, 0, 0].double().numpy(), vv[0, 0, 0].double().numpy()))
+
+    def run(item, lo, hi):
+        u, q, k, v = item
+        for i in range(lo, hi):
+            u.step(np.ascontiguousarray(q[:, i]), k[i], v[i])
+
+    for item in work:
+        run(item, 0, warm)
+    threads = [threading.Thread(target=run, args=(item, warm, warm + steps)) for item in work]
+    t0 = time.perf_counter()
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    dt = time.perf_counter() - t0
+    sample = (f"{n_units} units x {steps} steady-state steps of {w.name} (stored-profile fp64 oracle, one thread per "
+              f"unit), scaled by batch/units")
+    return n_units * steps / dt, n_units, sample, dt
+
+
+def run_reference(args, w):
+    """The oracle arm: each step is one decode step of a bounded sample of units."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    n_units = max(1, min(cores, w.units))
+    ups, used, sample, dt = oracle_throughput(w, n_units, args.steps, warm=args.warmup)
+    tok = ups * w.batch / w.units
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tok, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
+                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "C": w.C, "R": w.R, "fusion": w.fusion,
+                   "prompt_len": w.prompt_len},
+        "cpu_baseline": {"value": tok, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tok, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w):
+    import torch.distributed as dist
+    from paper_2503_00979_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    w = w.replace(seed=w.seed + 1000 * rank)       # every rank its own replica (different batch content)
+    tdt = synth.torch_dtype(w.dtype)
+    K, W = args.steps, args.warmup
+    P, Rw = w.prompt_len, min(w.R, w.prompt_len)
+
+    st = synth.Stream(w, dev)
+    mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
+                         kernel=args.kernel, splits=args.splits, device=str(dev))
+    # prompt phase (untimed), drawn layer by layer to bound the temporary memory
+    ks, vs, qws = [], [], []
+    for l in range(w.layers):
+        k, v = st.kv(np.arange(P), [l])
+        ks.append(k.to(tdt)); vs.append(v.to(tdt))
+        qws.append(st.q(np.arange(P - Rw, P), [l]).to(tdt))
+    k, v, qw = torch.cat(ks), torch.cat(vs), torch.cat(qws)
+    del ks, vs, qws
+    mk.prefill(k.contiguous(), v.contiguous(), qw.contiguous())
+    del k, v, qw
+    n0 = mk.view(0)["count"]
+
+    total = 2 * (W + K)                            # device-resident arm, then host-buffer arm
+    pos = np.arange(P, P + total)
+    kk, vv = st.kv(pos)
+    qs = st.q(pos).permute(3, 0, 1, 2, 4).to(tdt).contiguous()       # [steps,L,B,Hq,d]
+    kn = kk.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+    vn = vv.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+    del kk, vv
+    outs = torch.empty_like(qs[:W + K])
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- arm 1: inputs resident in HBM ----
+    mk.decode_steps(qs[:W], kn[:W], vn[:W], outs[:W])
+    mk.sync()
+    n_steady = mk.view(0)["count"]
+    launches0 = mk.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local) as clocks:
+        e0.record(stream)
+        mk.decode_steps(qs[W:W + K], kn[W:W + K], vn[W:W + K], outs[W:W + K])
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    launches = mk.launch_count - launches0
+    mk.sync()
+    barrier()
+
+    # ---- arm 2: host buffers through the C ABI, copies inside the timed region ----
+    hq = qs[W + K:].cpu().pin_memory(); hk = kn[W + K:].cpu().pin_memory(); hv = vn[W + K:].cpu().pin_memory()
+    ho = torch.empty_like(hq).pin_memory()
+    for i in range(W):
+        mk.decode_step_host(hq[i], hk[i], hv[i], ho[i])
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    for i in range(W, W + K):
+        mk.decode_step_host(hq[i], hk[i], hv[i], ho[i])
+    e3.record(stream)
+    torch.cuda.synchronize()
+    ms_e2e = e2.elapsed_time(e3)
+    mk.sync()
+    checksum = float(ho[W:].float().abs().mean())
+    assert np.isfinite(checksum)
+
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+    if rank == 0:
+        bytes_step = algorithmic_bytes_per_step(w, n_steady)
+        peak, peak_src = measured_peak_gbs()
+        achieved = bytes_step / (ms / K * 1e-3) / 1e9
+        e = 2 if w.dtype == "bf16" else 4
+        h2d = (w.units * w.group + 2 * w.units) * w.head_dim * e
+        d2h = w.units * w.group * w.head_dim * e
+        line = {
+            "metric": METRIC, "value": world * w.batch * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
+                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "C": w.C, "R": w.R, "fusion": w.fusion,
+                       "prompt_len": P, "cached_tokens_per_unit": n_steady, "units_per_gpu": w.units,
+                       "kernel": mk.kernel_name, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2: each step streams the whole K/V cache "
+                             f"({bytes_step / 1e6:.0f} MB per step against 126 MB of L2)"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": world * w.batch * K / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": peak_src, "kernel": f"decode_{mk.kernel_name}",
+                         "algorithmic_bytes_per_launch": bytes_step},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            cores = len(os.sched_getaffinity(0))
+            n_units = max(1, min(cores, w.units))
+            ups, used, sample, _ = oracle_throughput(synth.WORKLOADS[args.workload], n_units, args.cpu_steps)
+            line["cpu_baseline"] = {"value": ups * w.batch / w.units, "unit": UNIT, "cores": used, "kind": "oracle",
+                                    "sample": sample, "unit_steps_per_s": ups}
+        print(json.dumps(line), flush=True)
+    mk.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c1", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--cpu-steps", type=int, default=512, help="steady-state steps per unit for the CPU baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
