@@ -119,6 +119,28 @@ void mkv_destroy(mkv_ctx *ctx);
 mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
                        int prompt_len, void *stream);
 
+/* mkv_prefill for callers that must not allocate (the paper has no counterpart: this is an
+ * integration aid, not part of the method).  Some hosts of this library cannot let it call
+ * cudaMalloc: a serving engine that has already handed all of HBM to its own pool, where a
+ * further allocation fails or fragments; and latency-critical threads, for which the
+ * device-wide synchronisation inside cudaMalloc/cudaFree stalls every other stream.  Give
+ * the context a caller-owned workspace (mkv_create_ex) and use this call instead of
+ * mkv_prefill: same arguments, same result, but the temporary table of window-row logits
+ * lives in a fixed 16 MiB device array that is part of the library image (every GPU that
+ * loads the library holds those 16 MiB until the process exits).
+ *   - Limit: (min(R, prompt_len) * G + 1) * prompt_len <= 4 Mi floats for one unit;
+ *     beyond that it returns MKV_UNSUPPORTED with an explanatory mkv_last_error and does
+ *     nothing.  Units are pushed through the array a few at a time.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device looks up the array's device address (once per device,
+ *     with that device current); make that first call outside any stream capture.
+ *   - All contexts and calls share the one array.  Nothing in it has to start at zero (every
+ *     element is written before it is read within a call), but two calls whose kernels
+ *     overlap on the GPU (different streams or threads) race on it: serialise them.
+ * Synchronises the stream before returning, like mkv_prefill. */
+mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
+                              int prompt_len, void *stream);
+
 /* One decode step for every unit (Eq. 1, Eq. 4-7, Algorithm 1): q, out
  * [layers][batch][n_q_heads][head_dim]; k_new, v_new [layers][batch][n_kv_heads][head_dim].
  * Asynchronous; launches a fixed kernel sequence with no host-side dependence on the step

@@ -25,6 +25,7 @@ KERNEL = {"auto": 0, "simt": 1, "tc": 2}
 
 EXPORTS = [
     "mkv_default_params", "mkv_workspace_bytes", "mkv_create", "mkv_create_ex", "mkv_destroy", "mkv_prefill",
+    "mkv_prefill_static",
     "mkv_decode_step", "mkv_decode_steps", "mkv_decode_step_host", "mkv_cache_view", "mkv_sync", "mkv_last_error",
     "mkv_launch_count", "mkv_kernel_name",
 ]
@@ -74,6 +75,7 @@ def lib() -> C.CDLL:
         L.mkv_destroy.argtypes = [vp]
         L.mkv_destroy.restype = None
         L.mkv_prefill.argtypes = [vp, vp, vp, vp, ip, vp]
+        L.mkv_prefill_static.argtypes = [vp, vp, vp, vp, ip, vp]
         L.mkv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
         L.mkv_decode_steps.argtypes = [vp, vp, vp, vp, vp, ip, vp]
         L.mkv_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -132,6 +134,11 @@ def mkv_destroy(ctx) -> None:
 
 def mkv_prefill(ctx, k, v, q_window, prompt_len, stream=None) -> int:
     return lib().mkv_prefill(ctx, _ptr(k), _ptr(v), _ptr(q_window), prompt_len, _stream(stream))
+
+
+def mkv_prefill_static(ctx, k, v, q_window, prompt_len, stream=None) -> int:
+    """mkv_prefill without any device allocation (scratch in the library's fixed 16 MiB array)."""
+    return lib().mkv_prefill_static(ctx, _ptr(k), _ptr(v), _ptr(q_window), prompt_len, _stream(stream))
 
 
 def mkv_decode_step(ctx, q, k_new, v_new, out, stream=None) -> int:
@@ -231,6 +238,10 @@ class MorphKV:
 
     def prefill(self, k, v, q_window, stream=None):
         self._check(mkv_prefill(self.ctx, k, v, q_window, k.shape[-2], stream), "mkv_prefill")
+
+    def prefill_static(self, k, v, q_window, stream=None):
+        """Prompt phase for hosts that cannot allocate device memory; see mkv_prefill_static in mkv.h."""
+        self._check(mkv_prefill_static(self.ctx, k, v, q_window, k.shape[-2], stream), "mkv_prefill_static")
 
     def decode_step(self, q, k_new, v_new, out=None, stream=None):
         if out is None:

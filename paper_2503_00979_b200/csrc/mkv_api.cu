@@ -241,6 +241,30 @@ mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q
     return MKV_OK;
 }
 
+mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, void *stream)
+{
+    if (!ctx) return MKV_INVALID_ARG;
+    if (!k || !v || !q_window) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_static: NULL tensor%s");
+    if (prompt_len < 1 || prompt_len > (1 << 24)) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_static: prompt_len out of range%s");
+    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill_static: context already holds a sequence%s");
+    const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
+    const size_t need = ((size_t)Rw * ctx->s.G + 1) * (size_t)prompt_len;
+    if (need > prefill_static_max_floats()) {
+        snprintf(ctx->err, sizeof(ctx->err),
+                 "mkv_prefill_static: one unit needs (min(R,P)*G + 1) * prompt_len = %zu floats of scratch, the fixed "
+                 "array holds %zu; use mkv_prefill for this prompt", need, prefill_static_max_floats());
+        return MKV_UNSUPPORTED;
+    }
+    const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
+    const cudaError_t e = run_prefill_static(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, k, v, q_window, prompt_len,
+                                             (cudaStream_t)stream, &ctx->launches);
+    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_prefill_static: %s", cudaGetErrorString(e));
+    ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
+    ctx->t = prompt_len;
+    ctx->prefilled = true;
+    return MKV_OK;
+}
+
 mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *out, void *stream)
 {
     if (!ctx) return MKV_INVALID_ARG;

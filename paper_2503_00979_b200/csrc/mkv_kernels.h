@@ -15,4 +15,11 @@ int simt_default_splits(int U, int cap);
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
                         int P, cudaStream_t stream, unsigned long long *launches);
 
+// The same prompt phase with its scratch in a fixed device array of prefill_static_max_floats()
+// floats instead of a temporary allocation; cudaErrorInvalidConfiguration if one unit's
+// (R*G + 1) * P floats do not fit.
+size_t prefill_static_max_floats();
+cudaError_t run_prefill_static(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
+                               int P, cudaStream_t stream, unsigned long long *launches);
+
 }  // namespace mkv

@@ -309,6 +309,88 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     return e != cudaSuccess ? e : e2;
 }
 
+
+// ---- prompt phase without any allocation ---------------------------------------------------
+// Scratch for the logits table S and the fused scores lives in a fixed device array that every
+// GPU loading this library holds until the process exits.  16 MiB: one unit of a 4096-token
+// prompt with R*G = 128 window rows needs 2.1 MB, so the units go through it a few at a time.
+constexpr size_t kStaticScratchFloats = (size_t)4 << 20;
+static __device__ __align__(256) float g_prefill_scratch[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+static float *g_scratch_addr[kMaxDevices];   // device address of the array, per device ordinal
+
+// The array's name is only a host-side handle here; a kernel needs its device address, which
+// the runtime hands out per device.  Looked up once per device, with that device current.
+cudaError_t static_scratch_address(float **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_scratch_addr[dev]) {
+        float *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_prefill_scratch);
+        if (e != cudaSuccess) return e;
+        g_scratch_addr[dev] = ptr;
+    }
+    *out = g_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+template <typename T, int D>
+cudaError_t run_prefill_static_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
+                                 unsigned long long *launches)
+{
+    const int U = a.U, G = a.G, R = a.R, C = a.C;
+    const int Rw = P < R ? P : R, rows = Rw * G;
+    const bool select = P - Rw > C;
+    const int n = select ? C + Rw : P;
+    if (n > a.cap) return cudaErrorInvalidValue;
+    const size_t per_unit = (size_t)rows * P + P;            // floats
+    if (per_unit > kStaticScratchFloats) return cudaErrorInvalidConfiguration;
+    size_t ub = kStaticScratchFloats / per_unit;
+    if (ub > (size_t)U) ub = U;
+    if (ub > 65535) ub = 65535;
+    float *S = nullptr;
+    cudaError_t e = static_scratch_address(&S);
+    if (e != cudaSuccess) return e;
+    // every element of S and Fp that a kernel reads was written earlier in the same batch,
+    // so what an earlier call left in the array never matters and nothing has to be cleared
+    float *Fp = S + ub * (size_t)rows * P;
+    const size_t logits_smem = (size_t)(kPK * (D + 4) + kPR * (D + 4) + kPK * (kPR + 1)) * sizeof(float);
+    e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
+    if (e != cudaSuccess) return e;
+    const size_t init_n = max((size_t)U * a.cap, (size_t)U * R * G);
+    init_arena_kernel<<<(unsigned)((init_n + 255) / 256), 256, 0, stream>>>(a);
+    ++*launches;
+    for (int ub0 = 0; ub0 < U; ub0 += (int)ub) {
+        const int nb = min((int)ub, U - ub0);
+        prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw, G,
+                                                                                             a.scale2);
+        prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, G, R);
+        *launches += 2;
+        if (select) {
+            prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
+                S, a.ring_c, Fp, ub0, P, Rw, G, R, a.fusion);
+            prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
+            *launches += 2;
+        }
+    }
+    if (!select) {
+        prefill_identity_pos_kernel<<<(unsigned)(((size_t)U * n + 255) / 256), 256, 0, stream>>>(a.pos, U, n, a.cap);
+        ++*launches;
+    }
+    constexpr int CH = D * sizeof(T) / 16;
+    prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
+    prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
+    set_state_kernel<<<1, 1, 0, stream>>>(a.st, (long long)P, n);
+    *launches += 3;
+    e = cudaGetLastError();
+    const cudaError_t e2 = cudaStreamSynchronize(stream);
+    return e != cudaSuccess ? e : e2;
+}
+
 }  // namespace
 
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
@@ -323,6 +405,26 @@ cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, con
          qq = static_cast<const __nv_bfloat16 *>(q_window);
     return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches)
                    : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches);
+}
+
+}  // namespace mkv
+
+namespace mkv {
+
+size_t prefill_static_max_floats() { return kStaticScratchFloats; }
+
+cudaError_t run_prefill_static(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
+                               int P, cudaStream_t stream, unsigned long long *launches)
+{
+    if (f32) {
+        auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
+        return D == 64 ? run_prefill_static_t<float, 64>(a, kk, vv, qq, P, stream, launches)
+                       : run_prefill_static_t<float, 128>(a, kk, vv, qq, P, stream, launches);
+    }
+    auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
+         qq = static_cast<const __nv_bfloat16 *>(q_window);
+    return D == 64 ? run_prefill_static_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches)
+                   : run_prefill_static_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches);
 }
 
 }  // namespace mkv
