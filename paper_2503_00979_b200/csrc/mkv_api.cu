@@ -21,7 +21,7 @@ struct Layout {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Shape {
-    int U, G, D, R, C, cap, splits, T;
+    int U, G, D, R, C, cap, splits, T, ipu;
     size_t es;
 };
 
@@ -82,12 +82,26 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     s->cap = p->C + p->R + s->T - 1;
     s->es = p->dtype == MKV_DTYPE_F32 ? 4 : 2;
     if (s->T != 1) return false;
-    if (p->kernel == MKV_KERNEL_TC) return false;
+    const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R);
+    if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
+    if (tc_ok && p->kernel != MKV_KERNEL_SIMT) {
+        *kind = kKindTc;
+        const int ntiles = (s->cap + 127) / 128;
+        const int tpg_max = 32 / s->G < 1 ? 1 : 32 / s->G;
+        const int min_ipu = (ntiles + 2 * tpg_max - 1) / (2 * tpg_max);
+        int ipu = p->splits > 0 ? p->splits : tc_items_per_unit(s->U, s->cap, s->G, 148);
+        if (ipu < min_ipu) ipu = min_ipu;
+        if (ipu > ntiles) ipu = ntiles;
+        s->ipu = ipu;
+        s->splits = 2 * ipu;          // every item leaves one partial per compute group
+        return true;
+    }
     *kind = kKindSimt;
     const int max_splits = (s->cap + 31) / 32;
     int sp = p->splits > 0 ? p->splits : simt_default_splits(s->U, s->cap);
     if (sp > max_splits) sp = max_splits;
     s->splits = sp;
+    s->ipu = 0;
     return true;
 }
 
@@ -98,6 +112,7 @@ struct mkv_ctx {
     Shape s;
     Layout L;
     KernelKind kind;
+    TcPlan *plan;
     char *base;
     bool owns_workspace;
     bool prefilled;
@@ -133,10 +148,21 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     return a;
 }
 
+// Free slots and empty ring rows are read by the kernels as whole tiles (their results are
+// masked afterwards), so they must hold finite numbers: zero K, V and the query ring.
+bool clear_arena(mkv_ctx *c, cudaStream_t stream)
+{
+    const size_t kv = (size_t)c->s.U * c->s.cap * c->s.D * c->s.es, rq = (size_t)c->s.U * c->s.R * c->s.G * c->s.D * c->s.es;
+    return cudaMemsetAsync(c->base + c->L.K, 0, kv, stream) == cudaSuccess &&
+           cudaMemsetAsync(c->base + c->L.V, 0, kv, stream) == cudaSuccess &&
+           cudaMemsetAsync(c->base + c->L.ring_q, 0, rq, stream) == cudaSuccess;
+}
+
 mkv_status launch_step(mkv_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream)
 {
     const DecodeArgs a = make_args(ctx, q, k, v, out);
-    const cudaError_t e = launch_decode_simt(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
+    const cudaError_t e = ctx->kind == kKindTc ? launch_decode_tc(ctx->plan, a, stream)
+                                               : launch_decode_simt(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "decode launch failed: %s", cudaGetErrorString(e));
     ctx->launches += 1;
     const bool ev = step_evicts(ctx->t, ctx->n, ctx->s.R, ctx->s.C);
@@ -202,6 +228,17 @@ mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p)
         c->base = (char *)mem;
         c->owns_workspace = true;
     }
+    if (kind == kKindTc) {
+        const DecodeArgs a = make_args(c, nullptr, nullptr, nullptr, nullptr);
+        char msg[200] = "";
+        const cudaError_t e = tc_plan_create(&c->plan, a, s.ipu, msg, sizeof(msg));
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            if (c->owns_workspace) cudaFree(c->base);
+            delete c;
+            return e == cudaErrorMemoryAllocation ? MKV_OOM : MKV_CUDA;
+        }
+    }
     *out = c;
     return MKV_OK;
 }
@@ -219,6 +256,7 @@ mkv_status mkv_create(mkv_ctx **out, int layers, int batch, int n_q_heads, int n
 void mkv_destroy(mkv_ctx *ctx)
 {
     if (!ctx) return;
+    if (ctx->plan) tc_plan_destroy(ctx->plan);
     if (ctx->owns_workspace && ctx->base) cudaFree(ctx->base);
     delete ctx;
 }
@@ -230,6 +268,7 @@ mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q
     if (prompt_len < 1 || prompt_len > (1 << 24)) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill: prompt_len out of range%s");
     if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill: context already holds a sequence%s");
     const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
+    if (!clear_arena(ctx, (cudaStream_t)stream)) return fail(ctx, MKV_CUDA, "mkv_prefill: clearing the arena failed%s");
     const cudaError_t e = run_prefill(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, k, v, q_window, prompt_len,
                                       (cudaStream_t)stream, &ctx->launches);
     if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(ctx, MKV_OOM, "mkv_prefill: no memory for scratch%s"); }
@@ -256,6 +295,7 @@ mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const 
         return MKV_UNSUPPORTED;
     }
     const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
+    if (!clear_arena(ctx, (cudaStream_t)stream)) return fail(ctx, MKV_CUDA, "mkv_prefill_static: clearing the arena failed%s");
     const cudaError_t e = run_prefill_static(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, k, v, q_window, prompt_len,
                                              (cudaStream_t)stream, &ctx->launches);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_prefill_static: %s", cudaGetErrorString(e));

@@ -97,13 +97,22 @@ __host__ __device__ inline bool step_evicts(long long t, int n, int R, int C)
 
 constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32;
 
-// Per-unit epilogue, run by the whole CTA that finished a unit last.  Data written by other
-// CTAs is read with ld.global.cg so that no stale L1 line can be used.  `sm` needs
-// kFinalizeSmemFloats floats of shared memory, 8-byte aligned.
-template <typename T, int D>
-__device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, int active, bool evict, float *sm)
+// barrier over the `nthr` threads that run an epilogue together (id 0 with the whole CTA is
+// __syncthreads; warp-specialised kernels give each compute group its own id)
+__device__ __forceinline__ void group_sync(int bar_id, int nthr)
 {
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthr) : "memory");
+}
+
+// Per-unit epilogue, run by the group of threads that finished a unit last (`tid` in
+// [0, nthr), nthr a multiple of 32, all of them synchronising on barrier `bar_id`).  Data
+// written by other CTAs is read with ld.global.cg so that no stale L1 line can be used.
+// `sm` needs kFinalizeSmemFloats floats of shared memory, 8-byte aligned.
+template <typename T, int D>
+__device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, int active, bool evict, float *sm,
+                              int tid, int nthr, int bar_id)
+{
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const int G = a.G;
     float *s_self = sm, *mfin = sm + kMaxGroup, *lfin = sm + 2 * kMaxGroup, *cnew = sm + 3 * kMaxGroup;
     unsigned long long *red_key = reinterpret_cast<unsigned long long *>(sm + 4 * kMaxGroup);  // [32]
@@ -122,7 +131,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         acc = warp_sum(acc);
         if (lane == 0) s_self[g] = acc * a.scale2;
     }
-    __syncthreads();
+    group_sync(bar_id, nthr);
     if (tid < G) {
         float m = s_self[tid];
         for (int sp = 0; sp < active; ++sp) m = fmaxf(m, __ldcg(pml + (sp * G + tid) * 2));
@@ -133,12 +142,13 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         lfin[tid] = l;
         cnew[tid] = m + log2f(l);
     }
-    __syncthreads();
+    group_sync(bar_id, nthr);
     T *out = static_cast<T *>(a.out) + (size_t)u * G * D;
     for (int idx = tid; idx < G * D; idx += nthr) {
         const int g = idx / D, dd = idx % D;
         const float m = mfin[g];
         float o = exp2f(s_self[g] - m) * ldf(vn + dd);
+#pragma unroll 4
         for (int sp = 0; sp < active; ++sp)
             o += __ldcg(po + (sp * G + g) * D + dd) * exp2f(__ldcg(pml + (sp * G + g) * 2) - m);
         stf(out + idx, o / lfin[g]);
@@ -153,17 +163,38 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         const long long thr = t - a.R;
         unsigned long long best = ~0ull;
         int bslot = -1;
-        for (int k = tid; k < n; k += nthr) {
-            const int p = pos[k];
-            if ((long long)p <= thr) {
-                float s = 0.f;
-                for (int g = 0; g < G; ++g) s += exp2f(__ldcg(sn + (size_t)g * a.cap + k) - cnew[g]);
-                const float f = fuse(a.fusion, __ldcg(F + k), s);
-                F[k] = f;
-                const unsigned long long key = rank_key(__float_as_uint(f), p);
-                if (key < best) { best = key; bslot = k; }
-            } else {
-                F[k] = -1.f;   // window slot: not a candidate
+        // four slots per thread and round, so that their loads are in flight together
+        for (int kb = tid; kb < n; kb += 4 * nthr) {
+            int p[4];
+            float f0[4], s[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int k = kb + b * nthr;
+                p[b] = k < n ? pos[k] : 0x7fffffff;
+                f0[b] = k < n ? __ldcg(F + k) : 0.f;
+                s[b] = 0.f;
+            }
+            for (int g = 0; g < G; ++g) {
+                const float c = cnew[g];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int k = kb + b * nthr;
+                    const float x = k < n ? __ldcg(sn + (size_t)g * a.cap + k) : -INFINITY;
+                    s[b] += exp2f(x - c);
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int k = kb + b * nthr;
+                if (k >= n) continue;
+                if ((long long)p[b] <= thr) {
+                    const float f = fuse(a.fusion, f0[b], s[b]);
+                    F[k] = f;
+                    const unsigned long long key = rank_key(__float_as_uint(f), p[b]);
+                    if (key < best) { best = key; bslot = k; }
+                } else {
+                    F[k] = -1.f;   // window slot: not a candidate
+                }
             }
         }
 #pragma unroll
@@ -173,7 +204,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
             if (ok < best) { best = ok; bslot = os; }
         }
         if (lane == 0) { red_key[warp] = best; red_slot[warp] = bslot; }
-        __syncthreads();
+        group_sync(bar_id, nthr);
         if (warp == 0) {
             best = lane < nwarp ? red_key[lane] : ~0ull;
             bslot = lane < nwarp ? red_slot[lane] : -1;
@@ -185,10 +216,10 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
             }
             if (lane == 0) red_slot[0] = bslot;
         }
-        __syncthreads();
+        group_sync(bar_id, nthr);
         e_slot = red_slot[0];
         e_pos = pos[e_slot];
-        __syncthreads();
+        group_sync(bar_id, nthr);
     }
 
     // Eq. 7 update: the freed (or next free) slot takes the new token; the ring row of the

@@ -9,6 +9,16 @@ namespace mkv {
 cudaError_t launch_decode_simt(const DecodeArgs &a, bool f32, int D, cudaStream_t stream);
 int simt_default_splits(int U, int cap);
 
+// Tensor-core (tcgen05) decode step: bf16, head_dim 128, GQA group in {1,2,4,8,16} and
+// R*G padded to a multiple of 32 at most 256.  The plan holds the TMA tensor maps of a
+// context's arena and the launch geometry; `a.splits` must be 2 * items per unit.
+bool tc_shape_supported(bool f32, int D, int G, int R);
+int tc_items_per_unit(int U, int cap, int G, int n_sm);
+struct TcPlan;
+cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int items_per_unit, char *err, size_t err_len);
+void tc_plan_destroy(TcPlan *plan);
+cudaError_t launch_decode_tc(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream);
+
 // Prompt phase: fills the arena (K, V, pos, ring) and the step state from a prompt of P
 // tokens.  `a` supplies the arena pointers and shape; q/k_new/v_new/out are ignored.
 // Allocates and frees its own temporary scratch.  *launches is advanced per kernel launched.

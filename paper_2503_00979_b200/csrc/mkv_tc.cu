@@ -1,0 +1,764 @@
+// Tensor-core decode kernel for sm_100a: bf16, head_dim 128, GQA group in {1,2,4,8,16},
+// R*G (padded to a multiple of 32) at most 256.
+//
+// A persistent, warp-specialised CTA per SM walks a static list of work items; an item is a
+// run of 128-key tiles of one unit's cache.
+//   warp 0       TMA producer: the unit's recent-query ring once per unit, then the item's K
+//                tiles and V tiles (cp.async.bulk.tensor, 128-byte swizzle) into one ring of
+//                32 KB stages guarded by mbarriers.
+//   warp 1       writes the new query over the ring row that leaves the window, then issues
+//                tcgen05.mma: S^T[128 keys x R*G rows] = K_tile . Q^T, fp32 accumulators in
+//                TMEM (one key per TMEM lane), two accumulator buffers.
+//   warps 2-9    two compute groups of four warps; group b owns TMEM buffer b and every second
+//                tile.  K phase: tcgen05.ld of a key's R*G logits, frozen soft-max weights
+//                exp2(s*scale - c_row), GQA group sum, window fusion (Eq. 4-6, Algorithm 1);
+//                the new row's logits are kept.  V phase: soft-max of the new row over the
+//                group's keys and P.V with mma.sync (P split in two bf16 terms), Eq. 1.
+//   The group that takes a unit's last ticket runs the shared per-unit epilogue (Eq. 7).
+// Every mbarrier wait is bounded; a wait that runs out sets a device error flag and the CTA
+// drains and exits.
+#include <cuda.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "mkv_common.cuh"
+#include "mkv_kernels.h"
+
+namespace mkv {
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kTile = 128;                  // keys per tile = MMA M = TMEM lanes
+constexpr int kStageBytes = 2 * kTile * 128;   // one K or V tile: two 64-column boxes
+constexpr int kThreadsTc = 32 * 10;
+constexpr int kGroupThreads = 128;
+constexpr long long kWaitCycles = 4000000000ll;   // about two seconds
+
+struct TcGeom {
+    int rgpad;          // ring rows padded to a multiple of 32 (MMA N)
+    int ipu;            // work items per unit
+    int stages;         // K/V stages in shared memory
+    int tpg;            // most tiles one compute group takes from one item
+    int tmem_cols;      // allocated TMEM columns (power of two)
+    int region_bytes;   // per-group scratch: kept logits of the new row / output reduction
+    int grid;
+    int smem_bytes;
+};
+
+struct SmemLayout {
+    int q, stages, region, negc, small, bars, total;
+};
+
+__host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g)
+{
+    SmemLayout L;
+    int o = 0;
+    L.q = o; o += g.rgpad * 256;
+    L.stages = o; o += g.stages * kStageBytes;
+    L.region = o; o += 2 * g.region_bytes;
+    L.negc = o; o += 2 * g.rgpad * 4;
+    L.small = o; o += 2 * (4 * kMaxGroup * 4 /*gm*/ + 4 * kMaxGroup * 4 /*lred*/ + kMaxGroup * 4 /*mloc*/ +
+                           kFinalizeSmemFloats * 4 + 16);
+    o = (o + 15) & ~15;
+    L.bars = o; o += 8 * (2 * 8 + 8) + 64;
+    L.total = o;
+    return L;
+}
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Gives up after kWaitCycles or as soon as another thread has raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0) {
+            if (*abort) return false;
+            if (clock64() - t0 > kWaitCycles) { *abort = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
+{
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+template <int N> __device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&v)[N]);
+template <> __device__ __forceinline__ void tmem_ld_n<1>(uint32_t taddr, uint32_t (&v)[1])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v[0]) : "r"(taddr) : "memory");
+}
+template <> __device__ __forceinline__ void tmem_ld_n<2>(uint32_t taddr, uint32_t (&v)[2])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];" : "=r"(v[0]), "=r"(v[1]) : "r"(taddr) : "memory");
+}
+template <> __device__ __forceinline__ void tmem_ld_n<4>(uint32_t taddr, uint32_t (&v)[4])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(taddr) : "memory");
+}
+template <> __device__ __forceinline__ void tmem_ld_n<8>(uint32_t taddr, uint32_t (&v)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr) : "memory");
+}
+template <> __device__ __forceinline__ void tmem_ld_n<16>(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// p = hi + lo with hi, lo bf16: two tensor-core terms carry about 16 mantissa bits of p
+__device__ __forceinline__ void split_bf16x2(float x, float y, uint32_t &hi, uint32_t &lo)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+    const float2 hf = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x - hf.x, y - hf.y);
+    hi = *reinterpret_cast<const uint32_t *>(&h);
+    lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+
+// group barrier that also ORs a predicate over the group (uniform bail-out decisions)
+__device__ __forceinline__ bool group_any(int bar_id, bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\nsetp.ne.b32 p, %1, 0;\nbarrier.red.or.pred q, %2, %3, p;\nselp.u32 %0, 1, 0, q;\n}"
+        : "=r"(r) : "r"((uint32_t)pred), "r"(bar_id), "r"(kGroupThreads) : "memory");
+    return r != 0;
+}
+
+// ---------------------------------------------------------------- schedule shared by all roles
+struct Item {
+    int unit, sp, tile0, nk;
+};
+struct Walk {     // the same deterministic walk over this CTA's items in every role
+    long long it, it_end;
+    int ipu, tpi, ntiles;
+    int prev_unit;
+    int qseq;         // units seen so far (ring loads)
+    int L0, T0;       // running load / tile sequence numbers
+    __device__ Walk(const TcGeom &g, int U, int n)
+    {
+        const long long total = (long long)U * g.ipu;
+        it = total * blockIdx.x / gridDim.x;
+        it_end = total * (blockIdx.x + 1) / gridDim.x;
+        ipu = g.ipu;
+        ntiles = (n + kTile - 1) / kTile;
+        tpi = (ntiles + ipu - 1) / ipu;
+        prev_unit = -1; qseq = 0; L0 = 0; T0 = 0;
+    }
+    // next item with work; new_unit tells whether the ring must be (re)loaded
+    __device__ bool next(Item &x, bool &new_unit)
+    {
+        while (it < it_end) {
+            x.unit = (int)(it / ipu);
+            x.sp = (int)(it % ipu);
+            x.tile0 = x.sp * tpi;
+            x.nk = min(tpi, ntiles - x.tile0);
+            ++it;
+            if (x.nk > 0) {
+                new_unit = x.unit != prev_unit;
+                prev_unit = x.unit;
+                return true;
+            }
+        }
+        return false;
+    }
+    __device__ void advance(const Item &x, bool new_unit)
+    {
+        L0 += 2 * x.nk;
+        T0 += x.nk;
+        if (new_unit) ++qseq;
+    }
+    __device__ int active_items() const { return (ntiles + tpi - 1) / tpi; }
+};
+
+template <int G, int FUSION>
+__device__ __forceinline__ void score_chunk(const uint32_t (&v)[32], const float *negc, float scale2, float &F)
+{
+    float part = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+        const float4 nc = *reinterpret_cast<const float4 *>(negc + j);
+        const float w0 = ex2f(fmaf(__uint_as_float(v[j + 0]), scale2, nc.x));
+        const float w1 = ex2f(fmaf(__uint_as_float(v[j + 1]), scale2, nc.y));
+        const float w2 = ex2f(fmaf(__uint_as_float(v[j + 2]), scale2, nc.z));
+        const float w3 = ex2f(fmaf(__uint_as_float(v[j + 3]), scale2, nc.w));
+        if (FUSION == kFusionSum) {
+            F += (w0 + w1) + (w2 + w3);
+        } else if (G == 1) {
+            F = fmaxf(fmaxf(F, fmaxf(w0, w1)), fmaxf(w2, w3));
+        } else if (G == 2) {
+            F = fmaxf(F, fmaxf(w0 + w1, w2 + w3));
+        } else {
+            part += (w0 + w1) + (w2 + w3);
+            if ((j + 4) % G == 0) { F = fmaxf(F, part); part = 0.f; }
+        }
+    }
+}
+
+template <int G, int FUSION>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
+                 const __grid_constant__ TcGeom geo)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // the swizzled operand tiles need a 1024-byte aligned base; the launch asks for 1 KB of slack
+    unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const SmemLayout L = tc_smem_layout(geo);
+    const int S = geo.stages, RGP = geo.rgpad;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t q_addr = sbase + L.q, st_addr = sbase + L.stages;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
+    // barrier indices
+    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + 8);
+    const uint32_t bar_tfull = smem_u32(bars + 16), bar_tempty = smem_u32(bars + 18);
+    const uint32_t bar_qfull = smem_u32(bars + 20), bar_qempty = smem_u32(bars + 21);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 22);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 23);
+
+    const long long t = a.st->t;
+    const int n = a.st->n;
+    const bool evict = step_evicts(t, n, a.R, a.C);
+    const int rs_new = (int)(t % a.R);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        mbar_init(bar_qfull, 1);
+        mbar_init(bar_qempty, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)geo.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer (one lane)
+        if (lane == 0) {
+            Walk w(geo, a.U, n);
+            Item x; bool nu;
+            int issued = 0;
+            bool ok = true;
+            while (ok && w.next(x, nu)) {
+                if (nu) {
+                    ok = mbar_wait(bar_qempty, (uint32_t)((w.qseq & 1) ^ 1), abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
+                    tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
+                    tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
+                }
+                for (int j = 0; j < 2 * x.nk && ok; ++j) {
+                    const int Ls = w.L0 + j, s = Ls % S;
+                    ok = mbar_wait(bar_empty + 8 * s, (uint32_t)(((Ls / S) & 1) ^ 1), abort_flag);
+                    if (!ok) break;
+                    const CUtensorMap *map = j < x.nk ? &tmK : &tmV;
+                    const int row = (x.tile0 + (j < x.nk ? j : j - x.nk)) * kTile;
+                    mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+                    tma_load_3d(st_addr + s * kStageBytes, map, 0, row, x.unit, bar_full + 8 * s);
+                    tma_load_3d(st_addr + s * kStageBytes + kStageBytes / 2, map, 64, row, x.unit, bar_full + 8 * s);
+                    issued = Ls + 1;
+                }
+                w.advance(x, nu);
+            }
+            if (!ok) {
+                // give up: let the copies already in flight land before the CTA exits
+                int dummy = 0;
+                for (int Ls = max(0, issued - S); Ls < issued; ++Ls)
+                    mbar_wait(bar_full + 8 * (Ls % S), (uint32_t)((Ls / S) & 1), &dummy);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ new-query substitution + MMA issue
+        Walk w(geo, a.U, n);
+        Item x; bool nu;
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RGP >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+        bool ok = true;
+        while (ok && w.next(x, nu)) {
+            if (nu) {
+                if (w.qseq > 0 && lane == 0) umma_commit(bar_qempty);   // MMAs of the previous unit done with the ring
+                // the new query replaces ring row t % R (the row of the token leaving the window)
+                uint4 qv[kMaxGroup / 2];
+                const uint4 *qsrc = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(a.q) + (size_t)x.unit * G * kD);
+#pragma unroll
+                for (int i = 0; i < (G * 16 + 31) / 32; ++i)
+                    if (lane + 32 * i < G * 16) qv[i] = qsrc[lane + 32 * i];
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.qseq & 1), abort_flag));
+                if (!ok) break;
+#pragma unroll
+                for (int i = 0; i < (G * 16 + 31) / 32; ++i) {
+                    const int c = lane + 32 * i;
+                    if (c < G * 16) {
+                        const int row = rs_new * G + c / 16, ch = c % 16;
+                        const uint32_t off = (uint32_t)((ch >> 3) * (RGP * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4));
+                        *reinterpret_cast<uint4 *>(smem + L.q + off) = qv[i];
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+            }
+            for (int j = 0; j < x.nk; ++j) {
+                const int Ls = w.L0 + j, s = Ls % S, T = w.T0 + j, b = T & 1;
+                bool k = mbar_wait(bar_full + 8 * s, (uint32_t)((Ls / S) & 1), abort_flag);
+                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(((T >> 1) & 1) ^ 1), abort_flag);
+                ok = __all_sync(0xffffffffu, k);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(b * RGP);
+#pragma unroll
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint64_t ad = smem_desc_sw128(st_addr + s * kStageBytes + (ks >> 2) * (kStageBytes / 2) + (ks & 3) * 32);
+                        const uint64_t bd = smem_desc_sw128(q_addr + (ks >> 2) * (RGP * 128) + (ks & 3) * 32);
+                        umma_bf16(d_tmem, ad, bd, idesc, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(bar_empty + 8 * s);       // K tile consumed
+                    umma_commit(bar_tfull + 8 * b);       // accumulators ready
+                }
+                __syncwarp();
+            }
+            w.advance(x, nu);
+        }
+    } else {
+        // ------------------------------------------------ compute groups
+        const int b = (warp - 2) >> 2;          // group = TMEM buffer
+        const int wq = warp & 3;                // TMEM lane quarter of this warp
+        const int gtid = wq * 32 + lane;
+        const int bar_id = 1 + b;
+        float *region = reinterpret_cast<float *>(smem + L.region + b * geo.region_bytes);
+        float *negc = reinterpret_cast<float *>(smem + L.negc) + b * RGP;
+        float *small = reinterpret_cast<float *>(smem + L.small) + b * (9 * kMaxGroup + kFinalizeSmemFloats + 4);
+        float *gm = small, *lred = small + 4 * kMaxGroup, *mloc = small + 8 * kMaxGroup;
+        float *fin_sm = small + 9 * kMaxGroup;              // 8-byte aligned: 9*16 floats = 576 bytes
+        int *flag = reinterpret_cast<int *>(fin_sm + kFinalizeSmemFloats);
+        float *st_w = region + wq * (geo.tpg * G * 32);     // this warp's kept logits [tile][g][lane]
+        const int RG = a.R * G;
+        const int g0 = lane >> 2, tig = lane & 3;
+
+        Walk w(geo, a.U, n);
+        Item x; bool nu;
+        bool ok = true;
+        while (ok && w.next(x, nu)) {
+            const int u = x.unit;
+            if (nu) {
+                // frozen normalisers of the ring rows, negated; the new row and padding give weight 0
+                for (int c = gtid; c < RGP; c += kGroupThreads) {
+                    float v = -INFINITY;
+                    if (c < RG && c / G != rs_new) v = -a.ring_c[(size_t)u * RG + c];
+                    negc[c] = v;
+                }
+                group_sync(bar_id, kGroupThreads);
+            }
+            float mx[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) mx[g] = -INFINITY;
+            int nown = 0;
+            float *s_new = a.s_new + (size_t)u * G * a.cap;
+            // ---- K phase: this group's tiles
+            for (int j = 0; j < x.nk; ++j) {
+                const int T = w.T0 + j;
+                if ((T & 1) != b) continue;
+                if (group_any(bar_id, !mbar_wait(bar_tfull + 8 * b, (uint32_t)((T >> 1) & 1), abort_flag))) { ok = false; break; }
+                tc_fence_after();
+                const int key = (x.tile0 + j) * kTile + gtid;
+                const bool valid = key < n;
+                const uint32_t taddr = tmem_base + (uint32_t)(b * RGP) + ((uint32_t)(wq * 32) << 16);
+                uint32_t sv[G];
+                tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
+                float F = 0.f;
+                if (evict) {
+                    for (int c = 0; c < RGP; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + (uint32_t)c, v);
+                        tc_wait_ld();
+                        score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
+                    }
+                } else {
+                    tc_wait_ld();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * b);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const float s2 = valid ? __uint_as_float(sv[g]) * a.scale2 : -INFINITY;
+                    st_w[(nown * G + g) * 32 + lane] = s2;
+                    if (valid) s_new[(size_t)g * a.cap + key] = s2;
+                    mx[g] = fmaxf(mx[g], s2);
+                }
+                if (evict && valid) a.F[(size_t)u * a.cap + key] = F;
+                ++nown;
+            }
+            if (!ok) break;
+            // ---- soft-max reference of the group: max over its keys
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float m = warp_max(mx[g]);
+                if (lane == 0) gm[wq * kMaxGroup + g] = m;
+            }
+            group_sync(bar_id, kGroupThreads);
+            if (gtid < G) mloc[gtid] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
+            group_sync(bar_id, kGroupThreads);
+
+            // ---- V phase: P.V over this group's tiles, this warp's 32 keys of each
+            float acc[16][4];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { acc[i][0] = 0.f; acc[i][1] = 0.f; acc[i][2] = 0.f; acc[i][3] = 0.f; }
+            float lsum0 = 0.f, lsum1 = 0.f;
+            const float mA = g0 < G ? mloc[g0] : 0.f;
+            const float mB = (G > 8 && g0 + 8 < G) ? mloc[g0 + 8] : 0.f;
+            int jl = 0;
+            for (int j = 0; j < x.nk; ++j) {
+                const int T = w.T0 + j;
+                if ((T & 1) != b) continue;
+                const int Ls = w.L0 + x.nk + j, s = Ls % S;
+                if (group_any(bar_id, !mbar_wait(bar_full + 8 * s, (uint32_t)((Ls / S) & 1), abort_flag))) { ok = false; break; }
+                const uint32_t vbase = st_addr + s * kStageBytes;
+#pragma unroll
+                for (int ks = 0; ks < 2; ++ks) {
+                    uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
+                    if (g0 < G) {
+                        const float *sp = st_w + (jl * G + g0) * 32 + ks * 16 + tig * 2;
+                        const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
+                        const float p0 = ex2f(sa.x - mA), p1 = ex2f(sa.y - mA), p2 = ex2f(sb.x - mA), p3 = ex2f(sb.y - mA);
+                        lsum0 += (p0 + p1) + (p2 + p3);
+                        split_bf16x2(p0, p1, ahi[0], alo[0]);
+                        split_bf16x2(p2, p3, ahi[2], alo[2]);
+                    }
+                    if (G > 8 && g0 + 8 < G) {
+                        const float *sp = st_w + (jl * G + g0 + 8) * 32 + ks * 16 + tig * 2;
+                        const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
+                        const float p0 = ex2f(sa.x - mB), p1 = ex2f(sa.y - mB), p2 = ex2f(sb.x - mB), p3 = ex2f(sb.y - mB);
+                        lsum1 += (p0 + p1) + (p2 + p3);
+                        split_bf16x2(p0, p1, ahi[1], alo[1]);
+                        split_bf16x2(p2, p3, ahi[3], alo[3]);
+                    }
+                    const int mat = lane >> 3, r = lane & 7;
+                    const int krow = wq * 32 + ks * 16 + (mat & 1) * 8 + r;
+#pragma unroll
+                    for (int np = 0; np < 8; ++np) {
+                        const int ch = np * 2 + (mat >> 1);
+                        const uint32_t addr = vbase + (uint32_t)((ch >> 3) * (kStageBytes / 2) + krow * 128 + (((ch & 7) ^ (krow & 7)) << 4));
+                        uint32_t bf[4];
+                        ldmatrix_x4_trans(addr, bf);
+                        mma_bf16_16816(acc[2 * np], ahi, bf[0], bf[1]);
+                        mma_bf16_16816(acc[2 * np], alo, bf[0], bf[1]);
+                        mma_bf16_16816(acc[2 * np + 1], ahi, bf[2], bf[3]);
+                        mma_bf16_16816(acc[2 * np + 1], alo, bf[2], bf[3]);
+                    }
+                }
+                group_sync(bar_id, kGroupThreads);           // every warp has read its rows of the V tile
+                if (gtid == 0) mbar_arrive(bar_empty + 8 * s);
+                ++jl;
+            }
+            if (!ok) break;
+
+            // ---- group partial (max, denominator, un-normalised output) -> global
+            const int part = x.sp * 2 + b;
+            float *pml = a.part_ml + ((size_t)u * a.splits + part) * G * 2;
+            float *po = a.part_o + ((size_t)u * a.splits + part) * G * kD;
+            if (nown > 0) {
+                float *red = region;     // [4 warps][G][128]; the kept logits are no longer needed
+                lsum0 += __shfl_xor_sync(0xffffffffu, lsum0, 1);
+                lsum0 += __shfl_xor_sync(0xffffffffu, lsum0, 2);
+                lsum1 += __shfl_xor_sync(0xffffffffu, lsum1, 1);
+                lsum1 += __shfl_xor_sync(0xffffffffu, lsum1, 2);
+                if (tig == 0 && g0 < G) lred[wq * kMaxGroup + g0] = lsum0;
+                if (G > 8 && tig == 0 && g0 + 8 < G) lred[wq * kMaxGroup + g0 + 8] = lsum1;
+#pragma unroll
+                for (int nt = 0; nt < 16; ++nt) {
+                    if (g0 < G) *reinterpret_cast<float2 *>(red + (wq * G + g0) * kD + nt * 8 + tig * 2) = make_float2(acc[nt][0], acc[nt][1]);
+                    if (G > 8 && g0 + 8 < G)
+                        *reinterpret_cast<float2 *>(red + (wq * G + g0 + 8) * kD + nt * 8 + tig * 2) = make_float2(acc[nt][2], acc[nt][3]);
+                }
+                group_sync(bar_id, kGroupThreads);
+                for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
+                    po[idx] = (red[idx] + red[G * kD + idx]) + (red[2 * G * kD + idx] + red[3 * G * kD + idx]);
+                if (gtid < G) {
+                    pml[gtid * 2] = mloc[gtid];
+                    pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
+                }
+            } else {
+                for (int idx = gtid; idx < G * kD; idx += kGroupThreads) po[idx] = 0.f;
+                if (gtid < G) { pml[gtid * 2] = -INFINITY; pml[gtid * 2 + 1] = 0.f; }
+            }
+            __threadfence();
+            group_sync(bar_id, kGroupThreads);
+            const int active2 = 2 * w.active_items();
+            if (gtid == 0) *flag = (atomicAdd(&a.ticket[u], 1) == active2 - 1);
+            group_sync(bar_id, kGroupThreads);
+            if (*flag) {
+                __threadfence();
+                finalize_unit<__nv_bfloat16, kD>(a, u, t, n, active2, evict, fin_sm, gtid, kGroupThreads, bar_id);
+            }
+            group_sync(bar_id, kGroupThreads);
+            w.advance(x, nu);
+        }
+    }
+
+    // ------------------------------------------------ tail
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)geo.tmem_cols);
+    }
+    if (tid == 0 && *abort_flag) atomicExch(&a.st->err, (int)kErrBarrierTimeout);
+    finish_cta(a, t, n, evict);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [units][rows][128] bf16 tensor, boxes of 64 columns x box_rows rows, 128-byte swizzle
+bool encode_map(CUtensorMap *m, void *base, int units, int rows, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows, (cuuint64_t)units};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)rows * kD * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct TcPlan {
+    CUtensorMap tmK, tmV, tmQ;
+    TcGeom geo;
+    bool attr_set[5][2];
+};
+
+namespace {
+
+int group_index(int G) { return G == 1 ? 0 : G == 2 ? 1 : G == 4 ? 2 : G == 8 ? 3 : G == 16 ? 4 : -1; }
+
+template <int G, int FUSION>
+cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
+{
+    auto kern = decode_tc_kernel<G, FUSION>;
+    bool &set = plan->attr_set[group_index(G)][FUSION];
+    if (!set) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan->geo.smem_bytes);
+        if (e != cudaSuccess) return e;
+        set = true;
+    }
+    kern<<<plan->geo.grid, kThreadsTc, plan->geo.smem_bytes, stream>>>(a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
+    return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_g(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
+{
+    return a.fusion == kFusionSum ? launch_gf<G, kFusionSum>(plan, a, stream) : launch_gf<G, kFusionMax>(plan, a, stream);
+}
+
+int pad32(int x) { return (x + 31) & ~31; }
+
+}  // namespace
+
+bool tc_shape_supported(bool f32, int D, int G, int R)
+{
+    if (f32 || D != kD || group_index(G) < 0) return false;
+    return pad32(R * G) <= 256;
+}
+
+// Items per unit: enough that one item's tiles fit the per-group scratch, then the count that
+// fills whole waves of the persistent grid best (ties: fewer, larger items).
+int tc_items_per_unit(int U, int cap, int G, int n_sm)
+{
+    const int ntiles = (cap + kTile - 1) / kTile;
+    const int tpg_max = 32 / G < 1 ? 1 : 32 / G;
+    const int min_ipu = (ntiles + 2 * tpg_max - 1) / (2 * tpg_max);
+    int best = min_ipu;
+    double best_eff = -1.0;
+    for (int ipu = min_ipu; ipu <= ntiles; ++ipu) {
+        const int tpi = (ntiles + ipu - 1) / ipu;
+        if (tpi < 2 && ipu > min_ipu) break;
+        const long long items = (long long)U * ((ntiles + tpi - 1) / tpi);
+        const long long waves = (items + n_sm - 1) / n_sm;
+        // time ~ waves * tiles per item (+ a fixed cost per item)
+        const double cost = (double)waves * (tpi + 0.35);
+        const double eff = (double)U * ntiles / (cost * n_sm);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = ipu; }
+    }
+    return best;
+}
+
+cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err, size_t err_len)
+{
+    *out = nullptr;
+    TcPlan *p = new (std::nothrow) TcPlan;
+    if (!p) return cudaErrorMemoryAllocation;
+    memset(p, 0, sizeof(*p));
+    int dev = 0, n_sm = 0, max_smem = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) { delete p; return e; }
+    TcGeom &g = p->geo;
+    const int G = a.G;
+    g.rgpad = pad32(a.R * G);
+    g.ipu = ipu;
+    const int ntiles = (a.cap + kTile - 1) / kTile;
+    const int tpi = (ntiles + ipu - 1) / ipu;
+    g.tpg = (tpi + 1) / 2;
+    g.tmem_cols = 64;
+    while (g.tmem_cols < 2 * g.rgpad) g.tmem_cols *= 2;
+    const int stw = 4 * g.tpg * G * 32 * 4, red = 4 * G * kD * 4;
+    g.region_bytes = ((stw > red ? stw : red) + 127) & ~127;
+    const long long items = (long long)a.U * ipu;
+    g.grid = (int)(items < n_sm ? items : n_sm);
+    for (g.stages = 6; g.stages >= 2; --g.stages) {
+        g.smem_bytes = tc_smem_layout(g).total + 1024;
+        if (g.smem_bytes <= max_smem) break;
+    }
+    if (g.stages < 2 || g.stages > 8) {
+        snprintf(err, err_len, "tensor-core kernel: shared memory does not fit (need %d bytes)", g.smem_bytes);
+        delete p;
+        return cudaErrorInvalidConfiguration;
+    }
+    if (!encode_map(&p->tmK, a.K, a.U, a.cap, kTile) || !encode_map(&p->tmV, a.V, a.U, a.cap, kTile) ||
+        !encode_map(&p->tmQ, a.ring_q, a.U, a.R * G, g.rgpad)) {
+        snprintf(err, err_len, "tensor-core kernel: cuTensorMapEncodeTiled failed");
+        delete p;
+        return cudaErrorInvalidValue;
+    }
+    *out = p;
+    return cudaSuccess;
+}
+
+void tc_plan_destroy(TcPlan *plan) { delete plan; }
+
+cudaError_t launch_decode_tc(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
+{
+    switch (a.G) {
+        case 1: return launch_g<1>(plan, a, stream);
+        case 2: return launch_g<2>(plan, a, stream);
+        case 4: return launch_g<4>(plan, a, stream);
+        case 8: return launch_g<8>(plan, a, stream);
+        case 16: return launch_g<16>(plan, a, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace mkv

@@ -161,3 +161,99 @@ def test_slot_permutation_does_not_change_results():
         mk.close()
     assert torch.equal(outs[0][1], outs[1][1])
     assert (outs[0][0] - outs[1][0]).abs().max() < 2e-2
+
+
+# ---- tensor-core kernel (bf16, d = 128) ----------------------------------------------------
+def test_tc_smallest_case_first():
+    w = SMALL.replace(layers=1, batch=1, steps=24)
+    rep = run_parity(w, steps=w.steps, n_units=2, kernel="tc")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+
+
+def test_auto_picks_the_tensor_core_kernel_for_bf16_d128():
+    mk = binding.MorphKV(1, 1, 8, 2, 128, 64, 16, "sum", "bf16")
+    assert mk.kernel_name == "tc"
+    mk.close()
+    mk = binding.MorphKV(1, 1, 8, 2, 64, 64, 16, "sum", "bf16")
+    assert mk.kernel_name == "simt"
+    mk.close()
+    mk = binding.MorphKV(1, 1, 14, 2, 128, 64, 16, "sum", "bf16")      # G = 7: CUDA-core kernel
+    assert mk.kernel_name == "simt"
+    mk.close()
+    p = binding.mkv_default_params()
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 14, 2, 128, 64, 16
+    p.kernel = binding.KERNEL["tc"]
+    st, h = binding.mkv_create_ex(p)
+    assert st == binding.UNSUPPORTED and h is None
+
+
+@pytest.mark.parametrize("fusion", ["sum", "max"])
+@pytest.mark.parametrize("G,R", [(1, 32), (2, 24), (4, 32), (4, 30), (8, 16), (16, 9), (4, 64)])
+def test_tc_groups_windows_and_fusions(fusion, G, R):
+    # R*G = 120 and 144 are padded to a multiple of 32; R*G = 256 fills both accumulator buffers
+    w = SMALL.replace(layers=1, batch=2, n_q_heads=2 * G, n_kv_heads=2, R=R, C=301, prompt_len=411, steps=40,
+                      fusion=fusion)
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel="tc")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0 and rep.F_compared > 0
+
+
+@pytest.mark.parametrize("ipu", [1, 2, 3, 7])
+def test_tc_item_counts_give_the_same_answer(ipu):
+    w = SMALL.replace(layers=1, C=1500, R=32, prompt_len=1700, steps=36, fusion="max")     # 12 tiles, ragged tail
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel="tc", splits=ipu)
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_tc_fill_phase_warmup_and_single_tile():
+    rep = run_parity(SMALL.replace(C=120, R=16, prompt_len=100, steps=80), steps=80, n_units=8, kernel="tc")
+    _report(rep)
+    assert rep.evictions == 8 * (80 - 36)
+    rep = run_parity(SMALL.replace(C=20, R=16, prompt_len=5, steps=60, layers=1), steps=60, n_units=4, kernel="tc")
+    _report(rep)
+    assert rep.evictions > 0
+    rep = run_parity(SMALL.replace(C=300, R=16, prompt_len=120, steps=200, layers=1), steps=200, n_units=4, kernel="tc")
+    _report(rep)       # crosses from one tile to three while filling
+    assert rep.evictions == 0
+
+
+def test_tc_llama_shape_two_layers():
+    w = synth.WORKLOADS["c1"].replace(layers=2, steps=96)
+    rep = run_parity(w, steps=w.steps, n_units=8, kernel="tc")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions == 8 * 96
+
+
+def test_tc_stress_shape_window_64():
+    w = synth.WORKLOADS["c3"].replace(layers=1, batch=2, prompt_len=4100, steps=48)    # starts full: C=4000, R=64
+    rep = run_parity(w, steps=w.steps, n_units=6, kernel="tc")
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_tc_matches_cuda_core_kernel_on_device():
+    # the two kernels share only the per-unit epilogue; their outputs must agree closely
+    w = SMALL.replace(layers=1, batch=2, C=700, R=32, prompt_len=900, steps=12, fusion="max")
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    k, v = st.kv(np.arange(w.prompt_len))
+    qw = st.q(np.arange(w.prompt_len - w.R, w.prompt_len))
+    res = {}
+    for kern in ("simt", "tc"):
+        mk = binding.MorphKV(1, 2, 8, 2, 128, w.C, w.R, w.fusion, "bf16", kernel=kern)
+        mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+        outs, ev = [], []
+        for i in range(w.steps):
+            p = [w.prompt_len + i]
+            kk, vv = st.kv(p)
+            outs.append(mk.decode_step(st.q(p)[:, :, :, 0].bfloat16().contiguous(), kk[:, :, :, 0].bfloat16().contiguous(),
+                                       vv[:, :, :, 0].bfloat16().contiguous()).float())
+            ev.append(mk.view(0)["evicted_pos"].clone())
+        mk.sync()
+        res[kern] = (torch.stack(outs), torch.stack(ev), mk.view(0)["ring_c"].clone())
+        mk.close()
+    assert torch.equal(res["simt"][1], res["tc"][1])
+    assert (res["simt"][0] - res["tc"][0]).abs().max() <= 2 ** -6       # one bf16 ulp at |o| < 4
+    assert torch.allclose(res["simt"][2], res["tc"][2], rtol=0, atol=2e-4)
