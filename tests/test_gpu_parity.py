@@ -214,7 +214,7 @@ def test_tc_fill_phase_warmup_and_single_tile():
     rep = run_parity(SMALL.replace(C=20, R=16, prompt_len=5, steps=60, layers=1), steps=60, n_units=4, kernel="tc")
     _report(rep)
     assert rep.evictions > 0
-    rep = run_parity(SMALL.replace(C=300, R=16, prompt_len=120, steps=200, layers=1), steps=200, n_units=4, kernel="tc")
+    rep = run_parity(SMALL.replace(C=300, R=16, prompt_len=120, steps=190, layers=1), steps=190, n_units=4, kernel="tc")
     _report(rep)       # crosses from one tile to three while filling
     assert rep.evictions == 0
 
