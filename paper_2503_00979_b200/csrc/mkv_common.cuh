@@ -107,13 +107,17 @@ __device__ __forceinline__ void group_sync(int bar_id, int nthr)
 // Per-unit epilogue, run by the group of threads that finished a unit last (`tid` in
 // [0, nthr), nthr a multiple of 32, all of them synchronising on barrier `bar_id`).  Data
 // written by other CTAs is read with ld.global.cg so that no stale L1 line can be used.
-// `sm` needs kFinalizeSmemFloats floats of shared memory, 8-byte aligned.
-template <typename T, int D>
+// `sm` needs kFinalizeSmemFloats floats of shared memory, 8-byte aligned.  GT is the GQA
+// group size when known at compile time (0: use a.G); it lets the loads of a round be
+// issued together.  Loads are batched so that the whole epilogue costs a handful of L2
+// round trips.
+template <typename T, int D, int GT>
 __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, int active, bool evict, float *sm,
                               int tid, int nthr, int bar_id)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
-    const int G = a.G;
+    const int G = GT > 0 ? GT : a.G;
+    constexpr int GU = GT > 0 ? GT : 1;    // unroll width of the per-head loads
     float *s_self = sm, *mfin = sm + kMaxGroup, *lfin = sm + 2 * kMaxGroup, *cnew = sm + 3 * kMaxGroup;
     unsigned long long *red_key = reinterpret_cast<unsigned long long *>(sm + 4 * kMaxGroup);  // [32]
     int *red_slot = reinterpret_cast<int *>(sm + 4 * kMaxGroup + 64);                          // [32]
@@ -133,11 +137,27 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     }
     group_sync(bar_id, nthr);
     if (tid < G) {
+        // two passes over the partial (max, denominator) pairs, eight loads in flight at a time
         float m = s_self[tid];
-        for (int sp = 0; sp < active; ++sp) m = fmaxf(m, __ldcg(pml + (sp * G + tid) * 2));
+        for (int sp0 = 0; sp0 < active; sp0 += 8) {
+            float pm[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pm[i] = sp0 + i < active ? __ldcg(pml + ((sp0 + i) * G + tid) * 2) : -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) m = fmaxf(m, pm[i]);
+        }
         float l = exp2f(s_self[tid] - m);
-        for (int sp = 0; sp < active; ++sp)
-            l += __ldcg(pml + (sp * G + tid) * 2 + 1) * exp2f(__ldcg(pml + (sp * G + tid) * 2) - m);
+        for (int sp0 = 0; sp0 < active; sp0 += 8) {
+            float pm[8], pl[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool ok = sp0 + i < active;
+                pm[i] = ok ? __ldcg(pml + ((sp0 + i) * G + tid) * 2) : -INFINITY;
+                pl[i] = ok ? __ldcg(pml + ((sp0 + i) * G + tid) * 2 + 1) : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) l += pl[i] * exp2f(pm[i] - m);
+        }
         mfin[tid] = m;
         lfin[tid] = l;
         cnew[tid] = m + log2f(l);
@@ -148,9 +168,17 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         const int g = idx / D, dd = idx % D;
         const float m = mfin[g];
         float o = exp2f(s_self[g] - m) * ldf(vn + dd);
-#pragma unroll 4
-        for (int sp = 0; sp < active; ++sp)
-            o += __ldcg(po + (sp * G + g) * D + dd) * exp2f(__ldcg(pml + (sp * G + g) * 2) - m);
+        for (int sp0 = 0; sp0 < active; sp0 += 8) {
+            float pv[8], pm[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool ok = sp0 + i < active;
+                pv[i] = ok ? __ldcg(po + ((sp0 + i) * G + g) * D + dd) : 0.f;
+                pm[i] = ok ? __ldcg(pml + ((sp0 + i) * G + g) * 2) : -INFINITY;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o += pv[i] * exp2f(pm[i] - m);
+        }
         stf(out + idx, o / lfin[g]);
     }
 
@@ -163,7 +191,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         const long long thr = t - a.R;
         unsigned long long best = ~0ull;
         int bslot = -1;
-        // four slots per thread and round, so that their loads are in flight together
+        // four slots per thread and round, all their loads in flight together
         for (int kb = tid; kb < n; kb += 4 * nthr) {
             int p[4];
             float f0[4], s[4];
@@ -174,14 +202,19 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
                 f0[b] = k < n ? __ldcg(F + k) : 0.f;
                 s[b] = 0.f;
             }
-            for (int g = 0; g < G; ++g) {
-                const float c = cnew[g];
+            for (int g0 = 0; g0 < G; g0 += GU) {
+                float x[GU][4];
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    const int k = kb + b * nthr;
-                    const float x = k < n ? __ldcg(sn + (size_t)g * a.cap + k) : -INFINITY;
-                    s[b] += exp2f(x - c);
-                }
+                for (int gi = 0; gi < GU; ++gi)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const int k = kb + b * nthr;
+                        x[gi][b] = k < n ? __ldcg(sn + (size_t)(g0 + gi) * a.cap + k) : -INFINITY;
+                    }
+#pragma unroll
+                for (int gi = 0; gi < GU; ++gi)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) s[b] += exp2f(x[gi][b] - cnew[g0 + gi]);
             }
 #pragma unroll
             for (int b = 0; b < 4; ++b) {

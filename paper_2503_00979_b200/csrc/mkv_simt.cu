@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(const __grid_cons
         __syncthreads();
         if (is_last) {
             __threadfence();
-            finalize_unit<T, D>(a, u, t, n, active, evict, misc + 64, tid, kThreads, 0);
+            finalize_unit<T, D, 0>(a, u, t, n, active, evict, misc + 64, tid, kThreads, 0);
         }
     }
     finish_cta(a, t, n, evict);

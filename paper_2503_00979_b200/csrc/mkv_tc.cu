@@ -126,6 +126,22 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// wait for outstanding tcgen05.ld; the registers are operands so that no use of them can be
+// scheduled before the wait
+__device__ __forceinline__ void tc_wait_ld32(uint32_t (&v)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                   "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                   "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+                 :: "memory");
+}
+template <int N> __device__ __forceinline__ void tc_tie(uint32_t (&v)[N])
+{
+#pragma unroll
+    for (int i = 0; i < N; ++i) asm volatile("" : "+r"(v[i]));
+}
 
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
 {
@@ -234,15 +250,34 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
     int prev_unit;
     int qseq;         // units seen so far (ring loads)
     int L0, T0;       // running load / tile sequence numbers
+    long long total;
     __device__ Walk(const TcGeom &g, int U, int n)
     {
-        const long long total = (long long)U * g.ipu;
-        it = total * blockIdx.x / gridDim.x;
-        it_end = total * (blockIdx.x + 1) / gridDim.x;
+        total = (long long)U * g.ipu;
+        // item i belongs to CTA (i * grid) / total, so CTA c owns [ceil(c*total/grid), ceil((c+1)*total/grid))
+        it = (total * blockIdx.x + gridDim.x - 1) / gridDim.x;
+        it_end = (total * (blockIdx.x + 1) + gridDim.x - 1) / gridDim.x;
         ipu = g.ipu;
         ntiles = (n + kTile - 1) / kTile;
         tpi = (ntiles + ipu - 1) / ipu;
         prev_unit = -1; qseq = 0; L0 = 0; T0 = 0;
+    }
+    // A unit's active items may spread over several CTAs; each CTA's share is one *segment* per
+    // compute group.  Returns the number of segments of unit u and this CTA's first slot.
+    __device__ int segments(int u, int &my_first) const
+    {
+        const long long i0 = (long long)u * ipu, i1 = i0 + active_items() - 1;
+        const int c0 = (int)(i0 * gridDim.x / total), c1 = (int)(i1 * gridDim.x / total);
+        my_first = ((int)blockIdx.x - c0) * 2;
+        return 2 * (c1 - c0 + 1);
+    }
+    // true if the next item with work (if any) belongs to another unit
+    __device__ bool last_of_unit_here(const Item &x) const
+    {
+        const long long nxt = (long long)x.unit * ipu + x.sp + 1;     // == it after next()
+        if (nxt >= it_end) return true;
+        if (nxt / ipu != x.unit) return true;
+        return (int)(nxt % ipu) * tpi >= ntiles;                       // remaining items of this unit are empty
     }
     // next item with work; new_unit tells whether the ring must be (re)loaded
     __device__ bool next(Item &x, bool &new_unit)
@@ -430,12 +465,20 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         float *region = reinterpret_cast<float *>(smem + L.region + b * geo.region_bytes);
         float *negc = reinterpret_cast<float *>(smem + L.negc) + b * RGP;
         float *small = reinterpret_cast<float *>(smem + L.small) + b * (9 * kMaxGroup + kFinalizeSmemFloats + 4);
-        float *gm = small, *lred = small + 4 * kMaxGroup, *mloc = small + 8 * kMaxGroup;
+        float *gm = small, *lred = small + 4 * kMaxGroup, *mrun = small + 8 * kMaxGroup;
         float *fin_sm = small + 9 * kMaxGroup;              // 8-byte aligned: 9*16 floats = 576 bytes
         int *flag = reinterpret_cast<int *>(fin_sm + kFinalizeSmemFloats);
         float *st_w = region + wq * (geo.tpg * G * 32);     // this warp's kept logits [tile][g][lane]
         const int RG = a.R * G;
-        const int g0 = lane >> 2, tig = lane & 3;
+        const int gid = lane >> 2, tig = lane & 3;
+        constexpr int NT = G > 8 ? 2 : 1;                   // 8-head column tiles of the transposed output
+
+        // Running soft-max state of the open segment (consecutive items of one unit): the
+        // reference max per head in shared memory, this thread's share of the denominator and
+        // of the un-normalised output O^T[d][g] in registers.
+        float acc[NT][8][4];
+        float lsum[NT];
+        int seg_unit = -1, seg_tiles = 0;
 
         Walk w(geo, a.U, n);
         Item x; bool nu;
@@ -449,6 +492,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     if (c < RG && c / G != rs_new) v = -a.ring_c[(size_t)u * RG + c];
                     negc[c] = v;
                 }
+                if (gtid < G) mrun[gtid] = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    lsum[nt] = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
+                }
+                seg_unit = u; seg_tiles = 0;
                 group_sync(bar_id, kGroupThreads);
             }
             float mx[G];
@@ -469,15 +520,23 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
                 float F = 0.f;
                 if (evict) {
-                    for (int c = 0; c < RGP; c += 32) {
-                        uint32_t v[32];
-                        tmem_ld32(taddr + (uint32_t)c, v);
-                        tc_wait_ld();
-                        score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
+                    // chunk c+1 is in flight while chunk c is turned into weights
+                    uint32_t v[2][32];
+                    const int nch = RGP >> 5;
+                    tmem_ld32(taddr, v[0]);
+                    tc_wait_ld32(v[0]);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        if (c < nch) {
+                            if (c + 1 < nch) tmem_ld32(taddr + (uint32_t)((c + 1) * 32), v[(c + 1) & 1]);
+                            score_chunk<G, FUSION>(v[c & 1], negc + c * 32, a.scale2, F);
+                            if (c + 1 < nch) tc_wait_ld32(v[(c + 1) & 1]);
+                        }
                     }
                 } else {
                     tc_wait_ld();
                 }
+                tc_tie<G>(sv);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * b);
@@ -492,23 +551,40 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 ++nown;
             }
             if (!ok) break;
-            // ---- soft-max reference of the group: max over its keys
+
+            // ---- new reference max of the segment; rescale what has been accumulated so far
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const float m = warp_max(mx[g]);
                 if (lane == 0) gm[wq * kMaxGroup + g] = m;
             }
             group_sync(bar_id, kGroupThreads);
-            if (gtid < G) mloc[gtid] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
-            group_sync(bar_id, kGroupThreads);
-
-            // ---- V phase: P.V over this group's tiles, this warp's 32 keys of each
-            float acc[16][4];
+            float mnew_row[NT], mnew_c0[NT], mnew_c1[NT];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) { acc[i][0] = 0.f; acc[i][1] = 0.f; acc[i][2] = 0.f; acc[i][3] = 0.f; }
-            float lsum0 = 0.f, lsum1 = 0.f;
-            const float mA = g0 < G ? mloc[g0] : 0.f;
-            const float mB = (G > 8 && g0 + 8 < G) ? mloc[g0 + 8] : 0.f;
+            for (int nt = 0; nt < NT; ++nt) {
+                // heads this thread needs: row gid (+8 nt) for P, columns tig*2, tig*2+1 (+8 nt) of O^T
+                const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
+                auto mnew = [&](int g) {
+                    return fmaxf(fmaxf(mrun[g], fmaxf(gm[g], gm[kMaxGroup + g])), fmaxf(gm[2 * kMaxGroup + g], gm[3 * kMaxGroup + g]));
+                };
+                mnew_row[nt] = gr < G ? mnew(gr) : 0.f;
+                mnew_c0[nt] = gc < G ? mnew(gc) : 0.f;
+                mnew_c1[nt] = gc + 1 < G ? mnew(gc + 1) : 0.f;
+                if (seg_tiles > 0 && nown > 0) {
+                    const float fr = gr < G ? ex2f(mrun[gr] - mnew_row[nt]) : 0.f;
+                    const float f0 = gc < G ? ex2f(mrun[gc] - mnew_c0[nt]) : 0.f;
+                    const float f1 = gc + 1 < G ? ex2f(mrun[gc + 1] - mnew_c1[nt]) : 0.f;
+                    lsum[nt] *= fr;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { acc[nt][i][0] *= f0; acc[nt][i][1] *= f1; acc[nt][i][2] *= f0; acc[nt][i][3] *= f1; }
+                }
+            }
+            group_sync(bar_id, kGroupThreads);         // everyone has read the old reference
+            if (gtid < G && nown > 0)
+                mrun[gtid] = fmaxf(fmaxf(mrun[gtid], fmaxf(gm[gtid], gm[kMaxGroup + gtid])),
+                                   fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
+
+            // ---- V phase: O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys of each tile
             int jl = 0;
             for (int j = 0; j < x.nk; ++j) {
                 const int T = w.T0 + j;
@@ -518,35 +594,34 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 const uint32_t vbase = st_addr + s * kStageBytes;
 #pragma unroll
                 for (int ks = 0; ks < 2; ++ks) {
-                    uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
-                    if (g0 < G) {
-                        const float *sp = st_w + (jl * G + g0) * 32 + ks * 16 + tig * 2;
-                        const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
-                        const float p0 = ex2f(sa.x - mA), p1 = ex2f(sa.y - mA), p2 = ex2f(sb.x - mA), p3 = ex2f(sb.y - mA);
-                        lsum0 += (p0 + p1) + (p2 + p3);
-                        split_bf16x2(p0, p1, ahi[0], alo[0]);
-                        split_bf16x2(p2, p3, ahi[2], alo[2]);
-                    }
-                    if (G > 8 && g0 + 8 < G) {
-                        const float *sp = st_w + (jl * G + g0 + 8) * 32 + ks * 16 + tig * 2;
-                        const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
-                        const float p0 = ex2f(sa.x - mB), p1 = ex2f(sa.y - mB), p2 = ex2f(sb.x - mB), p3 = ex2f(sb.y - mB);
-                        lsum1 += (p0 + p1) + (p2 + p3);
-                        split_bf16x2(p0, p1, ahi[1], alo[1]);
-                        split_bf16x2(p2, p3, ahi[3], alo[3]);
+                    uint32_t bhi[NT][2], blo[NT][2];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        bhi[nt][0] = bhi[nt][1] = blo[nt][0] = blo[nt][1] = 0u;
+                        const int gr = gid + 8 * nt;
+                        if (gr < G) {
+                            const float *sp = st_w + (jl * G + gr) * 32 + ks * 16 + tig * 2;
+                            const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
+                            const float m = mnew_row[nt];
+                            const float p0 = ex2f(sa.x - m), p1 = ex2f(sa.y - m), p2 = ex2f(sb.x - m), p3 = ex2f(sb.y - m);
+                            lsum[nt] += (p0 + p1) + (p2 + p3);
+                            split_bf16x2(p0, p1, bhi[nt][0], blo[nt][0]);
+                            split_bf16x2(p2, p3, bhi[nt][1], blo[nt][1]);
+                        }
                     }
                     const int mat = lane >> 3, r = lane & 7;
-                    const int krow = wq * 32 + ks * 16 + (mat & 1) * 8 + r;
+                    const int krow = wq * 32 + ks * 16 + (mat >> 1) * 8 + r;
 #pragma unroll
-                    for (int np = 0; np < 8; ++np) {
-                        const int ch = np * 2 + (mat >> 1);
+                    for (int db = 0; db < 8; ++db) {
+                        const int ch = db * 2 + (mat & 1);
                         const uint32_t addr = vbase + (uint32_t)((ch >> 3) * (kStageBytes / 2) + krow * 128 + (((ch & 7) ^ (krow & 7)) << 4));
-                        uint32_t bf[4];
-                        ldmatrix_x4_trans(addr, bf);
-                        mma_bf16_16816(acc[2 * np], ahi, bf[0], bf[1]);
-                        mma_bf16_16816(acc[2 * np], alo, bf[0], bf[1]);
-                        mma_bf16_16816(acc[2 * np + 1], ahi, bf[2], bf[3]);
-                        mma_bf16_16816(acc[2 * np + 1], alo, bf[2], bf[3]);
+                        uint32_t af[4];
+                        ldmatrix_x4_trans(addr, af);      // V^T fragment: rows = 16 d, columns = 16 keys
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            mma_bf16_16816(acc[nt][db], af, bhi[nt][0], bhi[nt][1]);
+                            mma_bf16_16816(acc[nt][db], af, blo[nt][0], blo[nt][1]);
+                        }
                     }
                 }
                 group_sync(bar_id, kGroupThreads);           // every warp has read its rows of the V tile
@@ -554,48 +629,64 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 ++jl;
             }
             if (!ok) break;
+            seg_tiles += nown;
 
-            // ---- group partial (max, denominator, un-normalised output) -> global
-            const int part = x.sp * 2 + b;
-            float *pml = a.part_ml + ((size_t)u * a.splits + part) * G * 2;
-            float *po = a.part_o + ((size_t)u * a.splits + part) * G * kD;
-            if (nown > 0) {
-                float *red = region;     // [4 warps][G][128]; the kept logits are no longer needed
-                lsum0 += __shfl_xor_sync(0xffffffffu, lsum0, 1);
-                lsum0 += __shfl_xor_sync(0xffffffffu, lsum0, 2);
-                lsum1 += __shfl_xor_sync(0xffffffffu, lsum1, 1);
-                lsum1 += __shfl_xor_sync(0xffffffffu, lsum1, 2);
-                if (tig == 0 && g0 < G) lred[wq * kMaxGroup + g0] = lsum0;
-                if (G > 8 && tig == 0 && g0 + 8 < G) lred[wq * kMaxGroup + g0 + 8] = lsum1;
+            // ---- close the segment when the unit's items in this CTA are done
+            if (w.last_of_unit_here(x)) {
+                int my_first;
+                const int nseg = w.segments(u, my_first);
+                const int slot = my_first + b;
+                float *pml = a.part_ml + ((size_t)u * a.splits + slot) * G * 2;
+                float *po = a.part_o + ((size_t)u * a.splits + slot) * G * kD;
+                if (seg_tiles > 0) {
+                    float *red = region;     // [4 warps][G][128]; the kept logits are no longer needed
 #pragma unroll
-                for (int nt = 0; nt < 16; ++nt) {
-                    if (g0 < G) *reinterpret_cast<float2 *>(red + (wq * G + g0) * kD + nt * 8 + tig * 2) = make_float2(acc[nt][0], acc[nt][1]);
-                    if (G > 8 && g0 + 8 < G)
-                        *reinterpret_cast<float2 *>(red + (wq * G + g0 + 8) * kD + nt * 8 + tig * 2) = make_float2(acc[nt][2], acc[nt][3]);
+                    for (int nt = 0; nt < NT; ++nt) {
+                        float l = lsum[nt];
+                        l += __shfl_xor_sync(0xffffffffu, l, 1);
+                        l += __shfl_xor_sync(0xffffffffu, l, 2);
+                        const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
+                        if (tig == 0 && gr < G) lred[wq * kMaxGroup + gr] = l;
+#pragma unroll
+                        for (int db = 0; db < 8; ++db) {
+                            if (gc < G) {
+                                red[(wq * G + gc) * kD + db * 16 + gid] = acc[nt][db][0];
+                                red[(wq * G + gc) * kD + db * 16 + gid + 8] = acc[nt][db][2];
+                            }
+                            if (gc + 1 < G) {
+                                red[(wq * G + gc + 1) * kD + db * 16 + gid] = acc[nt][db][1];
+                                red[(wq * G + gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3];
+                            }
+                        }
+                    }
+                    group_sync(bar_id, kGroupThreads);
+                    for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
+                        po[idx] = (red[idx] + red[G * kD + idx]) + (red[2 * G * kD + idx] + red[3 * G * kD + idx]);
+                    if (gtid < G) {
+                        pml[gtid * 2] = mrun[gtid];
+                        pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
+                    }
+                } else {
+                    for (int idx = gtid; idx < G * kD; idx += kGroupThreads) po[idx] = 0.f;
+                    if (gtid < G) { pml[gtid * 2] = -INFINITY; pml[gtid * 2 + 1] = 0.f; }
+                }
+                // publish: the group's writes are ordered before the ticket by the barrier plus one
+                // device-scope fence of the thread that takes the ticket
+                group_sync(bar_id, kGroupThreads);
+                if (gtid == 0) {
+                    __threadfence();
+                    const int last = atomicAdd(&a.ticket[u], 1) == nseg - 1;
+                    if (last) __threadfence();
+                    *flag = last;
                 }
                 group_sync(bar_id, kGroupThreads);
-                for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
-                    po[idx] = (red[idx] + red[G * kD + idx]) + (red[2 * G * kD + idx] + red[3 * G * kD + idx]);
-                if (gtid < G) {
-                    pml[gtid * 2] = mloc[gtid];
-                    pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
-                }
-            } else {
-                for (int idx = gtid; idx < G * kD; idx += kGroupThreads) po[idx] = 0.f;
-                if (gtid < G) { pml[gtid * 2] = -INFINITY; pml[gtid * 2 + 1] = 0.f; }
+                if (*flag) finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, nseg, evict, fin_sm, gtid, kGroupThreads, bar_id);
+                group_sync(bar_id, kGroupThreads);
+                seg_unit = -1;
             }
-            __threadfence();
-            group_sync(bar_id, kGroupThreads);
-            const int active2 = 2 * w.active_items();
-            if (gtid == 0) *flag = (atomicAdd(&a.ticket[u], 1) == active2 - 1);
-            group_sync(bar_id, kGroupThreads);
-            if (*flag) {
-                __threadfence();
-                finalize_unit<__nv_bfloat16, kD>(a, u, t, n, active2, evict, fin_sm, gtid, kGroupThreads, bar_id);
-            }
-            group_sync(bar_id, kGroupThreads);
             w.advance(x, nu);
         }
+        (void)seg_unit;
     }
 
     // ------------------------------------------------ tail
