@@ -87,10 +87,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     if (tc_ok && p->kernel != MKV_KERNEL_SIMT) {
         *kind = kKindTc;
         const int ntiles = (s->cap + 127) / 128;
-        const int tpg_max = 32 / s->G < 1 ? 1 : 32 / s->G;
-        const int min_ipu = (ntiles + 2 * tpg_max - 1) / (2 * tpg_max);
         int ipu = p->splits > 0 ? p->splits : tc_items_per_unit(s->U, s->cap, s->G, 148);
-        if (ipu < min_ipu) ipu = min_ipu;
         if (ipu > ntiles) ipu = ntiles;
         s->ipu = ipu;
         s->splits = 2 * ipu;          // every item leaves one partial per compute group

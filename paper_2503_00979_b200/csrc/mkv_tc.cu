@@ -2,19 +2,23 @@
 // R*G (padded to a multiple of 32) at most 256.
 //
 // A persistent, warp-specialised CTA per SM walks a static list of work items; an item is a
-// run of 128-key tiles of one unit's cache.
-//   warp 0       TMA producer: the unit's recent-query ring once per unit, then the item's K
-//                tiles and V tiles (cp.async.bulk.tensor, 128-byte swizzle) into one ring of
-//                32 KB stages guarded by mbarriers.
+// run of 128-key tiles of one unit's cache.  Per tile the K rows feed the scoring contraction
+// and the V rows the attention output; both are read from HBM exactly once.
+//   warp 0       TMA producer of the unit's recent-query ring (once per unit) and of K tiles
+//                (cp.async.bulk.tensor, 128-byte swizzle) into a short ring of 32 KB stages.
 //   warp 1       writes the new query over the ring row that leaves the window, then issues
 //                tcgen05.mma: S^T[128 keys x R*G rows] = K_tile . Q^T, fp32 accumulators in
-//                TMEM (one key per TMEM lane), two accumulator buffers.
-//   warps 2-9    two compute groups of four warps; group b owns TMEM buffer b and every second
-//                tile.  K phase: tcgen05.ld of a key's R*G logits, frozen soft-max weights
-//                exp2(s*scale - c_row), GQA group sum, window fusion (Eq. 4-6, Algorithm 1);
-//                the new row's logits are kept.  V phase: soft-max of the new row over the
-//                group's keys and P.V with mma.sync (P split in two bf16 terms), Eq. 1.
-//   The group that takes a unit's last ticket runs the shared per-unit epilogue (Eq. 7).
+//                TMEM (one key per TMEM lane), up to four accumulator buffers, so K stages are
+//                released as soon as their MMA has run.
+//   warp 2       TMA producer of V tiles into their own ring of stages.
+//   warps 3-10   two compute groups of four warps; tiles alternate between the groups and
+//                each warp owns the 32 keys of its TMEM lane quarter.  Per tile: tcgen05.ld of
+//                a key's R*G logits, frozen soft-max weights exp2(s*scale - c_row), GQA group
+//                sum, window fusion (Eq. 4-6, Algorithm 1); then the new row's soft-max is
+//                continued online (running max per head, rescale) and P.V for the warp's keys
+//                runs on mma.sync with P split in two bf16 terms (Eq. 1).  Warps only meet at
+//                mbarriers; a group synchronises once per unit to publish its partial.
+//   The group that takes a unit's last ticket runs the per-unit epilogue (Eq. 7).
 // Every mbarrier wait is bounded; a wait that runs out sets a device error flag and the CTA
 // drains and exits.
 #include <cuda.h>
@@ -33,37 +37,41 @@ namespace {
 constexpr int kD = 128;
 constexpr int kTile = 128;                  // keys per tile = MMA M = TMEM lanes
 constexpr int kStageBytes = 2 * kTile * 128;   // one K or V tile: two 64-column boxes
-constexpr int kThreadsTc = 32 * 10;
+constexpr int kWarpsTc = 11;
+constexpr int kThreadsTc = 32 * kWarpsTc;
+constexpr int kFirstComputeWarp = 3;
 constexpr int kGroupThreads = 128;
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds
+constexpr int kFinFloats = 4 * kMaxGroup + 128 + 256 + 64 + 32 + 8;   // per-group epilogue scratch
 
 struct TcGeom {
     int rgpad;          // ring rows padded to a multiple of 32 (MMA N)
     int ipu;            // work items per unit
-    int stages;         // K/V stages in shared memory
-    int tpg;            // most tiles one compute group takes from one item
+    int sk, sv;         // K stages, V stages
+    int nb;             // TMEM accumulator buffers (even)
     int tmem_cols;      // allocated TMEM columns (power of two)
-    int region_bytes;   // per-group scratch: kept logits of the new row / output reduction
+    int red_bytes;      // per-group scratch for the output reduction at publish time
     int grid;
     int smem_bytes;
 };
 
 struct SmemLayout {
-    int q, stages, region, negc, small, bars, total;
+    int q, kst, vst, red, negc, stw, small, bars, total;
 };
 
-__host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g)
+__host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g, int G)
 {
     SmemLayout L;
     int o = 0;
     L.q = o; o += g.rgpad * 256;
-    L.stages = o; o += g.stages * kStageBytes;
-    L.region = o; o += 2 * g.region_bytes;
-    L.negc = o; o += 2 * g.rgpad * 4;
-    L.small = o; o += 2 * (4 * kMaxGroup * 4 /*gm*/ + 4 * kMaxGroup * 4 /*lred*/ + kMaxGroup * 4 /*mloc*/ +
-                           kFinalizeSmemFloats * 4 + 16);
+    L.kst = o; o += g.sk * kStageBytes;
+    L.vst = o; o += g.sv * kStageBytes;
+    L.red = o; o += 2 * g.red_bytes;
+    L.negc = o; o += 2 * g.rgpad * 4;                 // one copy per compute group
+    L.stw = o; o += 8 * (G * 32 + 2 * kMaxGroup) * 4; // per warp: kept logits of one tile, rescale factors, reference
+    L.small = o; o += 2 * (8 * kMaxGroup + kFinFloats + 4) * 4;
     o = (o + 15) & ~15;
-    L.bars = o; o += 8 * (2 * 8 + 8) + 64;
+    L.bars = o; o += 8 * 40;
     L.total = o;
     return L;
 }
@@ -245,12 +253,11 @@ struct Item {
     int unit, sp, tile0, nk;
 };
 struct Walk {     // the same deterministic walk over this CTA's items in every role
-    long long it, it_end;
+    long long it, it_end, total;
     int ipu, tpi, ntiles;
     int prev_unit;
     int qseq;         // units seen so far (ring loads)
-    int L0, T0;       // running load / tile sequence numbers
-    long long total;
+    int T0;           // running tile sequence number
     __device__ Walk(const TcGeom &g, int U, int n)
     {
         total = (long long)U * g.ipu;
@@ -260,8 +267,9 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
         ipu = g.ipu;
         ntiles = (n + kTile - 1) / kTile;
         tpi = (ntiles + ipu - 1) / ipu;
-        prev_unit = -1; qseq = 0; L0 = 0; T0 = 0;
+        prev_unit = -1; qseq = 0; T0 = 0;
     }
+    __device__ int active_items() const { return (ntiles + tpi - 1) / tpi; }
     // A unit's active items may spread over several CTAs; each CTA's share is one *segment* per
     // compute group.  Returns the number of segments of unit u and this CTA's first slot.
     __device__ int segments(int u, int &my_first) const
@@ -270,14 +278,6 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
         const int c0 = (int)(i0 * gridDim.x / total), c1 = (int)(i1 * gridDim.x / total);
         my_first = ((int)blockIdx.x - c0) * 2;
         return 2 * (c1 - c0 + 1);
-    }
-    // true if the next item with work (if any) belongs to another unit
-    __device__ bool last_of_unit_here(const Item &x) const
-    {
-        const long long nxt = (long long)x.unit * ipu + x.sp + 1;     // == it after next()
-        if (nxt >= it_end) return true;
-        if (nxt / ipu != x.unit) return true;
-        return (int)(nxt % ipu) * tpi >= ntiles;                       // remaining items of this unit are empty
     }
     // next item with work; new_unit tells whether the ring must be (re)loaded
     __device__ bool next(Item &x, bool &new_unit)
@@ -296,13 +296,19 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
         }
         return false;
     }
+    // true if the next item with work (if any) belongs to another unit
+    __device__ bool last_of_unit_here(const Item &x) const
+    {
+        const long long nxt = (long long)x.unit * ipu + x.sp + 1;     // == it after next()
+        if (nxt >= it_end) return true;
+        if (nxt / ipu != x.unit) return true;
+        return (int)(nxt % ipu) * tpi >= ntiles;                       // the unit's remaining items are empty
+    }
     __device__ void advance(const Item &x, bool new_unit)
     {
-        L0 += 2 * x.nk;
         T0 += x.nk;
         if (new_unit) ++qseq;
     }
-    __device__ int active_items() const { return (ntiles + tpi - 1) / tpi; }
 };
 
 template <int G, int FUSION>
@@ -329,6 +335,176 @@ __device__ __forceinline__ void score_chunk(const uint32_t (&v)[32], const float
     }
 }
 
+// Per-unit epilogue for a compute group of 128 threads (same result as finalize_unit): merge the
+// segments' partials, write the attention output, add the new row's term to the fused scores,
+// evict the minimum, append (Eq. 1 merge, Eq. 4-7).  All loads of a phase are issued together, so
+// the whole epilogue costs a few L2 round trips.  Requires nseg <= 8 and nseg*G*2 <= 256.
+template <int G>
+__device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, int nseg, bool evict, float *sm, int tid,
+                              int bar_id)
+{
+    constexpr int NT_ = kGroupThreads;
+    const int lane = tid & 31, warp = tid >> 5;
+    float *s_self = sm, *mfin = sm + kMaxGroup, *lfin = sm + 2 * kMaxGroup, *cnew = sm + 3 * kMaxGroup;
+    float *vsm = sm + 4 * kMaxGroup;                       // [128] new value row as floats
+    float *pml_s = vsm + 128;                              // [nseg][G][2]
+    unsigned long long *red_key = reinterpret_cast<unsigned long long *>(pml_s + 256);   // [32]
+    int *red_slot = reinterpret_cast<int *>(pml_s + 256 + 64);                           // [32]
+
+    const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(a.q) + (size_t)u * G * kD;
+    const __nv_bfloat16 *kn = static_cast<const __nv_bfloat16 *>(a.k_new) + (size_t)u * kD;
+    const __nv_bfloat16 *vn = static_cast<const __nv_bfloat16 *>(a.v_new) + (size_t)u * kD;
+    const float *pml = a.part_ml + (size_t)u * a.splits * G * 2;
+    const float *po = a.part_o + (size_t)u * a.splits * G * kD;
+
+    // ---- phase A: every load that does not depend on another one
+    constexpr int QCH = (G * 16 + NT_ - 1) / NT_;          // 16-byte chunks of q per thread
+    uint4 qv[QCH], kv[QCH];
+#pragma unroll
+    for (int i = 0; i < QCH; ++i) {
+        const int c = tid + i * NT_;
+        if (c < G * 16) {
+            qv[i] = reinterpret_cast<const uint4 *>(q)[c];
+            kv[i] = reinterpret_cast<const uint4 *>(kn)[c & 15];
+        }
+    }
+    uint4 vv = make_uint4(0, 0, 0, 0);
+    if (tid < 16) vv = reinterpret_cast<const uint4 *>(vn)[tid];
+    for (int i = tid; i < nseg * G * 2; i += NT_) pml_s[i] = __ldcg(pml + i);
+    float pov[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp) pov[g][sp] = sp < nseg ? __ldcg(po + (sp * G + g) * kD + tid) : 0.f;
+
+    // self logit: 8-element partial dots, reduced over the 16 threads that share a head
+#pragma unroll
+    for (int i = 0; i < QCH; ++i) {
+        const int c = tid + i * NT_;
+        float acc = 0.f;
+        if (c < G * 16) {
+            const uint32_t *qa = reinterpret_cast<const uint32_t *>(&qv[i]), *ka = reinterpret_cast<const uint32_t *>(&kv[i]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc += __uint_as_float(qa[e] << 16) * __uint_as_float(ka[e] << 16);
+                acc += __uint_as_float(qa[e] & 0xffff0000u) * __uint_as_float(ka[e] & 0xffff0000u);
+            }
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (c < G * 16 && (c & 15) == 0) s_self[c >> 4] = acc * a.scale2;
+    }
+    if (tid < 16) {
+        const uint32_t *va = reinterpret_cast<const uint32_t *>(&vv);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            vsm[tid * 8 + 2 * e] = __uint_as_float(va[e] << 16);
+            vsm[tid * 8 + 2 * e + 1] = __uint_as_float(va[e] & 0xffff0000u);
+        }
+    }
+    group_sync(bar_id, NT_);
+
+    // ---- phase B: merged soft-max statistics, attention output
+    if (tid < G) {
+        float m = s_self[tid];
+        for (int sp = 0; sp < nseg; ++sp) m = fmaxf(m, pml_s[(sp * G + tid) * 2]);
+        float l = exp2f(s_self[tid] - m);
+        for (int sp = 0; sp < nseg; ++sp) l += pml_s[(sp * G + tid) * 2 + 1] * exp2f(pml_s[(sp * G + tid) * 2] - m);
+        mfin[tid] = m;
+        lfin[tid] = l;
+        cnew[tid] = m + log2f(l);
+    }
+    group_sync(bar_id, NT_);
+    __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(a.out) + (size_t)u * G * kD;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const float m = mfin[g];
+        float o = exp2f(s_self[g] - m) * vsm[tid];
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp)
+            if (sp < nseg) o += pov[g][sp] * exp2f(pml_s[(sp * G + g) * 2] - m);
+        out[g * kD + tid] = __float2bfloat16_rn(o / lfin[g]);
+    }
+
+    // ---- phase C: final fused scores and the eviction (Algorithm 1 / Eq. 7)
+    int *pos = a.pos + (size_t)u * a.cap;
+    float *F = a.F + (size_t)u * a.cap;
+    int e_slot = n, e_pos = -1;
+    if (evict) {
+        const float *sn = a.s_new + (size_t)u * G * a.cap;
+        const long long thr = t - a.R;
+        float cn[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) cn[g] = cnew[g];
+        unsigned long long best = ~0ull;
+        int bslot = -1;
+        constexpr int B = 8;          // slots per thread and round, all their loads in flight together
+        for (int kb = tid; kb < n; kb += B * NT_) {
+            int p[B];
+            float f0[B], x[G][B];
+#pragma unroll
+            for (int b = 0; b < B; ++b) {
+                const int k = kb + b * NT_;
+                p[b] = k < n ? pos[k] : 0x7fffffff;
+                f0[b] = k < n ? __ldcg(F + k) : 0.f;
+#pragma unroll
+                for (int g = 0; g < G; ++g) x[g][b] = k < n ? __ldcg(sn + (size_t)g * a.cap + k) : -INFINITY;
+            }
+#pragma unroll
+            for (int b = 0; b < B; ++b) {
+                const int k = kb + b * NT_;
+                if (k >= n) continue;
+                if ((long long)p[b] <= thr) {
+                    float s = 0.f;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) s += exp2f(x[g][b] - cn[g]);
+                    const float f = fuse(a.fusion, f0[b], s);
+                    F[k] = f;
+                    const unsigned long long key = rank_key(__float_as_uint(f), p[b]);
+                    if (key < best) { best = key; bslot = k; }
+                } else {
+                    F[k] = -1.f;   // window slot: not a candidate
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+            const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+            if (ok < best) { best = ok; bslot = os; }
+        }
+        if (lane == 0) { red_key[warp] = best; red_slot[warp] = bslot; }
+        group_sync(bar_id, NT_);
+        best = red_key[0]; bslot = red_slot[0];
+#pragma unroll
+        for (int w = 1; w < NT_ / 32; ++w)
+            if (red_key[w] < best) { best = red_key[w]; bslot = red_slot[w]; }
+        e_slot = bslot;
+        e_pos = (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull));   // the rank key carries the position
+    }
+
+    // ---- phase D: Eq. 7 update from the registers loaded in phase A
+    __nv_bfloat16 *Kd = static_cast<__nv_bfloat16 *>(a.K) + ((size_t)u * a.cap + e_slot) * kD;
+    __nv_bfloat16 *Vd = static_cast<__nv_bfloat16 *>(a.V) + ((size_t)u * a.cap + e_slot) * kD;
+    if (tid < 16) {
+        reinterpret_cast<uint4 *>(Kd)[tid] = kv[0];
+        reinterpret_cast<uint4 *>(Vd)[tid] = vv;
+    }
+    const int rs = (int)(t % a.R);
+    __nv_bfloat16 *rq = static_cast<__nv_bfloat16 *>(a.ring_q) + ((size_t)u * a.R + rs) * G * kD;
+#pragma unroll
+    for (int i = 0; i < QCH; ++i) {
+        const int c = tid + i * NT_;
+        if (c < G * 16) reinterpret_cast<uint4 *>(rq)[c] = qv[i];
+    }
+    if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
+    if (tid == 0) {
+        pos[e_slot] = (int)t;
+        a.evicted_pos[u] = e_pos;
+        a.ticket[u] = 0;
+    }
+}
+
 template <int G, int FUSION>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmK,
@@ -339,17 +515,17 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     // the swizzled operand tiles need a 1024-byte aligned base; the launch asks for 1 KB of slack
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const SmemLayout L = tc_smem_layout(geo);
-    const int S = geo.stages, RGP = geo.rgpad;
+    const SmemLayout L = tc_smem_layout(geo, G);
+    const int SK = geo.sk, SV = geo.sv, NB = geo.nb, RGP = geo.rgpad;
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t q_addr = sbase + L.q, st_addr = sbase + L.stages;
+    const uint32_t q_addr = sbase + L.q, kst_addr = sbase + L.kst, vst_addr = sbase + L.vst;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
-    // barrier indices
-    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + 8);
-    const uint32_t bar_tfull = smem_u32(bars + 16), bar_tempty = smem_u32(bars + 18);
-    const uint32_t bar_qfull = smem_u32(bars + 20), bar_qempty = smem_u32(bars + 21);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 22);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 23);
+    const uint32_t bar_kfull = smem_u32(bars), bar_kempty = smem_u32(bars + 4);
+    const uint32_t bar_vfull = smem_u32(bars + 8), bar_vempty = smem_u32(bars + 16);
+    const uint32_t bar_tfull = smem_u32(bars + 24), bar_tempty = smem_u32(bars + 28);
+    const uint32_t bar_qfull = smem_u32(bars + 32), bar_qempty = smem_u32(bars + 33);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 34);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 35);
 
     const long long t = a.st->t;
     const int n = a.st->n;
@@ -357,8 +533,9 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const int rs_new = (int)(t % a.R);
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        for (int s = 0; s < SK; ++s) { mbar_init(bar_kfull + 8 * s, 1); mbar_init(bar_kempty + 8 * s, 1); }
+        for (int s = 0; s < SV; ++s) { mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_vempty + 8 * s, 4); }
+        for (int b = 0; b < NB; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
         mbar_init(bar_qfull, 1);
         mbar_init(bar_qempty, 1);
         *abort_flag = 0;
@@ -371,7 +548,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------ TMA producer (one lane)
+        // ------------------------------------------------ TMA producer: query ring and K tiles (one lane)
         if (lane == 0) {
             Walk w(geo, a.U, n);
             Item x; bool nu;
@@ -385,24 +562,48 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
                     tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
                 }
-                for (int j = 0; j < 2 * x.nk && ok; ++j) {
-                    const int Ls = w.L0 + j, s = Ls % S;
-                    ok = mbar_wait(bar_empty + 8 * s, (uint32_t)(((Ls / S) & 1) ^ 1), abort_flag);
+                for (int j = 0; j < x.nk && ok; ++j) {
+                    const int T = w.T0 + j, s = T % SK;
+                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(((T / SK) & 1) ^ 1), abort_flag);
                     if (!ok) break;
-                    const CUtensorMap *map = j < x.nk ? &tmK : &tmV;
-                    const int row = (x.tile0 + (j < x.nk ? j : j - x.nk)) * kTile;
-                    mbar_expect_tx(bar_full + 8 * s, kStageBytes);
-                    tma_load_3d(st_addr + s * kStageBytes, map, 0, row, x.unit, bar_full + 8 * s);
-                    tma_load_3d(st_addr + s * kStageBytes + kStageBytes / 2, map, 64, row, x.unit, bar_full + 8 * s);
-                    issued = Ls + 1;
+                    const int row = (x.tile0 + j) * kTile;
+                    mbar_expect_tx(bar_kfull + 8 * s, kStageBytes);
+                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, x.unit, bar_kfull + 8 * s);
+                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, x.unit, bar_kfull + 8 * s);
+                    issued = T + 1;
+                }
+                w.advance(x, nu);
+            }
+            if (!ok) {   // give up: let the copies already in flight land before the CTA exits
+                int dummy = 0;
+                for (int T = max(0, issued - SK); T < issued; ++T)
+                    mbar_wait(bar_kfull + 8 * (T % SK), (uint32_t)((T / SK) & 1), &dummy);
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------ TMA producer: V tiles (one lane)
+        if (lane == 0) {
+            Walk w(geo, a.U, n);
+            Item x; bool nu;
+            int issued = 0;
+            bool ok = true;
+            while (ok && w.next(x, nu)) {
+                for (int j = 0; j < x.nk && ok; ++j) {
+                    const int T = w.T0 + j, s = T % SV;
+                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(((T / SV) & 1) ^ 1), abort_flag);
+                    if (!ok) break;
+                    const int row = (x.tile0 + j) * kTile;
+                    mbar_expect_tx(bar_vfull + 8 * s, kStageBytes);
+                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, x.unit, bar_vfull + 8 * s);
+                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, x.unit, bar_vfull + 8 * s);
+                    issued = T + 1;
                 }
                 w.advance(x, nu);
             }
             if (!ok) {
-                // give up: let the copies already in flight land before the CTA exits
                 int dummy = 0;
-                for (int Ls = max(0, issued - S); Ls < issued; ++Ls)
-                    mbar_wait(bar_full + 8 * (Ls % S), (uint32_t)((Ls / S) & 1), &dummy);
+                for (int T = max(0, issued - SV); T < issued; ++T)
+                    mbar_wait(bar_vfull + 8 * (T % SV), (uint32_t)((T / SV) & 1), &dummy);
             }
         }
     } else if (warp == 1) {
@@ -435,9 +636,9 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 __syncwarp();
             }
             for (int j = 0; j < x.nk; ++j) {
-                const int Ls = w.L0 + j, s = Ls % S, T = w.T0 + j, b = T & 1;
-                bool k = mbar_wait(bar_full + 8 * s, (uint32_t)((Ls / S) & 1), abort_flag);
-                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(((T >> 1) & 1) ^ 1), abort_flag);
+                const int T = w.T0 + j, s = T % SK, b = T % NB;
+                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)((T / SK) & 1), abort_flag);
+                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(((T / NB) & 1) ^ 1), abort_flag);
                 ok = __all_sync(0xffffffffu, k);
                 if (!ok) break;
                 tc_fence_after();
@@ -445,11 +646,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     const uint32_t d_tmem = tmem_base + (uint32_t)(b * RGP);
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint64_t ad = smem_desc_sw128(st_addr + s * kStageBytes + (ks >> 2) * (kStageBytes / 2) + (ks & 3) * 32);
+                        const uint64_t ad = smem_desc_sw128(kst_addr + s * kStageBytes + (ks >> 2) * (kStageBytes / 2) + (ks & 3) * 32);
                         const uint64_t bd = smem_desc_sw128(q_addr + (ks >> 2) * (RGP * 128) + (ks & 3) * 32);
                         umma_bf16(d_tmem, ad, bd, idesc, ks > 0 ? 1u : 0u);
                     }
-                    umma_commit(bar_empty + 8 * s);       // K tile consumed
+                    umma_commit(bar_kempty + 8 * s);      // K tile consumed
                     umma_commit(bar_tfull + 8 * b);       // accumulators ready
                 }
                 __syncwarp();
@@ -458,64 +659,67 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------ compute groups
-        const int b = (warp - 2) >> 2;          // group = TMEM buffer
-        const int wq = warp & 3;                // TMEM lane quarter of this warp
-        const int gtid = wq * 32 + lane;
-        const int bar_id = 1 + b;
-        float *region = reinterpret_cast<float *>(smem + L.region + b * geo.region_bytes);
-        float *negc = reinterpret_cast<float *>(smem + L.negc) + b * RGP;
-        float *small = reinterpret_cast<float *>(smem + L.small) + b * (9 * kMaxGroup + kFinalizeSmemFloats + 4);
-        float *gm = small, *lred = small + 4 * kMaxGroup, *mrun = small + 8 * kMaxGroup;
-        float *fin_sm = small + 9 * kMaxGroup;              // 8-byte aligned: 9*16 floats = 576 bytes
-        int *flag = reinterpret_cast<int *>(fin_sm + kFinalizeSmemFloats);
-        float *st_w = region + wq * (geo.tpg * G * 32);     // this warp's kept logits [tile][g][lane]
+        const int cw = warp - kFirstComputeWarp;     // 0..7
+        const int grp = cw >> 2;                     // tiles alternate between the two groups
+        const int wq = warp & 3;                     // TMEM lane quarter of this warp
+        const int gtid = wq * 32 + lane;             // position among the group's 128 key lanes
+        const int bar_id = 1 + grp;
+        float *red = reinterpret_cast<float *>(smem + L.red + grp * geo.red_bytes);
+        float *negc = reinterpret_cast<float *>(smem + L.negc) + grp * RGP;
+        float *st_w = reinterpret_cast<float *>(smem + L.stw) + cw * (G * 32 + 2 * kMaxGroup);   // [g][lane]
+        float *fac = st_w + G * 32, *mref = fac + kMaxGroup;         // warp-private, indexed by head
+        float *small = reinterpret_cast<float *>(smem + L.small) + grp * (8 * kMaxGroup + kFinFloats + 4);
+        float *gm = small, *lred = small + 4 * kMaxGroup;            // [4 warps][head]
+        float *fin_sm = small + 8 * kMaxGroup;
+        int *flag = reinterpret_cast<int *>(fin_sm + kFinFloats);
         const int RG = a.R * G;
         const int gid = lane >> 2, tig = lane & 3;
-        constexpr int NT = G > 8 ? 2 : 1;                   // 8-head column tiles of the transposed output
+        constexpr int NT = G > 8 ? 2 : 1;            // 8-head column tiles of the transposed output
 
-        // Running soft-max state of the open segment (consecutive items of one unit): the
-        // reference max per head in shared memory, this thread's share of the denominator and
-        // of the un-normalised output O^T[d][g] in registers.
+        // Running soft-max state of this warp over its keys of the open segment: reference max
+        // per head (replicated in every lane), this lane's share of the denominator and of the
+        // un-normalised output O^T[d][g].
+        float mrun[G];
         float acc[NT][8][4];
         float lsum[NT];
-        int seg_unit = -1, seg_tiles = 0;
+        int seg_tiles = 0;
 
         Walk w(geo, a.U, n);
         Item x; bool nu;
         bool ok = true;
-        while (ok && w.next(x, nu)) {
+        while (w.next(x, nu)) {
             const int u = x.unit;
             if (nu) {
                 // frozen normalisers of the ring rows, negated; the new row and padding give weight 0
+                // (the group's warps all passed the previous unit's publish barriers, so nobody reads the old table)
                 for (int c = gtid; c < RGP; c += kGroupThreads) {
                     float v = -INFINITY;
                     if (c < RG && c / G != rs_new) v = -a.ring_c[(size_t)u * RG + c];
                     negc[c] = v;
                 }
-                if (gtid < G) mrun[gtid] = -INFINITY;
+#pragma unroll
+                for (int g = 0; g < G; ++g) mrun[g] = -INFINITY;
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     lsum[nt] = 0.f;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
                 }
-                seg_unit = u; seg_tiles = 0;
+                seg_tiles = 0;
                 group_sync(bar_id, kGroupThreads);
             }
-            float mx[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) mx[g] = -INFINITY;
-            int nown = 0;
             float *s_new = a.s_new + (size_t)u * G * a.cap;
-            // ---- K phase: this group's tiles
-            for (int j = 0; j < x.nk; ++j) {
+            for (int j = 0; j < x.nk && ok; ++j) {
                 const int T = w.T0 + j;
-                if ((T & 1) != b) continue;
-                if (group_any(bar_id, !mbar_wait(bar_tfull + 8 * b, (uint32_t)((T >> 1) & 1), abort_flag))) { ok = false; break; }
+                if ((T & 1) != grp) continue;
+                const int buf = T % NB;
+                // ---- scores of this warp's 32 keys (Eq. 4-6) and the new row's logits
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)((T / NB) & 1), abort_flag));
+                if (!ok) break;
                 tc_fence_after();
                 const int key = (x.tile0 + j) * kTile + gtid;
                 const bool valid = key < n;
-                const uint32_t taddr = tmem_base + (uint32_t)(b * RGP) + ((uint32_t)(wq * 32) << 16);
+                const uint32_t taddr = tmem_base + (uint32_t)(buf * RGP) + ((uint32_t)(wq * 32) << 16);
                 uint32_t sv[G];
                 tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
                 float F = 0.f;
@@ -539,59 +743,40 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 tc_tie<G>(sv);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_tempty + 8 * b);
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                if (evict && valid) a.F[(size_t)u * a.cap + key] = F;
+
+                // ---- online soft-max of the new row over this warp's keys (Eq. 1)
+                bool changed = false;
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     const float s2 = valid ? __uint_as_float(sv[g]) * a.scale2 : -INFINITY;
-                    st_w[(nown * G + g) * 32 + lane] = s2;
+                    st_w[g * 32 + lane] = s2;
                     if (valid) s_new[(size_t)g * a.cap + key] = s2;
-                    mx[g] = fmaxf(mx[g], s2);
+                    const float mn = fmaxf(mrun[g], warp_max(s2));
+                    // factor that brings what was accumulated under the old reference to the new one
+                    const float f = mn == mrun[g] ? 1.f : ex2f(mrun[g] - mn);
+                    changed |= mn != mrun[g];
+                    mrun[g] = mn;
+                    if (lane == 0) { fac[g] = f; mref[g] = mn == -INFINITY ? 0.f : mn; }
                 }
-                if (evict && valid) a.F[(size_t)u * a.cap + key] = F;
-                ++nown;
-            }
-            if (!ok) break;
-
-            // ---- new reference max of the segment; rescale what has been accumulated so far
+                __syncwarp();
+                if (changed && seg_tiles > 0) {
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const float m = warp_max(mx[g]);
-                if (lane == 0) gm[wq * kMaxGroup + g] = m;
-            }
-            group_sync(bar_id, kGroupThreads);
-            float mnew_row[NT], mnew_c0[NT], mnew_c1[NT];
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
+                        const float fr = gr < G ? fac[gr] : 0.f, f0 = gc < G ? fac[gc] : 0.f, f1 = gc + 1 < G ? fac[gc + 1] : 0.f;
+                        lsum[nt] *= fr;
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                // heads this thread needs: row gid (+8 nt) for P, columns tig*2, tig*2+1 (+8 nt) of O^T
-                const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
-                auto mnew = [&](int g) {
-                    return fmaxf(fmaxf(mrun[g], fmaxf(gm[g], gm[kMaxGroup + g])), fmaxf(gm[2 * kMaxGroup + g], gm[3 * kMaxGroup + g]));
-                };
-                mnew_row[nt] = gr < G ? mnew(gr) : 0.f;
-                mnew_c0[nt] = gc < G ? mnew(gc) : 0.f;
-                mnew_c1[nt] = gc + 1 < G ? mnew(gc + 1) : 0.f;
-                if (seg_tiles > 0 && nown > 0) {
-                    const float fr = gr < G ? ex2f(mrun[gr] - mnew_row[nt]) : 0.f;
-                    const float f0 = gc < G ? ex2f(mrun[gc] - mnew_c0[nt]) : 0.f;
-                    const float f1 = gc + 1 < G ? ex2f(mrun[gc + 1] - mnew_c1[nt]) : 0.f;
-                    lsum[nt] *= fr;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) { acc[nt][i][0] *= f0; acc[nt][i][1] *= f1; acc[nt][i][2] *= f0; acc[nt][i][3] *= f1; }
+                        for (int i = 0; i < 8; ++i) { acc[nt][i][0] *= f0; acc[nt][i][1] *= f1; acc[nt][i][2] *= f0; acc[nt][i][3] *= f1; }
+                    }
                 }
-            }
-            group_sync(bar_id, kGroupThreads);         // everyone has read the old reference
-            if (gtid < G && nown > 0)
-                mrun[gtid] = fmaxf(fmaxf(mrun[gtid], fmaxf(gm[gtid], gm[kMaxGroup + gtid])),
-                                   fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
 
-            // ---- V phase: O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys of each tile
-            int jl = 0;
-            for (int j = 0; j < x.nk; ++j) {
-                const int T = w.T0 + j;
-                if ((T & 1) != b) continue;
-                const int Ls = w.L0 + x.nk + j, s = Ls % S;
-                if (group_any(bar_id, !mbar_wait(bar_full + 8 * s, (uint32_t)((Ls / S) & 1), abort_flag))) { ok = false; break; }
-                const uint32_t vbase = st_addr + s * kStageBytes;
+                // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys
+                const int s = T % SV;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_vfull + 8 * s, (uint32_t)((T / SV) & 1), abort_flag));
+                if (!ok) break;
+                const uint32_t vbase = vst_addr + s * kStageBytes;
 #pragma unroll
                 for (int ks = 0; ks < 2; ++ks) {
                     uint32_t bhi[NT][2], blo[NT][2];
@@ -600,9 +785,9 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                         bhi[nt][0] = bhi[nt][1] = blo[nt][0] = blo[nt][1] = 0u;
                         const int gr = gid + 8 * nt;
                         if (gr < G) {
-                            const float *sp = st_w + (jl * G + gr) * 32 + ks * 16 + tig * 2;
+                            const float *sp = st_w + gr * 32 + ks * 16 + tig * 2;
                             const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
-                            const float m = mnew_row[nt];
+                            const float m = mref[gr];
                             const float p0 = ex2f(sa.x - m), p1 = ex2f(sa.y - m), p2 = ex2f(sb.x - m), p3 = ex2f(sb.y - m);
                             lsum[nt] += (p0 + p1) + (p2 + p3);
                             split_bf16x2(p0, p1, bhi[nt][0], blo[nt][0]);
@@ -624,51 +809,68 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                         }
                     }
                 }
-                group_sync(bar_id, kGroupThreads);           // every warp has read its rows of the V tile
-                if (gtid == 0) mbar_arrive(bar_empty + 8 * s);
-                ++jl;
+                __syncwarp();                               // every lane has read its rows of the V tile
+                if (lane == 0) mbar_arrive(bar_vempty + 8 * s);
+                ++seg_tiles;
             }
-            if (!ok) break;
-            seg_tiles += nown;
 
             // ---- close the segment when the unit's items in this CTA are done
             if (w.last_of_unit_here(x)) {
+                if (group_any(bar_id, !ok)) { ok = false; break; }       // all four warps agree to go on
                 int my_first;
                 const int nseg = w.segments(u, my_first);
-                const int slot = my_first + b;
+                const int slot = my_first + grp;
                 float *pml = a.part_ml + ((size_t)u * a.splits + slot) * G * 2;
                 float *po = a.part_o + ((size_t)u * a.splits + slot) * G * kD;
-                if (seg_tiles > 0) {
-                    float *red = region;     // [4 warps][G][128]; the kept logits are no longer needed
+                // merge the four warps: common reference = max of theirs
+                if (lane == 0) {
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        float l = lsum[nt];
-                        l += __shfl_xor_sync(0xffffffffu, l, 1);
-                        l += __shfl_xor_sync(0xffffffffu, l, 2);
-                        const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
-                        if (tig == 0 && gr < G) lred[wq * kMaxGroup + gr] = l;
+                    for (int g = 0; g < G; ++g) gm[wq * kMaxGroup + g] = mrun[g];
+                }
+                group_sync(bar_id, kGroupThreads);
 #pragma unroll
-                        for (int db = 0; db < 8; ++db) {
-                            if (gc < G) {
-                                red[(wq * G + gc) * kD + db * 16 + gid] = acc[nt][db][0];
-                                red[(wq * G + gc) * kD + db * 16 + gid + 8] = acc[nt][db][2];
-                            }
-                            if (gc + 1 < G) {
-                                red[(wq * G + gc + 1) * kD + db * 16 + gid] = acc[nt][db][1];
-                                red[(wq * G + gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3];
-                            }
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
+                    auto gmax = [&](int g) {
+                        return fmaxf(fmaxf(gm[g], gm[kMaxGroup + g]), fmaxf(gm[2 * kMaxGroup + g], gm[3 * kMaxGroup + g]));
+                    };
+                    auto scale = [&](int g) {     // this warp's reference -> the group's
+                        const float mw = gm[wq * kMaxGroup + g];
+                        return mw == -INFINITY ? 0.f : ex2f(mw - gmax(g));
+                    };
+                    float l = lsum[nt];
+                    l += __shfl_xor_sync(0xffffffffu, l, 1);
+                    l += __shfl_xor_sync(0xffffffffu, l, 2);
+                    if (tig == 0 && gr < G) lred[wq * kMaxGroup + gr] = l * scale(gr);
+                    const float f0 = gc < G ? scale(gc) : 0.f, f1 = gc + 1 < G ? scale(gc + 1) : 0.f;
+#pragma unroll
+                    for (int db = 0; db < 8; ++db) {
+                        if (gc < G) {
+                            red[(wq * G + gc) * kD + db * 16 + gid] = acc[nt][db][0] * f0;
+                            red[(wq * G + gc) * kD + db * 16 + gid + 8] = acc[nt][db][2] * f0;
+                        }
+                        if (gc + 1 < G) {
+                            red[(wq * G + gc + 1) * kD + db * 16 + gid] = acc[nt][db][1] * f1;
+                            red[(wq * G + gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3] * f1;
                         }
                     }
-                    group_sync(bar_id, kGroupThreads);
-                    for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
-                        po[idx] = (red[idx] + red[G * kD + idx]) + (red[2 * G * kD + idx] + red[3 * G * kD + idx]);
-                    if (gtid < G) {
-                        pml[gtid * 2] = mrun[gtid];
-                        pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
-                    }
-                } else {
-                    for (int idx = gtid; idx < G * kD; idx += kGroupThreads) po[idx] = 0.f;
-                    if (gtid < G) { pml[gtid * 2] = -INFINITY; pml[gtid * 2 + 1] = 0.f; }
+                }
+                // the segment's state is spent (the next item starts a new unit)
+#pragma unroll
+                for (int g = 0; g < G; ++g) mrun[g] = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    lsum[nt] = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
+                }
+                seg_tiles = 0;
+                group_sync(bar_id, kGroupThreads);
+                for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
+                    po[idx] = (red[idx] + red[G * kD + idx]) + (red[2 * G * kD + idx] + red[3 * G * kD + idx]);
+                if (gtid < G) {
+                    pml[gtid * 2] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
+                    pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
                 }
                 // publish: the group's writes are ordered before the ticket by the barrier plus one
                 // device-scope fence of the thread that takes the ticket
@@ -680,13 +882,16 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     *flag = last;
                 }
                 group_sync(bar_id, kGroupThreads);
-                if (*flag) finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, nseg, evict, fin_sm, gtid, kGroupThreads, bar_id);
+                if (*flag) {
+                    if (nseg <= 8 && nseg * G * 2 <= 256)
+                        finalize_fast<G>(a, u, t, n, nseg, evict, fin_sm, gtid, bar_id);
+                    else
+                        finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, nseg, evict, fin_sm, gtid, kGroupThreads, bar_id);
+                }
                 group_sync(bar_id, kGroupThreads);
-                seg_unit = -1;
             }
             w.advance(x, nu);
         }
-        (void)seg_unit;
     }
 
     // ------------------------------------------------ tail
@@ -773,22 +978,22 @@ bool tc_shape_supported(bool f32, int D, int G, int R)
     return pad32(R * G) <= 256;
 }
 
-// Items per unit: enough that one item's tiles fit the per-group scratch, then the count that
-// fills whole waves of the persistent grid best (ties: fewer, larger items).
+// Items per unit: the count that fills whole waves of the persistent grid best (ties: fewer,
+// larger items).  Items are scheduling quanta only; consecutive items of a unit in one CTA
+// are accumulated into one partial.
 int tc_items_per_unit(int U, int cap, int G, int n_sm)
 {
+    (void)G;
     const int ntiles = (cap + kTile - 1) / kTile;
-    const int tpg_max = 32 / G < 1 ? 1 : 32 / G;
-    const int min_ipu = (ntiles + 2 * tpg_max - 1) / (2 * tpg_max);
-    int best = min_ipu;
+    int best = 1;
     double best_eff = -1.0;
-    for (int ipu = min_ipu; ipu <= ntiles; ++ipu) {
+    for (int ipu = 1; ipu <= ntiles; ++ipu) {
         const int tpi = (ntiles + ipu - 1) / ipu;
-        if (tpi < 2 && ipu > min_ipu) break;
+        if (tpi < 2 && ipu > 1) break;
         const long long items = (long long)U * ((ntiles + tpi - 1) / tpi);
         const long long waves = (items + n_sm - 1) / n_sm;
         // time ~ waves * tiles per item (+ a fixed cost per item)
-        const double cost = (double)waves * (tpi + 0.35);
+        const double cost = (double)waves * (tpi + 0.25);
         const double eff = (double)U * ntiles / (cost * n_sm);
         if (eff > best_eff + 1e-9) { best_eff = eff; best = ipu; }
     }
@@ -810,24 +1015,23 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err
     const int G = a.G;
     g.rgpad = pad32(a.R * G);
     g.ipu = ipu;
-    const int ntiles = (a.cap + kTile - 1) / kTile;
-    const int tpi = (ntiles + ipu - 1) / ipu;
-    g.tpg = (tpi + 1) / 2;
-    g.tmem_cols = 64;
-    while (g.tmem_cols < 2 * g.rgpad) g.tmem_cols *= 2;
-    const int stw = 4 * g.tpg * G * 32 * 4, red = 4 * G * kD * 4;
-    g.region_bytes = ((stw > red ? stw : red) + 127) & ~127;
+    g.nb = g.rgpad <= 128 ? 4 : 2;
+    g.tmem_cols = 32;
+    while (g.tmem_cols < g.nb * g.rgpad) g.tmem_cols *= 2;
+    g.red_bytes = (4 * G * kD * 4 + 127) & ~127;
     const long long items = (long long)a.U * ipu;
     g.grid = (int)(items < n_sm ? items : n_sm);
-    for (g.stages = 6; g.stages >= 2; --g.stages) {
-        g.smem_bytes = tc_smem_layout(g).total + 1024;
+    g.sk = 2;
+    for (g.sv = 8; g.sv >= 2; --g.sv) {
+        g.smem_bytes = tc_smem_layout(g, G).total + 1024;
         if (g.smem_bytes <= max_smem) break;
     }
-    if (g.stages < 2 || g.stages > 8) {
+    if (g.sv < 2) {
         snprintf(err, err_len, "tensor-core kernel: shared memory does not fit (need %d bytes)", g.smem_bytes);
         delete p;
         return cudaErrorInvalidConfiguration;
     }
+    if (g.sv >= 6) { g.sk = 3; g.sv -= 1; g.smem_bytes = tc_smem_layout(g, G).total + 1024; }
     if (!encode_map(&p->tmK, a.K, a.U, a.cap, kTile) || !encode_map(&p->tmV, a.V, a.U, a.cap, kTile) ||
         !encode_map(&p->tmQ, a.ring_q, a.U, a.R * G, g.rgpad)) {
         snprintf(err, err_len, "tensor-core kernel: cuTensorMapEncodeTiled failed");
