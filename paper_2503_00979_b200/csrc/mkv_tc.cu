@@ -77,6 +77,7 @@ __host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g, int G)
 }
 
 // ---------------------------------------------------------------- PTX helpers
+// (tmem_ld32 / tmem_ld_n include the tcgen05.wait::ld that makes their registers valid)
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -134,23 +135,6 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// wait for outstanding tcgen05.ld; the registers are operands so that no use of them can be
-// scheduled before the wait
-__device__ __forceinline__ void tc_wait_ld32(uint32_t (&v)[32])
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
-                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
-                   "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
-                   "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
-                 :: "memory");
-}
-template <int N> __device__ __forceinline__ void tc_tie(uint32_t (&v)[N])
-{
-#pragma unroll
-    for (int i = 0; i < N; ++i) asm volatile("" : "+r"(v[i]));
-}
-
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
 {
     asm volatile(
@@ -173,7 +157,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+        "tcgen05.wait::ld.sync.aligned;"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
           "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
           "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
@@ -183,27 +168,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
 template <int N> __device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&v)[N]);
 template <> __device__ __forceinline__ void tmem_ld_n<1>(uint32_t taddr, uint32_t (&v)[1])
 {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v[0]) : "r"(taddr) : "memory");
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\ntcgen05.wait::ld.sync.aligned;" : "=r"(v[0]) : "r"(taddr) : "memory");
 }
 template <> __device__ __forceinline__ void tmem_ld_n<2>(uint32_t taddr, uint32_t (&v)[2])
 {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];" : "=r"(v[0]), "=r"(v[1]) : "r"(taddr) : "memory");
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];\ntcgen05.wait::ld.sync.aligned;" : "=r"(v[0]), "=r"(v[1]) : "r"(taddr) : "memory");
 }
 template <> __device__ __forceinline__ void tmem_ld_n<4>(uint32_t taddr, uint32_t (&v)[4])
 {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\ntcgen05.wait::ld.sync.aligned;"
                  : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(taddr) : "memory");
 }
 template <> __device__ __forceinline__ void tmem_ld_n<8>(uint32_t taddr, uint32_t (&v)[8])
 {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\ntcgen05.wait::ld.sync.aligned;"
                  : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                  : "r"(taddr) : "memory");
 }
 template <> __device__ __forceinline__ void tmem_ld_n<16>(uint32_t taddr, uint32_t (&v)[16])
 {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        "tcgen05.wait::ld.sync.aligned;"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
           "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr) : "memory");
@@ -720,27 +706,18 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 const int key = (x.tile0 + j) * kTile + gtid;
                 const bool valid = key < n;
                 const uint32_t taddr = tmem_base + (uint32_t)(buf * RGP) + ((uint32_t)(wq * 32) << 16);
+                // Each TMEM load and its wait form one asm statement: the destination registers are
+                // written asynchronously, so nothing may touch them between the two.
                 uint32_t sv[G];
                 tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
                 float F = 0.f;
                 if (evict) {
-                    // chunk c+1 is in flight while chunk c is turned into weights
-                    uint32_t v[2][32];
-                    const int nch = RGP >> 5;
-                    tmem_ld32(taddr, v[0]);
-                    tc_wait_ld32(v[0]);
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        if (c < nch) {
-                            if (c + 1 < nch) tmem_ld32(taddr + (uint32_t)((c + 1) * 32), v[(c + 1) & 1]);
-                            score_chunk<G, FUSION>(v[c & 1], negc + c * 32, a.scale2, F);
-                            if (c + 1 < nch) tc_wait_ld32(v[(c + 1) & 1]);
-                        }
+                    for (int c = 0; c < RGP; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + (uint32_t)c, v);
+                        score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
                     }
-                } else {
-                    tc_wait_ld();
                 }
-                tc_tie<G>(sv);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
@@ -872,16 +849,13 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     pml[gtid * 2] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
                     pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
                 }
-                // publish: the group's writes are ordered before the ticket by the barrier plus one
-                // device-scope fence of the thread that takes the ticket
+                // publish: every thread makes its own writes visible device-wide, then one thread
+                // takes the ticket (a fence by the ticket thread alone proved insufficient here)
+                __threadfence();
                 group_sync(bar_id, kGroupThreads);
-                if (gtid == 0) {
-                    __threadfence();
-                    const int last = atomicAdd(&a.ticket[u], 1) == nseg - 1;
-                    if (last) __threadfence();
-                    *flag = last;
-                }
+                if (gtid == 0) *flag = atomicAdd(&a.ticket[u], 1) == nseg - 1;
                 group_sync(bar_id, kGroupThreads);
+                if (*flag) __threadfence();
                 if (*flag) {
                     if (nseg <= 8 && nseg * G * 2 <= 256)
                         finalize_fast<G>(a, u, t, n, nseg, evict, fin_sm, gtid, bar_id);
@@ -1021,17 +995,20 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err
     g.red_bytes = (4 * G * kD * 4 + 127) & ~127;
     const long long items = (long long)a.U * ipu;
     g.grid = (int)(items < n_sm ? items : n_sm);
-    g.sk = 2;
-    for (g.sv = 8; g.sv >= 2; --g.sv) {
-        g.smem_bytes = tc_smem_layout(g, G).total + 1024;
-        if (g.smem_bytes <= max_smem) break;
+    // as many 32 KB stages as fit, split between the K ring (short-lived tiles) and the V ring
+    int total_stages = 0;
+    for (int st = 9; st >= 3; --st) {
+        g.sk = 1; g.sv = st - 1;
+        if (tc_smem_layout(g, G).total + 1024 <= max_smem) { total_stages = st; break; }
     }
-    if (g.sv < 2) {
-        snprintf(err, err_len, "tensor-core kernel: shared memory does not fit (need %d bytes)", g.smem_bytes);
+    if (total_stages < 3) {
+        snprintf(err, err_len, "tensor-core kernel: shared memory does not fit");
         delete p;
         return cudaErrorInvalidConfiguration;
     }
-    if (g.sv >= 6) { g.sk = 3; g.sv -= 1; g.smem_bytes = tc_smem_layout(g, G).total + 1024; }
+    g.sk = total_stages >= 7 ? 3 : total_stages >= 4 ? 2 : 1;
+    g.sv = total_stages - g.sk;
+    g.smem_bytes = tc_smem_layout(g, G).total + 1024;
     if (!encode_map(&p->tmK, a.K, a.U, a.cap, kTile) || !encode_map(&p->tmV, a.V, a.U, a.cap, kTile) ||
         !encode_map(&p->tmQ, a.ring_q, a.U, a.R * G, g.rgpad)) {
         snprintf(err, err_len, "tensor-core kernel: cuTensorMapEncodeTiled failed");
