@@ -90,7 +90,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
         int ipu = p->splits > 0 ? p->splits : tc_items_per_unit(s->U, s->cap, s->G, 148);
         if (ipu > ntiles) ipu = ntiles;
         s->ipu = ipu;
-        s->splits = 2 * ipu;          // every item leaves one partial per compute group
+        s->splits = tc_groups(s->R, s->G) * ipu;     // every item leaves one partial per compute group
         return true;
     }
     *kind = kKindSimt;

@@ -37,8 +37,8 @@ namespace {
 constexpr int kD = 128;
 constexpr int kTile = 128;                  // keys per tile = MMA M = TMEM lanes
 constexpr int kStageBytes = 2 * kTile * 128;   // one K or V tile: two 64-column boxes
-constexpr int kWarpsTc = 11;
-constexpr int kThreadsTc = 32 * kWarpsTc;
+constexpr int kMaxComputeGroups = 3;
+__host__ __device__ constexpr int tc_threads(int ng) { return 32 * (3 + 4 * ng); }   // 3 service warps + 4 per group
 constexpr int kFirstComputeWarp = 3;
 constexpr int kGroupThreads = 128;
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds
@@ -48,7 +48,8 @@ struct TcGeom {
     int rgpad;          // ring rows padded to a multiple of 32 (MMA N)
     int ipu;            // work items per unit
     int sk, sv;         // K stages, V stages
-    int nb;             // TMEM accumulator buffers (even)
+    int ng;             // compute groups (2 or 3); tile T belongs to group T % ng
+    int nb;             // TMEM accumulator buffers (a multiple of ng)
     int tmem_cols;      // allocated TMEM columns (power of two)
     int red_bytes;      // per-group scratch for the output reduction at publish time
     int grid;
@@ -66,12 +67,12 @@ __host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g, int G)
     L.q = o; o += g.rgpad * 256;
     L.kst = o; o += g.sk * kStageBytes;
     L.vst = o; o += g.sv * kStageBytes;
-    L.red = o; o += 2 * g.red_bytes;
-    L.negc = o; o += 2 * g.rgpad * 4;                 // one copy per compute group
-    L.stw = o; o += 8 * (G * 32 + 2 * kMaxGroup) * 4; // per warp: kept logits of one tile, rescale factors, reference
-    L.small = o; o += 2 * (8 * kMaxGroup + kFinFloats + 4) * 4;
+    L.red = o; o += g.ng * g.red_bytes;
+    L.negc = o; o += g.ng * g.rgpad * 4;              // one copy per compute group
+    L.stw = o; o += 4 * g.ng * (G * 32 + 2 * kMaxGroup) * 4; // per warp: kept logits of one tile, rescale factors, reference
+    L.small = o; o += g.ng * (8 * kMaxGroup + kFinFloats + 4) * 4;
     o = (o + 15) & ~15;
-    L.bars = o; o += 8 * 40;
+    L.bars = o; o += 8 * 48;
     L.total = o;
     return L;
 }
@@ -258,12 +259,12 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
     __device__ int active_items() const { return (ntiles + tpi - 1) / tpi; }
     // A unit's active items may spread over several CTAs; each CTA's share is one *segment* per
     // compute group.  Returns the number of segments of unit u and this CTA's first slot.
-    __device__ int segments(int u, int &my_first) const
+    __device__ int segments(int u, int ng, int &my_first) const
     {
         const long long i0 = (long long)u * ipu, i1 = i0 + active_items() - 1;
         const int c0 = (int)(i0 * gridDim.x / total), c1 = (int)(i1 * gridDim.x / total);
-        my_first = ((int)blockIdx.x - c0) * 2;
-        return 2 * (c1 - c0 + 1);
+        my_first = ((int)blockIdx.x - c0) * ng;
+        return ng * (c1 - c0 + 1);
     }
     // next item with work; new_unit tells whether the ring must be (re)loaded
     __device__ bool next(Item &x, bool &new_unit)
@@ -491,8 +492,8 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     }
 }
 
-template <int G, int FUSION>
-__global__ void __launch_bounds__(kThreadsTc, 1)
+template <int G, int FUSION, int NG>
+__global__ void __launch_bounds__(tc_threads(NG), 1)
 decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ TcGeom geo)
@@ -508,10 +509,10 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     const uint32_t bar_kfull = smem_u32(bars), bar_kempty = smem_u32(bars + 4);
     const uint32_t bar_vfull = smem_u32(bars + 8), bar_vempty = smem_u32(bars + 16);
-    const uint32_t bar_tfull = smem_u32(bars + 24), bar_tempty = smem_u32(bars + 28);
-    const uint32_t bar_qfull = smem_u32(bars + 32), bar_qempty = smem_u32(bars + 33);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 34);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 35);
+    const uint32_t bar_tfull = smem_u32(bars + 24), bar_tempty = smem_u32(bars + 32);
+    const uint32_t bar_qfull = smem_u32(bars + 40), bar_qempty = smem_u32(bars + 41);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 42);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 43);
 
     const long long t = a.st->t;
     const int n = a.st->n;
@@ -645,8 +646,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------ compute groups
-        const int cw = warp - kFirstComputeWarp;     // 0..7
-        const int grp = cw >> 2;                     // tiles alternate between the two groups
+        const int cw = warp - kFirstComputeWarp;     // 0 .. 4*NG-1
+        const int grp = cw >> 2;                     // tile T belongs to group T % NG
         const int wq = warp & 3;                     // TMEM lane quarter of this warp
         const int gtid = wq * 32 + lane;             // position among the group's 128 key lanes
         const int bar_id = 1 + grp;
@@ -697,7 +698,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             float *s_new = a.s_new + (size_t)u * G * a.cap;
             for (int j = 0; j < x.nk && ok; ++j) {
                 const int T = w.T0 + j;
-                if ((T & 1) != grp) continue;
+                if (T % NG != grp) continue;
                 const int buf = T % NB;
                 // ---- scores of this warp's 32 keys (Eq. 4-6) and the new row's logits
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)((T / NB) & 1), abort_flag));
@@ -795,7 +796,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             if (w.last_of_unit_here(x)) {
                 if (group_any(bar_id, !ok)) { ok = false; break; }       // all four warps agree to go on
                 int my_first;
-                const int nseg = w.segments(u, my_first);
+                const int nseg = w.segments(u, NG, my_first);
                 const int slot = my_first + grp;
                 float *pml = a.part_ml + ((size_t)u * a.splits + slot) * G * 2;
                 float *po = a.part_o + ((size_t)u * a.splits + slot) * G * kD;
@@ -819,19 +820,37 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     l += __shfl_xor_sync(0xffffffffu, l, 1);
                     l += __shfl_xor_sync(0xffffffffu, l, 2);
                     if (tig == 0 && gr < G) lred[wq * kMaxGroup + gr] = l * scale(gr);
+                    // bring this warp's accumulators to the group's reference
                     const float f0 = gc < G ? scale(gc) : 0.f, f1 = gc + 1 < G ? scale(gc + 1) : 0.f;
 #pragma unroll
-                    for (int db = 0; db < 8; ++db) {
-                        if (gc < G) {
-                            red[(wq * G + gc) * kD + db * 16 + gid] = acc[nt][db][0] * f0;
-                            red[(wq * G + gc) * kD + db * 16 + gid + 8] = acc[nt][db][2] * f0;
-                        }
-                        if (gc + 1 < G) {
-                            red[(wq * G + gc + 1) * kD + db * 16 + gid] = acc[nt][db][1] * f1;
-                            red[(wq * G + gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3] * f1;
+                    for (int db = 0; db < 8; ++db) { acc[nt][db][0] *= f0; acc[nt][db][1] *= f1; acc[nt][db][2] *= f0; acc[nt][db][3] *= f1; }
+                }
+                // four warps -> one output through a two-slot buffer: warps 2, 3 store; warps 0, 1 add
+                // theirs and store the sums; everybody adds the two slots
+                auto red_io = [&](bool store) {
+                    float *slot_ = red + (wq & 1) * G * kD;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int gc = tig * 2 + 8 * nt;
+#pragma unroll
+                        for (int db = 0; db < 8; ++db) {
+                            float *p0 = slot_ + gc * kD + db * 16 + gid, *p1 = slot_ + (gc + 1) * kD + db * 16 + gid;
+                            if (gc < G) {
+                                if (store) { p0[0] = acc[nt][db][0]; p0[8] = acc[nt][db][2]; }
+                                else { acc[nt][db][0] += p0[0]; acc[nt][db][2] += p0[8]; }
+                            }
+                            if (gc + 1 < G) {
+                                if (store) { p1[0] = acc[nt][db][1]; p1[8] = acc[nt][db][3]; }
+                                else { acc[nt][db][1] += p1[0]; acc[nt][db][3] += p1[8]; }
+                            }
                         }
                     }
-                }
+                };
+                if (wq >= 2) red_io(true);
+                group_sync(bar_id, kGroupThreads);
+                if (wq < 2) red_io(false);
+                group_sync(bar_id, kGroupThreads);
+                if (wq < 2) red_io(true);
                 // the segment's state is spent (the next item starts a new unit)
 #pragma unroll
                 for (int g = 0; g < G; ++g) mrun[g] = -INFINITY;
@@ -844,7 +863,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 seg_tiles = 0;
                 group_sync(bar_id, kGroupThreads);
                 for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
-                    po[idx] = (red[idx] + red[G * kD + idx]) + (red[2 * G * kD + idx] + red[3 * G * kD + idx]);
+                    po[idx] = red[idx] + red[G * kD + idx];
                 if (gtid < G) {
                     pml[gtid * 2] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
                     pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
@@ -915,25 +934,31 @@ bool encode_map(CUtensorMap *m, void *base, int units, int rows, int box_rows)
 struct TcPlan {
     CUtensorMap tmK, tmV, tmQ;
     TcGeom geo;
-    bool attr_set[5][2];
+    bool attr_set[5][2][2];
 };
 
 namespace {
 
 int group_index(int G) { return G == 1 ? 0 : G == 2 ? 1 : G == 4 ? 2 : G == 8 ? 3 : G == 16 ? 4 : -1; }
 
-template <int G, int FUSION>
-cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
+template <int G, int FUSION, int NG>
+cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    auto kern = decode_tc_kernel<G, FUSION>;
-    bool &set = plan->attr_set[group_index(G)][FUSION];
+    auto kern = decode_tc_kernel<G, FUSION, NG>;
+    bool &set = plan->attr_set[group_index(G)][FUSION][NG - 2];
     if (!set) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan->geo.smem_bytes);
         if (e != cudaSuccess) return e;
         set = true;
     }
-    kern<<<plan->geo.grid, kThreadsTc, plan->geo.smem_bytes, stream>>>(a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
+    kern<<<plan->geo.grid, tc_threads(NG), plan->geo.smem_bytes, stream>>>(a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
     return cudaGetLastError();
+}
+
+template <int G, int FUSION>
+cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
+{
+    return plan->geo.ng == 3 ? launch_gfn<G, FUSION, 3>(plan, a, stream) : launch_gfn<G, FUSION, 2>(plan, a, stream);
 }
 
 template <int G>
@@ -945,6 +970,9 @@ cudaError_t launch_g(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 int pad32(int x) { return (x + 31) & ~31; }
 
 }  // namespace
+
+// three compute groups when three accumulator buffers fit the 512 TMEM columns, else two
+int tc_groups(int R, int G) { return pad32(R * G) <= 128 ? 3 : 2; }
 
 bool tc_shape_supported(bool f32, int D, int G, int R)
 {
@@ -989,10 +1017,11 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err
     const int G = a.G;
     g.rgpad = pad32(a.R * G);
     g.ipu = ipu;
-    g.nb = g.rgpad <= 128 ? 4 : 2;
+    g.ng = tc_groups(a.R, G);
+    g.nb = g.ng == 3 ? (g.rgpad <= 64 ? 6 : 3) : (g.rgpad <= 128 ? 4 : 2);
     g.tmem_cols = 32;
     while (g.tmem_cols < g.nb * g.rgpad) g.tmem_cols *= 2;
-    g.red_bytes = (4 * G * kD * 4 + 127) & ~127;
+    g.red_bytes = (2 * G * kD * 4 + 127) & ~127;
     const long long items = (long long)a.U * ipu;
     g.grid = (int)(items < n_sm ? items : n_sm);
     // as many 32 KB stages as fit, split between the K ring (short-lived tiles) and the V ring
