@@ -89,6 +89,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
         const int ntiles = (s->cap + 127) / 128;
         int ipu = p->splits > 0 ? p->splits : tc_items_per_unit(s->U, s->cap, s->G, 148);
         if (ipu > ntiles) ipu = ntiles;
+        while (ipu > 1 && (long long)s->U * ipu > (1ll << 30)) --ipu;     // item indices stay 32-bit
         s->ipu = ipu;
         s->splits = tc_groups(s->R, s->G) * ipu;     // every item leaves one partial per compute group
         return true;

@@ -240,18 +240,22 @@ struct Item {
     int unit, sp, tile0, nk;
 };
 struct Walk {     // the same deterministic walk over this CTA's items in every role
-    long long it, it_end, total;
+    int it, it_end;   // item indices (the host keeps U * ipu below 2^31)
+    int unit, sp;     // unit and split index of item `it`, kept incrementally (no divisions per item)
     int ipu, tpi, ntiles;
     int prev_unit;
     int qseq;         // units seen so far (ring loads)
     int T0;           // running tile sequence number
+    long long total;
     __device__ Walk(const TcGeom &g, int U, int n)
     {
         total = (long long)U * g.ipu;
         // item i belongs to CTA (i * grid) / total, so CTA c owns [ceil(c*total/grid), ceil((c+1)*total/grid))
-        it = (total * blockIdx.x + gridDim.x - 1) / gridDim.x;
-        it_end = (total * (blockIdx.x + 1) + gridDim.x - 1) / gridDim.x;
+        it = (int)((total * blockIdx.x + gridDim.x - 1) / gridDim.x);
+        it_end = (int)((total * (blockIdx.x + 1) + gridDim.x - 1) / gridDim.x);
         ipu = g.ipu;
+        unit = it / ipu;
+        sp = it - unit * ipu;
         ntiles = (n + kTile - 1) / kTile;
         tpi = (ntiles + ipu - 1) / ipu;
         prev_unit = -1; qseq = 0; T0 = 0;
@@ -270,11 +274,12 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
     __device__ bool next(Item &x, bool &new_unit)
     {
         while (it < it_end) {
-            x.unit = (int)(it / ipu);
-            x.sp = (int)(it % ipu);
-            x.tile0 = x.sp * tpi;
+            x.unit = unit;
+            x.sp = sp;
+            x.tile0 = sp * tpi;
             x.nk = min(tpi, ntiles - x.tile0);
             ++it;
+            if (++sp == ipu) { sp = 0; ++unit; }
             if (x.nk > 0) {
                 new_unit = x.unit != prev_unit;
                 prev_unit = x.unit;
@@ -283,13 +288,12 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
         }
         return false;
     }
-    // true if the next item with work (if any) belongs to another unit
+    // true if the next item with work (if any) belongs to another unit; (unit, sp) already
+    // describe the item after x
     __device__ bool last_of_unit_here(const Item &x) const
     {
-        const long long nxt = (long long)x.unit * ipu + x.sp + 1;     // == it after next()
-        if (nxt >= it_end) return true;
-        if (nxt / ipu != x.unit) return true;
-        return (int)(nxt % ipu) * tpi >= ntiles;                       // the unit's remaining items are empty
+        if (it >= it_end || unit != x.unit) return true;
+        return sp * tpi >= ntiles;                       // the unit's remaining items are empty
     }
     __device__ void advance(const Item &x, bool new_unit)
     {
