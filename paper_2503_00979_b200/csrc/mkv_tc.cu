@@ -20,7 +20,9 @@
 //                mbarriers; a group synchronises once per unit to publish its partial.
 //   The group that takes a unit's last ticket runs the per-unit epilogue (Eq. 7).
 // Every mbarrier wait is bounded; a wait that runs out sets a device error flag and the CTA
-// drains and exits.
+// drains and exits.  Warp-collective .aligned instructions (ldmatrix, mma.sync, tcgen05.ld)
+// are only reached with the whole warp converged: the code before them is branch-free or
+// ends in a warp-level sync.
 #include <cuda.h>
 #include <stdio.h>
 #include <string.h>
@@ -302,6 +304,18 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
     }
 };
 
+// position in a ring of n slots (stage or accumulator buffer) and the parity of the lap,
+// advanced without divisions
+struct RingPos {
+    int idx, lap;
+    __device__ RingPos(int start, int n) : idx(start % n), lap((start / n) & 1) {}
+    __device__ __forceinline__ void step(int by, int n)
+    {
+        idx += by;
+        while (idx >= n) { idx -= n; lap ^= 1; }
+    }
+};
+
 template <int G, int FUSION>
 __device__ __forceinline__ void score_chunk(const uint32_t (&v)[32], const float *negc, float scale2, float &F)
 {
@@ -545,6 +559,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             Item x; bool nu;
             int issued = 0;
             bool ok = true;
+            RingPos rk(0, SK);
             while (ok && w.next(x, nu)) {
                 if (nu) {
                     ok = mbar_wait(bar_qempty, (uint32_t)((w.qseq & 1) ^ 1), abort_flag);
@@ -553,9 +568,9 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
                     tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
                 }
-                for (int j = 0; j < x.nk && ok; ++j) {
-                    const int T = w.T0 + j, s = T % SK;
-                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(((T / SK) & 1) ^ 1), abort_flag);
+                for (int j = 0; j < x.nk && ok; ++j, rk.step(1, SK)) {
+                    const int T = w.T0 + j, s = rk.idx;
+                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(rk.lap ^ 1), abort_flag);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_kfull + 8 * s, kStageBytes);
@@ -578,10 +593,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             Item x; bool nu;
             int issued = 0;
             bool ok = true;
+            RingPos rv(0, SV);
             while (ok && w.next(x, nu)) {
-                for (int j = 0; j < x.nk && ok; ++j) {
-                    const int T = w.T0 + j, s = T % SV;
-                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(((T / SV) & 1) ^ 1), abort_flag);
+                for (int j = 0; j < x.nk && ok; ++j, rv.step(1, SV)) {
+                    const int T = w.T0 + j, s = rv.idx;
+                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_vfull + 8 * s, kStageBytes);
@@ -603,6 +619,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         Item x; bool nu;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RGP >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
         bool ok = true;
+        RingPos rk(0, SK), rb(0, NB);
         while (ok && w.next(x, nu)) {
             if (nu) {
                 if (w.qseq > 0 && lane == 0) umma_commit(bar_qempty);   // MMAs of the previous unit done with the ring
@@ -626,10 +643,10 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 fence_proxy_async();
                 __syncwarp();
             }
-            for (int j = 0; j < x.nk; ++j) {
-                const int T = w.T0 + j, s = T % SK, b = T % NB;
-                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)((T / SK) & 1), abort_flag);
-                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(((T / NB) & 1) ^ 1), abort_flag);
+            for (int j = 0; j < x.nk; ++j, rk.step(1, SK), rb.step(1, NB)) {
+                const int s = rk.idx, b = rb.idx;
+                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)rk.lap, abort_flag);
+                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(rb.lap ^ 1), abort_flag);
                 ok = __all_sync(0xffffffffu, k);
                 if (!ok) break;
                 tc_fence_after();
@@ -678,6 +695,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         Walk w(geo, a.U, n);
         Item x; bool nu;
         bool ok = true;
+        int Tn = grp;                                  // next tile of this group
+        RingPos rb(grp, NB), rv(grp, SV);
         while (w.next(x, nu)) {
             const int u = x.unit;
             if (nu) {
@@ -700,12 +719,12 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 group_sync(bar_id, kGroupThreads);
             }
             float *s_new = a.s_new + (size_t)u * G * a.cap;
-            for (int j = 0; j < x.nk && ok; ++j) {
-                const int T = w.T0 + j;
-                if (T % NG != grp) continue;
-                const int buf = T % NB;
+            // this group's tiles are T = grp, grp + NG, ...: walk them directly
+            for (; Tn < w.T0 + x.nk && ok; Tn += NG, rb.step(NG, NB), rv.step(NG, SV)) {
+                const int j = Tn - w.T0;
+                const int buf = rb.idx;
                 // ---- scores of this warp's 32 keys (Eq. 4-6) and the new row's logits
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)((T / NB) & 1), abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)rb.lap, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 const int key = (x.tile0 + j) * kTile + gtid;
@@ -755,8 +774,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 }
 
                 // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys
-                const int s = T % SV;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_vfull + 8 * s, (uint32_t)((T / SV) & 1), abort_flag));
+                const int s = rv.idx;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag));
                 if (!ok) break;
                 const uint32_t vbase = vst_addr + s * kStageBytes;
 #pragma unroll
@@ -764,18 +783,21 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     uint32_t bhi[NT][2], blo[NT][2];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        bhi[nt][0] = bhi[nt][1] = blo[nt][0] = blo[nt][1] = 0u;
+                        // branch-free on purpose: ldmatrix / mma.sync below are .aligned and need the
+                        // whole warp converged; lanes whose row is not a head compute and discard
                         const int gr = gid + 8 * nt;
-                        if (gr < G) {
-                            const float *sp = st_w + gr * 32 + ks * 16 + tig * 2;
-                            const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
-                            const float m = mref[gr];
-                            const float p0 = ex2f(sa.x - m), p1 = ex2f(sa.y - m), p2 = ex2f(sb.x - m), p3 = ex2f(sb.y - m);
-                            lsum[nt] += (p0 + p1) + (p2 + p3);
-                            split_bf16x2(p0, p1, bhi[nt][0], blo[nt][0]);
-                            split_bf16x2(p2, p3, bhi[nt][1], blo[nt][1]);
-                        }
+                        const bool live = gr < G;
+                        const int grc = live ? gr : 0;
+                        const float *sp = st_w + grc * 32 + ks * 16 + tig * 2;
+                        const float2 sa = *reinterpret_cast<const float2 *>(sp), sb = *reinterpret_cast<const float2 *>(sp + 8);
+                        const float m = mref[grc];
+                        float p0 = ex2f(sa.x - m), p1 = ex2f(sa.y - m), p2 = ex2f(sb.x - m), p3 = ex2f(sb.y - m);
+                        p0 = live ? p0 : 0.f; p1 = live ? p1 : 0.f; p2 = live ? p2 : 0.f; p3 = live ? p3 : 0.f;
+                        lsum[nt] += (p0 + p1) + (p2 + p3);
+                        split_bf16x2(p0, p1, bhi[nt][0], blo[nt][0]);
+                        split_bf16x2(p2, p3, bhi[nt][1], blo[nt][1]);
                     }
+                    __syncwarp();
                     const int mat = lane >> 3, r = lane & 7;
                     const int krow = wq * 32 + ks * 16 + (mat >> 1) * 8 + r;
 #pragma unroll
@@ -872,11 +894,18 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     pml[gtid * 2] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
                     pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
                 }
-                // publish: every thread makes its own writes visible device-wide, then one thread
-                // takes the ticket (a fence by the ticket thread alone proved insufficient here)
+                // publish.  Writers: every thread fences its own writes; after the group barrier the
+                // ticket thread fences again (cumulative over what the barrier made it observe) and
+                // only then increments the ticket.  Reader: the thread that saw the last ticket
+                // fences before the barrier that lets the group read the other segments.
                 __threadfence();
                 group_sync(bar_id, kGroupThreads);
-                if (gtid == 0) *flag = atomicAdd(&a.ticket[u], 1) == nseg - 1;
+                if (gtid == 0) {
+                    __threadfence();
+                    const int last = atomicAdd(&a.ticket[u], 1) == nseg - 1;
+                    __threadfence();
+                    *flag = last;
+                }
                 group_sync(bar_id, kGroupThreads);
                 if (*flag) __threadfence();
                 if (*flag) {
@@ -1039,7 +1068,7 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err
         delete p;
         return cudaErrorInvalidConfiguration;
     }
-    g.sk = total_stages >= 7 ? 3 : total_stages >= 4 ? 2 : 1;
+    g.sk = total_stages >= 7 ? 3 : total_stages >= 5 ? 2 : 1;
     g.sv = total_stages - g.sk;
     g.smem_bytes = tc_smem_layout(g, G).total + 1024;
     if (!encode_map(&p->tmK, a.K, a.U, a.cap, kTile) || !encode_map(&p->tmV, a.V, a.U, a.cap, kTile) ||

@@ -257,3 +257,28 @@ def test_tc_matches_cuda_core_kernel_on_device():
     assert torch.equal(res["simt"][1], res["tc"][1])
     assert (res["simt"][0] - res["tc"][0]).abs().max() <= 2 ** -6       # one bf16 ulp at |o| < 4
     assert torch.allclose(res["simt"][2], res["tc"][2], rtol=0, atol=2e-4)
+
+
+@pytest.mark.parametrize("ipu", [0, 1])
+def test_tc_runs_are_bitwise_reproducible(ipu):
+    # static work assignment and fixed merge order: two runs on the same inputs agree bit for bit
+    # (this caught a warp-divergence bug in front of ldmatrix / mma.sync that tolerances had hidden)
+    w = SMALL.replace(layers=1, batch=2, C=1500, R=32, prompt_len=1700, steps=40, fusion="max")
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    k, v = st.kv(np.arange(w.prompt_len))
+    qw = st.q(np.arange(w.prompt_len - w.R, w.prompt_len))
+    pos = np.arange(w.prompt_len, w.prompt_len + w.steps)
+    kk, vv = st.kv(pos)
+    qq = st.q(pos)
+    runs = []
+    for _ in range(3):
+        mk = binding.MorphKV(1, 2, 8, 2, 128, w.C, w.R, w.fusion, "bf16", kernel="tc", splits=ipu)
+        mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+        outs = [mk.decode_step(qq[:, :, :, i].bfloat16().contiguous(), kk[:, :, :, i].bfloat16().contiguous(),
+                               vv[:, :, :, i].bfloat16().contiguous()).clone() for i in range(w.steps)]
+        mk.sync()
+        runs.append((torch.stack(outs), mk.view(0)["pos"].clone(), mk.view(0)["ring_c"].clone()))
+        mk.close()
+    for r in runs[1:]:
+        assert torch.equal(r[0], runs[0][0]) and torch.equal(r[1], runs[0][1]) and torch.equal(r[2], runs[0][2])
