@@ -278,7 +278,7 @@ def run_ours(args, w):
         if world == 1 and not args.no_cpu_baseline:
             cores = len(os.sched_getaffinity(0))
             n_units = max(1, min(cores, w.units))
-            ups, used, sample, _ = oracle_throughput(synth.WORKLOADS[args.workload], n_units, args.cpu_steps)
+            ups, used, sample, _ = oracle_throughput(w.replace(seed=synth.WORKLOADS[args.workload].seed), n_units, args.cpu_steps)
             line["cpu_baseline"] = {"value": ups * w.batch / w.units, "unit": UNIT, "cores": used, "kind": "oracle",
                                     "sample": sample, "unit_steps_per_s": ups}
         print(json.dumps(line), flush=True)
@@ -297,12 +297,16 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--cpu-steps", type=int, default=512, help="steady-state steps per unit for the CPU baseline")
+    ap.add_argument("--prompt-len", type=int, default=0,
+                    help="override the workload's prompt length (e.g. C + R to start config 3 with a full cache)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer arm (for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     w = synth.WORKLOADS[args.workload]
+    if args.prompt_len > 0:
+        w = w.replace(prompt_len=args.prompt_len)
     if args.impl == "reference":
         run_reference(args, w)
     else:
