@@ -91,7 +91,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
         if (ipu > ntiles) ipu = ntiles;
         while (ipu > 1 && (long long)s->U * ipu > (1ll << 30)) --ipu;     // item indices stay 32-bit
         s->ipu = ipu;
-        s->splits = tc_groups(s->R, s->G) * ipu;     // every item leaves one partial per compute group
+        s->splits = ipu;     // every CTA that holds items of a unit leaves one partial
         return true;
     }
     *kind = kKindSimt;

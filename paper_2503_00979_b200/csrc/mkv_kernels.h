@@ -11,10 +11,10 @@ int simt_default_splits(int U, int cap);
 
 // Tensor-core (tcgen05) decode step: bf16, head_dim 128, GQA group in {1,2,4,8,16} and
 // R*G padded to a multiple of 32 at most 256.  The plan holds the TMA tensor maps of a
-// context's arena and the launch geometry; `a.splits` must be tc_groups() * items per unit.
+// context's arena and the launch geometry; `a.splits` must be the items per unit
+// (a CTA that holds some of a unit's items leaves one partial, so that bounds the partials).
 bool tc_shape_supported(bool f32, int D, int G, int R);
 int tc_items_per_unit(int U, int cap, int G, int n_sm);
-int tc_groups(int R, int G);     // compute groups per CTA; every CTA leaves that many partials per unit
 struct TcPlan;
 cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int items_per_unit, char *err, size_t err_len);
 void tc_plan_destroy(TcPlan *plan);

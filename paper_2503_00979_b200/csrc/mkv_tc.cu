@@ -16,9 +16,13 @@
 //                a key's R*G logits, frozen soft-max weights exp2(s*scale - c_row), GQA group
 //                sum, window fusion (Eq. 4-6, Algorithm 1); then the new row's soft-max is
 //                continued online (running max per head, rescale) and P.V for the warp's keys
-//                runs on mma.sync with P split in two bf16 terms (Eq. 1).  Warps only meet at
-//                mbarriers; a group synchronises once per unit to publish its partial.
-//   The group that takes a unit's last ticket runs the per-unit epilogue (Eq. 7).
+//                runs on mma.sync with P split in two bf16 terms (Eq. 1).  Compute warps only
+//                meet at mbarriers; when a unit's tiles in this CTA are done each warp leaves
+//                its partial (m, l, O) in shared memory and goes on with the next unit.
+//   warps 11-14  epilogue group: merges the eight warp partials of a unit; if the unit spans
+//                several CTAs it publishes the CTA's partial and an atomic ticket (no waiting)
+//                elects the last CTA; that group merges, writes the output, adds the new row's
+//                term to the fused scores, evicts and appends (Eq. 7).  Compute never stalls on it.
 // Every mbarrier wait is bounded; a wait that runs out sets a device error flag and the CTA
 // drains and exits.  Warp-collective .aligned instructions (ldmatrix, mma.sync, tcgen05.ld)
 // are only reached with the whole warp converged: the code before them is branch-free or
@@ -39,27 +43,30 @@ namespace {
 constexpr int kD = 128;
 constexpr int kTile = 128;                  // keys per tile = MMA M = TMEM lanes
 constexpr int kStageBytes = 2 * kTile * 128;   // one K or V tile: two 64-column boxes
-constexpr int kMaxComputeGroups = 3;
-__host__ __device__ constexpr int tc_threads(int ng) { return 32 * (3 + 4 * ng); }   // 3 service warps + 4 per group
+constexpr int kComputeGroups = 2;
+constexpr int kMaxComputeWarps = 4 * kComputeGroups;
+// 3 service warps + 4 per compute group + 4 epilogue warps
+__host__ __device__ constexpr int tc_threads(int ng) { return 32 * (3 + 4 * ng + 4); }
 constexpr int kFirstComputeWarp = 3;
 constexpr int kGroupThreads = 128;
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds
-constexpr int kFinFloats = 4 * kMaxGroup + 128 + 256 + 64 + 32 + 8;   // per-group epilogue scratch
+constexpr int kFinFloats = 4 * kMaxGroup + 128 + 256 + 64 + 32 + 8;   // epilogue scratch of finalize_fast
+// epilogue group: finalize scratch, flag, merged (m, l), per-warp scale factors
+constexpr int kEpiFloats = kFinFloats + 8 + 2 * kMaxGroup + kMaxComputeWarps * kMaxGroup;
 
 struct TcGeom {
     int rgpad;          // ring rows padded to a multiple of 32 (MMA N)
     int ipu;            // work items per unit
     int sk, sv;         // K stages, V stages
-    int ng;             // compute groups (2 or 3); tile T belongs to group T % ng
+    int ng;             // compute groups; tile T belongs to group T % ng
     int nb;             // TMEM accumulator buffers (a multiple of ng)
     int tmem_cols;      // allocated TMEM columns (power of two)
-    int red_bytes;      // per-group scratch for the output reduction at publish time
     int grid;
     int smem_bytes;
 };
 
 struct SmemLayout {
-    int q, kst, vst, red, negc, stw, small, bars, total;
+    int q, kst, vst, wbuf, wml, negc, stw, epi, bars, total;
 };
 
 __host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g, int G)
@@ -69,12 +76,14 @@ __host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g, int G)
     L.q = o; o += g.rgpad * 256;
     L.kst = o; o += g.sk * kStageBytes;
     L.vst = o; o += g.sv * kStageBytes;
-    L.red = o; o += g.ng * g.red_bytes;
-    L.negc = o; o += g.ng * g.rgpad * 4;              // one copy per compute group
-    L.stw = o; o += 4 * g.ng * (G * 32 + 2 * kMaxGroup) * 4; // per warp: kept logits of one tile, rescale factors, reference
-    L.small = o; o += g.ng * (8 * kMaxGroup + kFinFloats + 4) * 4;
+    const int ncw = 4 * g.ng;                         // compute warps
+    L.wbuf = o; o += ncw * G * kD * 4;                // a warp's un-normalised output O[g][d] of a finished unit
+    L.wml = o; o += ncw * 2 * kMaxGroup * 4;          // ... and its (max, denominator) per head
+    L.negc = o; o += ncw * g.rgpad * 4;               // negated ring normalisers, one copy per compute warp
+    L.stw = o; o += ncw * (G * 32 + 2 * kMaxGroup) * 4; // per warp: kept logits of one tile, rescale factors, reference
+    L.epi = o; o += kEpiFloats * 4;
     o = (o + 15) & ~15;
-    L.bars = o; o += 8 * 48;
+    L.bars = o; o += 8 * 64;
     L.total = o;
     return L;
 }
@@ -242,7 +251,7 @@ struct Item {
     int unit, sp, tile0, nk;
 };
 struct Walk {     // the same deterministic walk over this CTA's items in every role
-    int it, it_end;   // item indices (the host keeps U * ipu below 2^31)
+    int it, it_end, it_begin;   // item indices (the host keeps U * ipu below 2^31)
     int unit, sp;     // unit and split index of item `it`, kept incrementally (no divisions per item)
     int ipu, tpi, ntiles;
     int prev_unit;
@@ -255,6 +264,7 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
         // item i belongs to CTA (i * grid) / total, so CTA c owns [ceil(c*total/grid), ceil((c+1)*total/grid))
         it = (int)((total * blockIdx.x + gridDim.x - 1) / gridDim.x);
         it_end = (int)((total * (blockIdx.x + 1) + gridDim.x - 1) / gridDim.x);
+        it_begin = it;
         ipu = g.ipu;
         unit = it / ipu;
         sp = it - unit * ipu;
@@ -263,14 +273,19 @@ struct Walk {     // the same deterministic walk over this CTA's items in every 
         prev_unit = -1; qseq = 0; T0 = 0;
     }
     __device__ int active_items() const { return (ntiles + tpi - 1) / tpi; }
-    // A unit's active items may spread over several CTAs; each CTA's share is one *segment* per
-    // compute group.  Returns the number of segments of unit u and this CTA's first slot.
-    __device__ int segments(int u, int ng, int &my_first) const
+    // A unit's active items may spread over several CTAs.  Returns how many and this CTA's index among them.
+    __device__ int ctas_of_unit(int u, int &my_index) const
     {
         const long long i0 = (long long)u * ipu, i1 = i0 + active_items() - 1;
         const int c0 = (int)(i0 * gridDim.x / total), c1 = (int)(i1 * gridDim.x / total);
-        my_first = ((int)blockIdx.x - c0) * ng;
-        return ng * (c1 - c0 + 1);
+        my_index = (int)blockIdx.x - c0;
+        return c1 - c0 + 1;
+    }
+    // true if every active item of unit u belongs to this CTA
+    __device__ bool unit_is_local(int u) const
+    {
+        const int first = u * ipu;
+        return first >= it_begin && first + active_items() - 1 < it_end;
     }
     // next item with work; new_unit tells whether the ring must be (re)loaded
     __device__ bool next(Item &x, bool &new_unit)
@@ -344,9 +359,11 @@ __device__ __forceinline__ void score_chunk(const uint32_t (&v)[32], const float
 // segments' partials, write the attention output, add the new row's term to the fused scores,
 // evict the minimum, append (Eq. 1 merge, Eq. 4-7).  All loads of a phase are issued together, so
 // the whole epilogue costs a few L2 round trips.  Requires nseg <= 8 and nseg*G*2 <= 256.
-template <int G>
+// LOCAL: the single partial is this CTA's own: l_o[g] is the thread's column of the merged output,
+// l_ml [G][2] sits in shared memory.
+template <int G, bool LOCAL>
 __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, int nseg, bool evict, float *sm, int tid,
-                              int bar_id)
+                              int bar_id, const float (&l_o)[G], const float *l_ml)
 {
     constexpr int NT_ = kGroupThreads;
     const int lane = tid & 31, warp = tid >> 5;
@@ -375,12 +392,13 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     }
     uint4 vv = make_uint4(0, 0, 0, 0);
     if (tid < 16) vv = reinterpret_cast<const uint4 *>(vn)[tid];
-    for (int i = tid; i < nseg * G * 2; i += NT_) pml_s[i] = __ldcg(pml + i);
+    for (int i = tid; i < nseg * G * 2; i += NT_) pml_s[i] = LOCAL ? l_ml[i] : __ldcg(pml + i);
     float pov[G][8];
 #pragma unroll
     for (int g = 0; g < G; ++g)
 #pragma unroll
-        for (int sp = 0; sp < 8; ++sp) pov[g][sp] = sp < nseg ? __ldcg(po + (sp * G + g) * kD + tid) : 0.f;
+        for (int sp = 0; sp < 8; ++sp)
+            pov[g][sp] = sp < nseg ? (LOCAL ? l_o[g] : __ldcg(po + (sp * G + g) * kD + tid)) : 0.f;
 
     // self logit: 8-element partial dots, reduced over the 16 threads that share a head
 #pragma unroll
@@ -531,6 +549,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const uint32_t bar_qfull = smem_u32(bars + 40), bar_qempty = smem_u32(bars + 41);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 42);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 43);
+    const uint32_t bar_udone = smem_u32(bars + 44);                    // all compute warps have left their partial of a unit
+    const uint32_t bar_pfree = smem_u32(bars + 48);                    // [8] a compute warp's partial has been read
 
     const long long t = a.st->t;
     const int n = a.st->n;
@@ -543,6 +563,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         for (int b = 0; b < NB; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
         mbar_init(bar_qfull, 1);
         mbar_init(bar_qempty, 1);
+        mbar_init(bar_udone, 4 * NG);
+        for (int i = 0; i < 4 * NG; ++i) mbar_init(bar_pfree + 8 * i, 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -665,32 +687,29 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             }
             w.advance(x, nu);
         }
-    } else {
-        // ------------------------------------------------ compute groups
+    } else if (warp < kFirstComputeWarp + 4 * NG) {
+        // ------------------------------------------------ compute warps
         const int cw = warp - kFirstComputeWarp;     // 0 .. 4*NG-1
         const int grp = cw >> 2;                     // tile T belongs to group T % NG
         const int wq = warp & 3;                     // TMEM lane quarter of this warp
         const int gtid = wq * 32 + lane;             // position among the group's 128 key lanes
-        const int bar_id = 1 + grp;
-        float *red = reinterpret_cast<float *>(smem + L.red + grp * geo.red_bytes);
-        float *negc = reinterpret_cast<float *>(smem + L.negc) + grp * RGP;
+        float *wbuf = reinterpret_cast<float *>(smem + L.wbuf) + cw * G * kD;            // [g][d]
+        float *wml = reinterpret_cast<float *>(smem + L.wml) + cw * 2 * kMaxGroup;         // [g][2]
+        float *negc = reinterpret_cast<float *>(smem + L.negc) + cw * RGP;
         float *st_w = reinterpret_cast<float *>(smem + L.stw) + cw * (G * 32 + 2 * kMaxGroup);   // [g][lane]
         float *fac = st_w + G * 32, *mref = fac + kMaxGroup;         // warp-private, indexed by head
-        float *small = reinterpret_cast<float *>(smem + L.small) + grp * (8 * kMaxGroup + kFinFloats + 4);
-        float *gm = small, *lred = small + 4 * kMaxGroup;            // [4 warps][head]
-        float *fin_sm = small + 8 * kMaxGroup;
-        int *flag = reinterpret_cast<int *>(fin_sm + kFinFloats);
         const int RG = a.R * G;
         const int gid = lane >> 2, tig = lane & 3;
         constexpr int NT = G > 8 ? 2 : 1;            // 8-head column tiles of the transposed output
 
-        // Running soft-max state of this warp over its keys of the open segment: reference max
+        // Running soft-max state of this warp over its keys of the open unit: reference max
         // per head (replicated in every lane), this lane's share of the denominator and of the
         // un-normalised output O^T[d][g].
         float mrun[G];
         float acc[NT][8][4];
         float lsum[NT];
         int seg_tiles = 0;
+        int npub = 0;                                  // partials this warp has handed to the epilogue group
 
         Walk w(geo, a.U, n);
         Item x; bool nu;
@@ -701,8 +720,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             const int u = x.unit;
             if (nu) {
                 // frozen normalisers of the ring rows, negated; the new row and padding give weight 0
-                // (the group's warps all passed the previous unit's publish barriers, so nobody reads the old table)
-                for (int c = gtid; c < RGP; c += kGroupThreads) {
+                for (int c = lane; c < RGP; c += 32) {
                     float v = -INFINITY;
                     if (c < RG && c / G != rs_new) v = -a.ring_c[(size_t)u * RG + c];
                     negc[c] = v;
@@ -716,7 +734,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
                 }
                 seg_tiles = 0;
-                group_sync(bar_id, kGroupThreads);
+                __syncwarp();
             }
             float *s_new = a.s_new + (size_t)u * G * a.cap;
             // this group's tiles are T = grp, grp + NG, ...: walk them directly
@@ -818,103 +836,125 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 ++seg_tiles;
             }
 
-            // ---- close the segment when the unit's items in this CTA are done
-            if (w.last_of_unit_here(x)) {
-                if (group_any(bar_id, !ok)) { ok = false; break; }       // all four warps agree to go on
-                int my_first;
-                const int nseg = w.segments(u, NG, my_first);
-                const int slot = my_first + grp;
-                float *pml = a.part_ml + ((size_t)u * a.splits + slot) * G * 2;
-                float *po = a.part_o + ((size_t)u * a.splits + slot) * G * kD;
-                // merge the four warps: common reference = max of theirs
-                if (lane == 0) {
-#pragma unroll
-                    for (int g = 0; g < G; ++g) gm[wq * kMaxGroup + g] = mrun[g];
-                }
-                group_sync(bar_id, kGroupThreads);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
-                    auto gmax = [&](int g) {
-                        return fmaxf(fmaxf(gm[g], gm[kMaxGroup + g]), fmaxf(gm[2 * kMaxGroup + g], gm[3 * kMaxGroup + g]));
-                    };
-                    auto scale = [&](int g) {     // this warp's reference -> the group's
-                        const float mw = gm[wq * kMaxGroup + g];
-                        return mw == -INFINITY ? 0.f : ex2f(mw - gmax(g));
-                    };
-                    float l = lsum[nt];
-                    l += __shfl_xor_sync(0xffffffffu, l, 1);
-                    l += __shfl_xor_sync(0xffffffffu, l, 2);
-                    if (tig == 0 && gr < G) lred[wq * kMaxGroup + gr] = l * scale(gr);
-                    // bring this warp's accumulators to the group's reference
-                    const float f0 = gc < G ? scale(gc) : 0.f, f1 = gc + 1 < G ? scale(gc + 1) : 0.f;
-#pragma unroll
-                    for (int db = 0; db < 8; ++db) { acc[nt][db][0] *= f0; acc[nt][db][1] *= f1; acc[nt][db][2] *= f0; acc[nt][db][3] *= f1; }
-                }
-                // four warps -> one output through a two-slot buffer: warps 2, 3 store; warps 0, 1 add
-                // theirs and store the sums; everybody adds the two slots
-                auto red_io = [&](bool store) {
-                    float *slot_ = red + (wq & 1) * G * kD;
+
+            // ---- the unit's tiles in this CTA are done: leave this warp's partial for the epilogue group
+            if (w.last_of_unit_here(x) && ok) {
+                // the previous partial must have been read before its buffer is overwritten
+                if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag));
+                if (ok) {
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        const int gc = tig * 2 + 8 * nt;
+                        const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
+                        float l = lsum[nt];
+                        l += __shfl_xor_sync(0xffffffffu, l, 1);
+                        l += __shfl_xor_sync(0xffffffffu, l, 2);
+                        float m = -INFINITY;
+#pragma unroll
+                        for (int g = 0; g < G; ++g) m = g == gr ? mrun[g] : m;
+                        if (tig == 0 && gr < G) { wml[gr * 2] = m; wml[gr * 2 + 1] = l; }
 #pragma unroll
                         for (int db = 0; db < 8; ++db) {
-                            float *p0 = slot_ + gc * kD + db * 16 + gid, *p1 = slot_ + (gc + 1) * kD + db * 16 + gid;
-                            if (gc < G) {
-                                if (store) { p0[0] = acc[nt][db][0]; p0[8] = acc[nt][db][2]; }
-                                else { acc[nt][db][0] += p0[0]; acc[nt][db][2] += p0[8]; }
-                            }
-                            if (gc + 1 < G) {
-                                if (store) { p1[0] = acc[nt][db][1]; p1[8] = acc[nt][db][3]; }
-                                else { acc[nt][db][1] += p1[0]; acc[nt][db][3] += p1[8]; }
-                            }
+                            if (gc < G) { wbuf[gc * kD + db * 16 + gid] = acc[nt][db][0]; wbuf[gc * kD + db * 16 + gid + 8] = acc[nt][db][2]; }
+                            if (gc + 1 < G) { wbuf[(gc + 1) * kD + db * 16 + gid] = acc[nt][db][1]; wbuf[(gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3]; }
                         }
                     }
-                };
-                if (wq >= 2) red_io(true);
-                group_sync(bar_id, kGroupThreads);
-                if (wq < 2) red_io(false);
-                group_sync(bar_id, kGroupThreads);
-                if (wq < 2) red_io(true);
-                // the segment's state is spent (the next item starts a new unit)
+                    // the unit's state is spent (the next item starts a new unit)
 #pragma unroll
-                for (int g = 0; g < G; ++g) mrun[g] = -INFINITY;
+                    for (int g = 0; g < G; ++g) mrun[g] = -INFINITY;
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    lsum[nt] = 0.f;
+                    for (int nt = 0; nt < NT; ++nt) {
+                        lsum[nt] = 0.f;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
+                        for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
+                    }
+                    seg_tiles = 0;
+                    // fused scores / new-row logits of this warp's keys are read by the epilogue group of
+                    // this CTA, or of another CTA when the unit is shared
+                    if (w.unit_is_local(u)) __threadfence_block(); else __threadfence();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_udone);
+                    ++npub;
                 }
-                seg_tiles = 0;
-                group_sync(bar_id, kGroupThreads);
-                for (int idx = gtid; idx < G * kD; idx += kGroupThreads)
-                    po[idx] = red[idx] + red[G * kD + idx];
-                if (gtid < G) {
-                    pml[gtid * 2] = fmaxf(fmaxf(gm[gtid], gm[kMaxGroup + gtid]), fmaxf(gm[2 * kMaxGroup + gtid], gm[3 * kMaxGroup + gtid]));
-                    pml[gtid * 2 + 1] = (lred[gtid] + lred[kMaxGroup + gtid]) + (lred[2 * kMaxGroup + gtid] + lred[3 * kMaxGroup + gtid]);
+            }
+            w.advance(x, nu);
+        }
+    } else {
+        // ------------------------------------------------ epilogue group (128 threads)
+        const int etid = tid - (kFirstComputeWarp + 4 * NG) * 32;
+        constexpr int NCW = 4 * NG;
+        constexpr int kEpiBar = 1;
+        const float *wbuf = reinterpret_cast<const float *>(smem + L.wbuf);
+        const float *wml = reinterpret_cast<const float *>(smem + L.wml);
+        float *epi = reinterpret_cast<float *>(smem + L.epi);
+        float *fin_sm = epi;                                          // kFinFloats
+        int *flag = reinterpret_cast<int *>(epi + kFinFloats);
+        float *cml = epi + kFinFloats + 8;                            // merged (m, l) [g][2]
+        float *sc = cml + 2 * kMaxGroup;                              // [warp][g] scale to the merged reference
+        Walk w(geo, a.U, n);
+        Item x; bool nu;
+        bool ok = true;
+        int k = 0;                                                    // units finished so far
+        while (ok && w.next(x, nu)) {
+            if (w.last_of_unit_here(x)) {
+                const int u = x.unit;
+                if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag))) { ok = false; break; }
+                // merge the compute warps' partials: common reference = max of theirs
+                if (etid < G) {
+                    float m = -INFINITY;
+                    for (int cwi = 0; cwi < NCW; ++cwi) m = fmaxf(m, wml[cwi * 2 * kMaxGroup + etid * 2]);
+                    float l = 0.f;
+                    for (int cwi = 0; cwi < NCW; ++cwi) {
+                        const float mw = wml[cwi * 2 * kMaxGroup + etid * 2];
+                        const float f = mw == -INFINITY ? 0.f : ex2f(mw - m);
+                        sc[cwi * kMaxGroup + etid] = f;
+                        l += wml[cwi * 2 * kMaxGroup + etid * 2 + 1] * f;
+                    }
+                    cml[etid * 2] = m;
+                    cml[etid * 2 + 1] = l;
                 }
-                // publish.  Writers: every thread fences its own writes; after the group barrier the
-                // ticket thread fences again (cumulative over what the barrier made it observe) and
-                // only then increments the ticket.  Reader: the thread that saw the last ticket
-                // fences before the barrier that lets the group read the other segments.
-                __threadfence();
-                group_sync(bar_id, kGroupThreads);
-                if (gtid == 0) {
+                group_sync(kEpiBar, kGroupThreads);
+                float o[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float v = 0.f;
+#pragma unroll
+                    for (int cwi = 0; cwi < NCW; ++cwi) v += wbuf[(cwi * G + g) * kD + etid] * sc[cwi * kMaxGroup + g];
+                    o[g] = v;
+                }
+                group_sync(kEpiBar, kGroupThreads);                       // every warp buffer has been read
+                if (etid < NCW) mbar_arrive(bar_pfree + 8 * etid);
+                int my_index;
+                const int ncta = w.ctas_of_unit(u, my_index);
+                if (ncta == 1) {
+                    finalize_fast<G, true>(a, u, t, n, 1, evict, fin_sm, etid, kEpiBar, o, cml);
+                } else {
+                    // the unit is shared: publish this CTA's partial; the last CTA to do so finishes the unit.
+                    // Writers fence their own writes; after the barrier the ticket thread fences again
+                    // (cumulative over what the barrier made it observe) and then takes the ticket.
+                    float *pml = a.part_ml + ((size_t)u * a.splits + my_index) * G * 2;
+                    float *po = a.part_o + ((size_t)u * a.splits + my_index) * G * kD;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) po[g * kD + etid] = o[g];
+                    if (etid < 2 * G) pml[etid] = cml[etid];
                     __threadfence();
-                    const int last = atomicAdd(&a.ticket[u], 1) == nseg - 1;
-                    __threadfence();
-                    *flag = last;
+                    group_sync(kEpiBar, kGroupThreads);
+                    if (etid == 0) {
+                        __threadfence();
+                        const int last = atomicAdd(&a.ticket[u], 1) == ncta - 1;
+                        __threadfence();
+                        *flag = last;
+                    }
+                    group_sync(kEpiBar, kGroupThreads);
+                    if (*flag) {
+                        __threadfence();
+                        if (ncta <= 8 && ncta * G * 2 <= 256)
+                            finalize_fast<G, false>(a, u, t, n, ncta, evict, fin_sm, etid, kEpiBar, o, nullptr);
+                        else
+                            finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, ncta, evict, fin_sm, etid, kGroupThreads, kEpiBar);
+                    }
                 }
-                group_sync(bar_id, kGroupThreads);
-                if (*flag) __threadfence();
-                if (*flag) {
-                    if (nseg <= 8 && nseg * G * 2 <= 256)
-                        finalize_fast<G>(a, u, t, n, nseg, evict, fin_sm, gtid, bar_id);
-                    else
-                        finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, nseg, evict, fin_sm, gtid, kGroupThreads, bar_id);
-                }
-                group_sync(bar_id, kGroupThreads);
+                group_sync(kEpiBar, kGroupThreads);
+                ++k;
             }
             w.advance(x, nu);
         }
@@ -967,7 +1007,7 @@ bool encode_map(CUtensorMap *m, void *base, int units, int rows, int box_rows)
 struct TcPlan {
     CUtensorMap tmK, tmV, tmQ;
     TcGeom geo;
-    bool attr_set[5][2][2];
+    bool attr_set[5][2];
 };
 
 namespace {
@@ -978,7 +1018,7 @@ template <int G, int FUSION, int NG>
 cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
     auto kern = decode_tc_kernel<G, FUSION, NG>;
-    bool &set = plan->attr_set[group_index(G)][FUSION][NG - 2];
+    bool &set = plan->attr_set[group_index(G)][FUSION];
     if (!set) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan->geo.smem_bytes);
         if (e != cudaSuccess) return e;
@@ -991,7 +1031,7 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 template <int G, int FUSION>
 cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    return plan->geo.ng == 3 ? launch_gfn<G, FUSION, 3>(plan, a, stream) : launch_gfn<G, FUSION, 2>(plan, a, stream);
+    return launch_gfn<G, FUSION, kComputeGroups>(plan, a, stream);
 }
 
 template <int G>
@@ -1003,9 +1043,6 @@ cudaError_t launch_g(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 int pad32(int x) { return (x + 31) & ~31; }
 
 }  // namespace
-
-// three compute groups when three accumulator buffers fit the 512 TMEM columns, else two
-int tc_groups(int R, int G) { return pad32(R * G) <= 128 ? 3 : 2; }
 
 bool tc_shape_supported(bool f32, int D, int G, int R)
 {
@@ -1050,20 +1087,19 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err
     const int G = a.G;
     g.rgpad = pad32(a.R * G);
     g.ipu = ipu;
-    g.ng = tc_groups(a.R, G);
-    g.nb = g.ng == 3 ? (g.rgpad <= 64 ? 6 : 3) : (g.rgpad <= 128 ? 4 : 2);
+    g.ng = kComputeGroups;
+    g.nb = g.rgpad <= 128 ? 4 : 2;
     g.tmem_cols = 32;
     while (g.tmem_cols < g.nb * g.rgpad) g.tmem_cols *= 2;
-    g.red_bytes = (2 * G * kD * 4 + 127) & ~127;
     const long long items = (long long)a.U * ipu;
     g.grid = (int)(items < n_sm ? items : n_sm);
     // as many 32 KB stages as fit, split between the K ring (short-lived tiles) and the V ring
     int total_stages = 0;
-    for (int st = 9; st >= 3; --st) {
+    for (int st = 9; st >= 2; --st) {
         g.sk = 1; g.sv = st - 1;
         if (tc_smem_layout(g, G).total + 1024 <= max_smem) { total_stages = st; break; }
     }
-    if (total_stages < 3) {
+    if (total_stages < 2) {
         snprintf(err, err_len, "tensor-core kernel: shared memory does not fit");
         delete p;
         return cudaErrorInvalidConfiguration;
