@@ -21,7 +21,7 @@ struct Layout {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Shape {
-    int U, G, D, R, C, cap, splits, T, ipu;
+    int U, G, D, R, C, cap, splits, T, tc_grid_size;
     size_t es;
 };
 
@@ -82,16 +82,14 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     s->cap = p->C + p->R + s->T - 1;
     s->es = p->dtype == MKV_DTYPE_F32 ? 4 : 2;
     if (s->T != 1) return false;
-    const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R);
+    const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R) &&
+                       (long long)s->U * ((s->cap + 127) / 128) <= (1ll << 30);     // tile indices stay 32-bit
     if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
     if (tc_ok && p->kernel != MKV_KERNEL_SIMT) {
         *kind = kKindTc;
-        const int ntiles = (s->cap + 127) / 128;
-        int ipu = p->splits > 0 ? p->splits : tc_items_per_unit(s->U, s->cap, s->G, 148);
-        if (ipu > ntiles) ipu = ntiles;
-        while (ipu > 1 && (long long)s->U * ipu > (1ll << 30)) --ipu;     // item indices stay 32-bit
-        s->ipu = ipu;
-        s->splits = ipu;     // every CTA that holds items of a unit leaves one partial
+        // the persistent grid (148 SMs on B200; correctness does not depend on the count)
+        s->tc_grid_size = tc_grid(s->U, s->cap, p->splits, 148);
+        s->splits = tc_partials_per_unit(s->U, s->cap, s->tc_grid_size);
         return true;
     }
     *kind = kKindSimt;
@@ -99,7 +97,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     int sp = p->splits > 0 ? p->splits : simt_default_splits(s->U, s->cap);
     if (sp > max_splits) sp = max_splits;
     s->splits = sp;
-    s->ipu = 0;
+    s->tc_grid_size = 0;
     return true;
 }
 
@@ -229,7 +227,7 @@ mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p)
     if (kind == kKindTc) {
         const DecodeArgs a = make_args(c, nullptr, nullptr, nullptr, nullptr);
         char msg[200] = "";
-        const cudaError_t e = tc_plan_create(&c->plan, a, s.ipu, msg, sizeof(msg));
+        const cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, msg, sizeof(msg));
         if (e != cudaSuccess) {
             cudaGetLastError();
             if (c->owns_workspace) cudaFree(c->base);

@@ -11,12 +11,13 @@ int simt_default_splits(int U, int cap);
 
 // Tensor-core (tcgen05) decode step: bf16, head_dim 128, GQA group in {1,2,4,8,16} and
 // R*G padded to a multiple of 32 at most 256.  The plan holds the TMA tensor maps of a
-// context's arena and the launch geometry; `a.splits` must be the items per unit
-// (a CTA that holds some of a unit's items leaves one partial, so that bounds the partials).
+// context's arena and the launch geometry; `a.splits` must be tc_partials_per_unit()
+// of the grid (every CTA that holds tiles of a unit leaves one partial).
 bool tc_shape_supported(bool f32, int D, int G, int R);
-int tc_items_per_unit(int U, int cap, int G, int n_sm);
+int tc_grid(int U, int cap, int splits_hint, int n_sm);
+int tc_partials_per_unit(int U, int cap, int grid);
 struct TcPlan;
-cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int items_per_unit, char *err, size_t err_len);
+cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int grid, char *err, size_t err_len);
 void tc_plan_destroy(TcPlan *plan);
 cudaError_t launch_decode_tc(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream);
 

@@ -1,9 +1,10 @@
 // Tensor-core decode kernel for sm_100a: bf16, head_dim 128, GQA group in {1,2,4,8,16},
 // R*G (padded to a multiple of 32) at most 256.
 //
-// A persistent, warp-specialised CTA per SM walks a static list of work items; an item is a
-// run of 128-key tiles of one unit's cache.  Per tile the K rows feed the scoring contraction
-// and the V rows the attention output; both are read from HBM exactly once.
+// The 128-key tiles of all units' caches form one sequence that is cut into equal contiguous
+// ranges, one per persistent, warp-specialised CTA; a work item is the run of a unit's tiles
+// inside a CTA's range.  Per tile the K rows feed the scoring contraction and the V rows the
+// attention output; both are read from HBM exactly once.
 //   warp 0       TMA producer of the unit's recent-query ring (once per unit) and of K tiles
 //                (cp.async.bulk.tensor, 128-byte swizzle) into a short ring of 32 KB stages.
 //   warp 1       writes the new query over the ring row that leaves the window, then issues
@@ -56,7 +57,6 @@ constexpr int kEpiFloats = kFinFloats + 8 + 2 * kMaxGroup + kMaxComputeWarps * k
 
 struct TcGeom {
     int rgpad;          // ring rows padded to a multiple of 32 (MMA N)
-    int ipu;            // work items per unit
     int sk, sv;         // K stages, V stages
     int ng;             // compute groups; tile T belongs to group T % ng
     int nb;             // TMEM accumulator buffers (a multiple of ng)
@@ -146,7 +146,6 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
 {
     asm volatile(
@@ -248,74 +247,67 @@ __device__ __forceinline__ bool group_any(int bar_id, bool pred)
 
 // ---------------------------------------------------------------- schedule shared by all roles
 struct Item {
-    int unit, sp, tile0, nk;
+    int unit, tile0, nk;      // tiles [tile0, tile0 + nk) of the unit
 };
-struct Walk {     // the same deterministic walk over this CTA's items in every role
-    int it, it_end, it_begin;   // item indices (the host keeps U * ipu below 2^31)
-    int unit, sp;     // unit and split index of item `it`, kept incrementally (no divisions per item)
-    int ipu, tpi, ntiles;
-    int prev_unit;
-    int qseq;         // units seen so far (ring loads)
-    int T0;           // running tile sequence number
+// The same deterministic walk over this CTA's items in every role.  With nt tiles per unit at
+// the current cache length, global tile i is tile i % nt of unit i / nt, and CTA c of the
+// E = min(grid, U * nt) working CTAs owns tiles [c * T / E, (c + 1) * T / E), T = U * nt: every
+// working CTA owns at least one tile and consecutive items belong to different units.
+struct Walk {
+    int tile, tile_begin, tile_end;   // the host keeps U * tiles per unit below 2^31
+    int nt;           // tiles per unit
+    int unit, off;    // unit and tile inside it of `tile`
+    int nitems;       // items returned so far (= units seen: ring loads, partials)
+    int T0;           // tiles of the items already advanced over
+    int eff;          // working CTAs
     long long total;
-    __device__ Walk(const TcGeom &g, int U, int n)
+    __device__ Walk(int U, int n)
     {
-        total = (long long)U * g.ipu;
-        // item i belongs to CTA (i * grid) / total, so CTA c owns [ceil(c*total/grid), ceil((c+1)*total/grid))
-        it = (int)((total * blockIdx.x + gridDim.x - 1) / gridDim.x);
-        it_end = (int)((total * (blockIdx.x + 1) + gridDim.x - 1) / gridDim.x);
-        it_begin = it;
-        ipu = g.ipu;
-        unit = it / ipu;
-        sp = it - unit * ipu;
-        ntiles = (n + kTile - 1) / kTile;
-        tpi = (ntiles + ipu - 1) / ipu;
-        prev_unit = -1; qseq = 0; T0 = 0;
+        nt = (n + kTile - 1) / kTile;
+        total = (long long)U * nt;
+        eff = (int)(total < (long long)gridDim.x ? total : (long long)gridDim.x);
+        if ((int)blockIdx.x < eff) {
+            tile = (int)(total * blockIdx.x / eff);
+            tile_end = (int)(total * (blockIdx.x + 1) / eff);
+        } else {
+            tile = tile_end = 0;
+        }
+        tile_begin = tile;
+        unit = tile / nt;
+        off = tile - unit * nt;
+        nitems = 0; T0 = 0;
     }
-    __device__ int active_items() const { return (ntiles + tpi - 1) / tpi; }
-    // A unit's active items may spread over several CTAs.  Returns how many and this CTA's index among them.
+    __device__ bool next(Item &x)
+    {
+        if (tile >= tile_end) return false;
+        x.unit = unit;
+        x.tile0 = off;
+        x.nk = min(nt - off, tile_end - tile);
+        tile += x.nk;
+        off += x.nk;
+        if (off == nt) { off = 0; ++unit; }
+        return true;
+    }
+    __device__ void advance(const Item &x)
+    {
+        T0 += x.nk;
+        ++nitems;
+    }
+    // the CTA that owns global tile i: the largest c with c * T / E <= i
+    __device__ int owner(long long i) const { return (int)(((i + 1) * eff - 1) / total); }
+    // How many CTAs hold tiles of unit u, and this CTA's index among them.
     __device__ int ctas_of_unit(int u, int &my_index) const
     {
-        const long long i0 = (long long)u * ipu, i1 = i0 + active_items() - 1;
-        const int c0 = (int)(i0 * gridDim.x / total), c1 = (int)(i1 * gridDim.x / total);
+        const long long i0 = (long long)u * nt;
+        const int c0 = owner(i0), c1 = owner(i0 + nt - 1);
         my_index = (int)blockIdx.x - c0;
         return c1 - c0 + 1;
     }
-    // true if every active item of unit u belongs to this CTA
+    // true if all tiles of unit u belong to this CTA
     __device__ bool unit_is_local(int u) const
     {
-        const int first = u * ipu;
-        return first >= it_begin && first + active_items() - 1 < it_end;
-    }
-    // next item with work; new_unit tells whether the ring must be (re)loaded
-    __device__ bool next(Item &x, bool &new_unit)
-    {
-        while (it < it_end) {
-            x.unit = unit;
-            x.sp = sp;
-            x.tile0 = sp * tpi;
-            x.nk = min(tpi, ntiles - x.tile0);
-            ++it;
-            if (++sp == ipu) { sp = 0; ++unit; }
-            if (x.nk > 0) {
-                new_unit = x.unit != prev_unit;
-                prev_unit = x.unit;
-                return true;
-            }
-        }
-        return false;
-    }
-    // true if the next item with work (if any) belongs to another unit; (unit, sp) already
-    // describe the item after x
-    __device__ bool last_of_unit_here(const Item &x) const
-    {
-        if (it >= it_end || unit != x.unit) return true;
-        return sp * tpi >= ntiles;                       // the unit's remaining items are empty
-    }
-    __device__ void advance(const Item &x, bool new_unit)
-    {
-        T0 += x.nk;
-        if (new_unit) ++qseq;
+        const int first = u * nt;
+        return first >= tile_begin && first + nt <= tile_end;
     }
 };
 
@@ -577,19 +569,17 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     if (warp == 0) {
         // ------------------------------------------------ TMA producer: query ring and K tiles (one lane)
         if (lane == 0) {
-            Walk w(geo, a.U, n);
-            Item x; bool nu;
+            Walk w(a.U, n);
+            Item x;
             int issued = 0;
             bool ok = true;
             RingPos rk(0, SK);
-            while (ok && w.next(x, nu)) {
-                if (nu) {
-                    ok = mbar_wait(bar_qempty, (uint32_t)((w.qseq & 1) ^ 1), abort_flag);
-                    if (!ok) break;
-                    mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
-                    tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
-                    tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
-                }
+            while (ok && w.next(x)) {
+                ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
+                tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
+                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
                 for (int j = 0; j < x.nk && ok; ++j, rk.step(1, SK)) {
                     const int T = w.T0 + j, s = rk.idx;
                     ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(rk.lap ^ 1), abort_flag);
@@ -600,7 +590,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, x.unit, bar_kfull + 8 * s);
                     issued = T + 1;
                 }
-                w.advance(x, nu);
+                w.advance(x);
             }
             if (!ok) {   // give up: let the copies already in flight land before the CTA exits
                 int dummy = 0;
@@ -611,12 +601,12 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     } else if (warp == 2) {
         // ------------------------------------------------ TMA producer: V tiles (one lane)
         if (lane == 0) {
-            Walk w(geo, a.U, n);
-            Item x; bool nu;
+            Walk w(a.U, n);
+            Item x;
             int issued = 0;
             bool ok = true;
             RingPos rv(0, SV);
-            while (ok && w.next(x, nu)) {
+            while (ok && w.next(x)) {
                 for (int j = 0; j < x.nk && ok; ++j, rv.step(1, SV)) {
                     const int T = w.T0 + j, s = rv.idx;
                     ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag);
@@ -627,7 +617,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, x.unit, bar_vfull + 8 * s);
                     issued = T + 1;
                 }
-                w.advance(x, nu);
+                w.advance(x);
             }
             if (!ok) {
                 int dummy = 0;
@@ -637,21 +627,21 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ------------------------------------------------ new-query substitution + MMA issue
-        Walk w(geo, a.U, n);
-        Item x; bool nu;
+        Walk w(a.U, n);
+        Item x;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RGP >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
         bool ok = true;
         RingPos rk(0, SK), rb(0, NB);
-        while (ok && w.next(x, nu)) {
-            if (nu) {
-                if (w.qseq > 0 && lane == 0) umma_commit(bar_qempty);   // MMAs of the previous unit done with the ring
+        while (ok && w.next(x)) {
+            {
+                if (w.nitems > 0 && lane == 0) umma_commit(bar_qempty);   // MMAs of the previous unit done with the ring
                 // the new query replaces ring row t % R (the row of the token leaving the window)
                 uint4 qv[kMaxGroup / 2];
                 const uint4 *qsrc = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(a.q) + (size_t)x.unit * G * kD);
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i)
                     if (lane + 32 * i < G * 16) qv[i] = qsrc[lane + 32 * i];
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.qseq & 1), abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.nitems & 1), abort_flag));
                 if (!ok) break;
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i) {
@@ -685,7 +675,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 }
                 __syncwarp();
             }
-            w.advance(x, nu);
+            w.advance(x);
         }
     } else if (warp < kFirstComputeWarp + 4 * NG) {
         // ------------------------------------------------ compute warps
@@ -711,14 +701,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         int seg_tiles = 0;
         int npub = 0;                                  // partials this warp has handed to the epilogue group
 
-        Walk w(geo, a.U, n);
-        Item x; bool nu;
+        Walk w(a.U, n);
+        Item x;
         bool ok = true;
         int Tn = grp;                                  // next tile of this group
         RingPos rb(grp, NB), rv(grp, SV);
-        while (w.next(x, nu)) {
+        while (w.next(x)) {
             const int u = x.unit;
-            if (nu) {
+            {
                 // frozen normalisers of the ring rows, negated; the new row and padding give weight 0
                 for (int c = lane; c < RGP; c += 32) {
                     float v = -INFINITY;
@@ -837,8 +827,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             }
 
 
-            // ---- the unit's tiles in this CTA are done: leave this warp's partial for the epilogue group
-            if (w.last_of_unit_here(x) && ok) {
+            // ---- the item is done: leave this warp's partial for the epilogue group
+            if (ok) {
                 // the previous partial must have been read before its buffer is overwritten
                 if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag));
                 if (ok) {
@@ -858,16 +848,6 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                             if (gc + 1 < G) { wbuf[(gc + 1) * kD + db * 16 + gid] = acc[nt][db][1]; wbuf[(gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3]; }
                         }
                     }
-                    // the unit's state is spent (the next item starts a new unit)
-#pragma unroll
-                    for (int g = 0; g < G; ++g) mrun[g] = -INFINITY;
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        lsum[nt] = 0.f;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) { acc[nt][i][0] = 0.f; acc[nt][i][1] = 0.f; acc[nt][i][2] = 0.f; acc[nt][i][3] = 0.f; }
-                    }
-                    seg_tiles = 0;
                     // fused scores / new-row logits of this warp's keys are read by the epilogue group of
                     // this CTA, or of another CTA when the unit is shared
                     if (w.unit_is_local(u)) __threadfence_block(); else __threadfence();
@@ -876,7 +856,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     ++npub;
                 }
             }
-            w.advance(x, nu);
+            w.advance(x);
         }
     } else {
         // ------------------------------------------------ epilogue group (128 threads)
@@ -890,12 +870,12 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         int *flag = reinterpret_cast<int *>(epi + kFinFloats);
         float *cml = epi + kFinFloats + 8;                            // merged (m, l) [g][2]
         float *sc = cml + 2 * kMaxGroup;                              // [warp][g] scale to the merged reference
-        Walk w(geo, a.U, n);
-        Item x; bool nu;
+        Walk w(a.U, n);
+        Item x;
         bool ok = true;
         int k = 0;                                                    // units finished so far
-        while (ok && w.next(x, nu)) {
-            if (w.last_of_unit_here(x)) {
+        while (ok && w.next(x)) {
+            {
                 const int u = x.unit;
                 if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag))) { ok = false; break; }
                 // merge the compute warps' partials: common reference = max of theirs
@@ -956,7 +936,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 group_sync(kEpiBar, kGroupThreads);
                 ++k;
             }
-            w.advance(x, nu);
+            w.advance(x);
         }
     }
 
@@ -1050,29 +1030,39 @@ bool tc_shape_supported(bool f32, int D, int G, int R)
     return pad32(R * G) <= 256;
 }
 
-// Items per unit: the count that fills whole waves of the persistent grid best (ties: fewer,
-// larger items).  Items are scheduling quanta only; consecutive items of a unit in one CTA
-// are accumulated into one partial.
-int tc_items_per_unit(int U, int cap, int G, int n_sm)
+// Grid of the persistent kernel.  `splits_hint` > 0 asks for about that many CTAs per unit
+// (ranges of cap_tiles / splits_hint tiles); otherwise one CTA per SM.
+int tc_grid(int U, int cap, int splits_hint, int n_sm)
 {
-    (void)G;
-    const int ntiles = (cap + kTile - 1) / kTile;
-    int best = 1;
-    double best_eff = -1.0;
-    for (int ipu = 1; ipu <= ntiles; ++ipu) {
-        const int tpi = (ntiles + ipu - 1) / ipu;
-        if (tpi < 2 && ipu > 1) break;
-        const long long items = (long long)U * ((ntiles + tpi - 1) / tpi);
-        const long long waves = (items + n_sm - 1) / n_sm;
-        // time ~ waves * tiles per item (+ a fixed cost per item)
-        const double cost = (double)waves * (tpi + 0.25);
-        const double eff = (double)U * ntiles / (cost * n_sm);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = ipu; }
+    const long long ntiles = (cap + kTile - 1) / kTile, total = (long long)U * ntiles;
+    long long grid = n_sm;
+    if (splits_hint > 0) {
+        const long long chunk = (ntiles + splits_hint - 1) / splits_hint;
+        grid = (total + chunk - 1) / chunk;
+        if (grid > n_sm) grid = n_sm;
     }
-    return best;
+    if (grid > total) grid = total;
+    return (int)(grid < 1 ? 1 : grid);
 }
 
-cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err, size_t err_len)
+// Upper bound, over every cache length up to cap, of the CTAs that hold tiles of one unit
+// (= partial slots a unit needs).
+int tc_partials_per_unit(int U, int cap, int grid)
+{
+    const int ntiles = (cap + kTile - 1) / kTile;
+    int worst = 1;
+    for (int nt = 1; nt <= ntiles; ++nt) {
+        const long long total = (long long)U * nt;
+        const long long eff = total < grid ? total : grid;
+        const long long len = total / eff;                     // shortest range of a CTA
+        long long c = (nt + len - 1) / len + 1;
+        if (c > nt) c = nt;
+        if (c > worst) worst = (int)c;
+    }
+    return worst;
+}
+
+cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, char *err, size_t err_len)
 {
     *out = nullptr;
     TcPlan *p = new (std::nothrow) TcPlan;
@@ -1086,13 +1076,11 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int ipu, char *err
     TcGeom &g = p->geo;
     const int G = a.G;
     g.rgpad = pad32(a.R * G);
-    g.ipu = ipu;
     g.ng = kComputeGroups;
     g.nb = g.rgpad <= 128 ? 4 : 2;
     g.tmem_cols = 32;
     while (g.tmem_cols < g.nb * g.rgpad) g.tmem_cols *= 2;
-    const long long items = (long long)a.U * ipu;
-    g.grid = (int)(items < n_sm ? items : n_sm);
+    g.grid = grid;
     // as many 32 KB stages as fit, split between the K ring (short-lived tiles) and the V ring
     int total_stages = 0;
     for (int st = 9; st >= 2; --st) {
