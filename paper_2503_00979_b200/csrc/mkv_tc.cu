@@ -544,11 +544,6 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const uint32_t bar_udone = smem_u32(bars + 44);                    // all compute warps have left their partial of a unit
     const uint32_t bar_pfree = smem_u32(bars + 48);                    // [8] a compute warp's partial has been read
 
-    const long long t = a.st->t;
-    const int n = a.st->n;
-    const bool evict = step_evicts(t, n, a.R, a.C);
-    const int rs_new = (int)(t % a.R);
-
     if (tid == 0) {
         for (int s = 0; s < SK; ++s) { mbar_init(bar_kfull + 8 * s, 1); mbar_init(bar_kempty + 8 * s, 1); }
         for (int s = 0; s < SV; ++s) { mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_vempty + 8 * s, 4); }
@@ -565,6 +560,17 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+
+    // Programmatic dependent launch: the CTA may have started, and set itself up, while the
+    // previous kernel of the stream was still finishing.  Nothing before this line reads global
+    // memory; from here on the previous kernel has completed and its writes are visible.  The
+    // next kernel of the stream may then be staged the same way.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const long long t = a.st->t;
+    const int n = a.st->n;
+    const bool evict = step_evicts(t, n, a.R, a.C);
+    const int rs_new = (int)(t % a.R);
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer: query ring and K tiles (one lane)
@@ -1004,8 +1010,19 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         set = true;
     }
-    kern<<<plan->geo.grid, tc_threads(NG), plan->geo.smem_bytes, stream>>>(a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
-    return cudaGetLastError();
+    // launched with programmatic stream serialization: the grid may be staged while the previous
+    // kernel of the stream drains (the kernel waits for it with griddepcontrol.wait)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)plan->geo.grid);
+    cfg.blockDim = dim3((unsigned)tc_threads(NG));
+    cfg.dynamicSmemBytes = (size_t)plan->geo.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
 }
 
 template <int G, int FUSION>
