@@ -158,6 +158,25 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of per-rank timings: the job is as slow as its slowest replica."""
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_tokens_per_s(world, batch_per_replica, steps, ms):
+    """Aggregate decode throughput of `world` independent replicas that all ran `steps` steps in `ms`."""
+    return world * batch_per_replica * steps / (ms * 1e-3)
+
+
+def replica_workload(w: synth.Workload, rank: int) -> synth.Workload:
+    """Every rank decodes its own replica of the workload: same shape, different content."""
+    return w.replace(seed=w.seed + 1000 * rank)
+
+
 def run_ours(args, w):
     import torch.distributed as dist
     from paper_2503_00979_b200 import binding
@@ -171,7 +190,7 @@ def run_ours(args, w):
         raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
     dev = torch.device(f"cuda:{local}")
     torch.cuda.set_device(dev)
-    w = w.replace(seed=w.seed + 1000 * rank)       # every rank its own replica (different batch content)
+    w = replica_workload(w, rank)
     tdt = synth.torch_dtype(w.dtype)
     K, W = args.steps, args.warmup
     P, Rw = w.prompt_len, min(w.R, w.prompt_len)
@@ -246,10 +265,7 @@ def run_ours(args, w):
     checksum = float(ho[W:].float().abs().mean())
     assert np.isfinite(checksum)
 
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev, world)
     if rank == 0:
         bytes_step = algorithmic_bytes_per_step(w, n_steady)
         peak, peak_src = measured_peak_gbs()
@@ -258,7 +274,7 @@ def run_ours(args, w):
         h2d = (w.units * w.group + 2 * w.units) * w.head_dim * e
         d2h = w.units * w.group * w.head_dim * e
         line = {
-            "metric": METRIC, "value": world * w.batch * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "metric": METRIC, "value": whole_job_tokens_per_s(world, w.batch, K, ms), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
@@ -268,7 +284,7 @@ def run_ours(args, w):
                        "l2": "inputs larger than L2: each step streams the whole K/V cache "
                              f"({bytes_step / 1e6:.0f} MB per step against 126 MB of L2)"},
             "clocks": clocks.summary(),
-            "e2e": {"value": world * w.batch * K / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": whole_job_tokens_per_s(world, w.batch, K, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -278,7 +294,7 @@ def run_ours(args, w):
         if world == 1 and not args.no_cpu_baseline:
             cores = len(os.sched_getaffinity(0))
             n_units = max(1, min(cores, w.units))
-            ups, used, sample, _ = oracle_throughput(w.replace(seed=synth.WORKLOADS[args.workload].seed), n_units, args.cpu_steps)
+            ups, used, sample, _ = oracle_throughput(w.replace(seed=w.seed - 1000 * rank), n_units, args.cpu_steps)
             line["cpu_baseline"] = {"value": ups * w.batch / w.units, "unit": UNIT, "cores": used, "kind": "oracle",
                                     "sample": sample, "unit_steps_per_s": ups}
         print(json.dumps(line), flush=True)

@@ -66,16 +66,29 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     tol = TOL_OUT[w.dtype]
     Rw = min(R, P)
 
-    # ---- prefill, layer by layer draws to bound memory ----
-    k32, v32 = st.kv(np.arange(P))
-    qw32 = st.q(np.arange(P - Rw, P))
-    mk.prefill(k32.to(tdt).contiguous(), v32.to(tdt).contiguous(), qw32.to(tdt).contiguous())
+    # ---- prefill: inputs are drawn layer by layer so that full-size workloads fit in memory ----
+    Hkv, Hq = w.n_kv_heads, w.n_q_heads
+    k_all = torch.empty((w.layers, w.batch, Hkv, P, d), dtype=tdt, device=dev)
+    v_all = torch.empty_like(k_all)
+    qw_all = torch.empty((w.layers, w.batch, Hq, Rw, d), dtype=tdt, device=dev)
+    prompt = {}
+    for l in range(w.layers):
+        k32, v32 = st.kv(np.arange(P), [l])
+        qw32 = st.q(np.arange(P - Rw, P), [l])
+        k_all[l], v_all[l], qw_all[l] = k32[0].to(tdt), v32[0].to(tdt), qw32[0].to(tdt)
+        for (ul, b, h) in units:
+            if ul == l:
+                prompt[(ul, b, h)] = (k32[0, b, h].double().cpu().numpy(), v32[0, b, h].double().cpu().numpy(),
+                                      qw32[0, b, h * G:(h + 1) * G].double().cpu().numpy(), k32[0, b, h].clone())
+        del k32, v32, qw32
+    mk.prefill(k_all, v_all, qw_all)
     mk.sync()
+    del k_all, v_all, qw_all
     orac = {}
     for (l, b, h) in units:
+        kp, vp, qp, k_dev = prompt[(l, b, h)]
         u = ora.Unit(G, d, C_, R, w.fusion)
-        u.prefill(k32[l, b, h].double().cpu().numpy(), v32[l, b, h].double().cpu().numpy(),
-                  qw32[l, b, h * G:(h + 1) * G].double().cpu().numpy())
+        u.prefill(kp, vp, qp)
         view = mk.view(l)
         gp = view["pos"][b, h, :view["count"]].cpu().numpy()
         assert view["count"] == u.count, (view["count"], u.count)
@@ -86,9 +99,9 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
             continue
         # K/V rows must be the prompt rows of those positions, bit for bit
         kk = view["K"][b, h, :view["count"]].float().cpu()
-        assert torch.equal(kk, k32[l, b, h][torch.from_numpy(gp).long().to(dev)].cpu())
+        assert torch.equal(kk, k_dev[torch.from_numpy(gp).long().to(dev)].cpu())
         orac[(l, b, h)] = u
-    del k32, v32, qw32
+    del prompt
 
     # ---- decode in chunks ----
     done = 0

@@ -233,6 +233,39 @@ def test_tc_stress_shape_window_64():
     assert rep.evictions > 0
 
 
+# ---- the benchmark's own sizes: every unit runs on the device, a seeded sample (first and last
+# layer / batch row included) is followed by the oracle step by step
+def test_full_size_config1_sampled_units():
+    w = synth.WORKLOADS["c1"]
+    rep = run_parity(w, steps=64, n_units=8, kernel="auto", check_F_every=32)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions >= 7 * 64
+
+
+def test_full_size_config2_sampled_units():
+    w = synth.WORKLOADS["c2"]
+    rep = run_parity(w, steps=48, n_units=8, kernel="auto", check_F_every=24)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions >= 7 * 48
+
+
+def test_full_size_config3_sampled_units_full_cache():
+    # config 3 fills its cache over thousands of steps; start it full so the sample sees evictions
+    w = synth.WORKLOADS["c3"].replace(prompt_len=4100)
+    rep = run_parity(w, steps=24, n_units=6, kernel="auto", check_F_every=12)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions >= 5 * 24
+
+
+@pytest.mark.parametrize("name", ["c4_C512_max", "c4_C8192_sum"])
+def test_full_size_config4_sampled_units(name):
+    w = synth.WORKLOADS[name]
+    steps = 48 if w.C <= 512 else 16
+    rep = run_parity(w, steps=steps, n_units=6, kernel="auto", check_F_every=8)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions >= 5 * steps
+
+
 def test_tc_matches_cuda_core_kernel_on_device():
     # the two kernels share only the per-unit epilogue; their outputs must agree closely
     w = SMALL.replace(layers=1, batch=2, C=700, R=32, prompt_len=900, steps=12, fusion="max")
