@@ -16,6 +16,7 @@ Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -38,6 +39,27 @@ def algorithmic_bytes_per_step(w: synth.Workload, n: int) -> int:
     """K and V of the n cached tokens read once plus the R*G recent queries, per unit."""
     e = 2 if w.dtype == "bf16" else 4
     return w.units * (2 * n * w.head_dim * e + w.R * w.group * w.head_dim * e)
+
+
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
+# capture of a launch of that workload), valid only for the kernel sources it was taken with.
+_TRAFFIC = {"c1": {"bytes": 300.6e6, "sources_sha256": "1950591ea5c9437ec53d86ec66228dec839cc76240d263250e5165069fcb7f83"}}
+
+
+def measured_traffic(workload: str):
+    """The captured DRAM traffic per launch, or None when the kernel has changed since the capture."""
+    ent = _TRAFFIC.get(workload)
+    if not ent:
+        return None
+    h = hashlib.sha256()
+    csrc = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2503_00979_b200", "csrc")
+    try:
+        for f in ("mkv_tc.cu", "mkv_common.cuh"):
+            with open(os.path.join(csrc, f), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return ent["bytes"] if h.hexdigest() == ent["sources_sha256"] else None
 
 
 def measured_peak_gbs():
@@ -288,7 +310,8 @@ def run_ours(args, w):
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_src, "kernel": f"decode_{mk.kernel_name}",
+                         "traffic": measured_traffic(w.name) if mk.kernel_name == "tc" and args.prompt_len == 0 else None,
+                         "peak_source": peak_src, "kernel": f"decode_{mk.kernel_name}",
                          "algorithmic_bytes_per_launch": bytes_step},
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -107,7 +107,8 @@ mkv_status mkv_create(mkv_ctx **out, int layers, int batch, int n_q_heads, int n
  * device memory for its state. */
 mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p);
 
-/* Releases the context (and its workspace if the library allocated it).  NULL is allowed. */
+/* Releases the context, the prompt-phase scratch it holds, and its workspace if the library
+ * allocated it.  NULL is allowed. */
 void mkv_destroy(mkv_ctx *ctx);
 
 /* Prompt phase (the paper gives no procedure; this applies Algorithm 1 once with the whole
@@ -115,7 +116,8 @@ void mkv_destroy(mkv_ctx *ctx);
  * [layers][batch][n_q_heads][min(R, prompt_len)][head_dim] = the queries of the last prompt
  * positions, oldest first.  If prompt_len <= C + R everything is kept; otherwise the window
  * rows are scored causally over all prompt keys and the top C older tokens are kept.
- * Allocates temporary device scratch; synchronises the stream before returning. */
+ * Allocates device scratch on its first call (up to 1 GiB, for the logits of the window rows);
+ * the context keeps it until mkv_destroy.  Synchronises the stream before returning. */
 mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
                        int prompt_len, void *stream);
 

@@ -115,6 +115,7 @@ struct mkv_ctx {
     long long t;      // host mirror of the device step state
     int n;
     unsigned long long launches;
+    PrefillScratch prefill_scratch;
     char err[256];
 };
 
@@ -253,6 +254,7 @@ void mkv_destroy(mkv_ctx *ctx)
 {
     if (!ctx) return;
     if (ctx->plan) tc_plan_destroy(ctx->plan);
+    if (ctx->prefill_scratch.ptr) cudaFree(ctx->prefill_scratch.ptr);
     if (ctx->owns_workspace && ctx->base) cudaFree(ctx->base);
     delete ctx;
 }
@@ -266,7 +268,7 @@ mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q
     const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
     if (!clear_arena(ctx, (cudaStream_t)stream)) return fail(ctx, MKV_CUDA, "mkv_prefill: clearing the arena failed%s");
     const cudaError_t e = run_prefill(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, k, v, q_window, prompt_len,
-                                      (cudaStream_t)stream, &ctx->launches);
+                                      (cudaStream_t)stream, &ctx->launches, &ctx->prefill_scratch);
     if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(ctx, MKV_OOM, "mkv_prefill: no memory for scratch%s"); }
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_prefill: %s", cudaGetErrorString(e));
     const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
@@ -373,7 +375,11 @@ mkv_status mkv_sync(mkv_ctx *ctx, void *stream)
     DevState st;
     e = cudaMemcpy(&st, ctx->base + ctx->L.state, sizeof(st), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e));
-    if (st.err != kErrNone) return fail(ctx, MKV_DEVICE_TIMEOUT, "a device-side wait ran out of iterations%s");
+    if (st.err != kErrNone) {
+        char code[32];
+        snprintf(code, sizeof(code), " (wait code %d)", st.err);
+        return fail(ctx, MKV_DEVICE_TIMEOUT, "a device-side wait ran out of iterations%s", code);
+    }
     // the device-resident state is authoritative (steps replayed from a CUDA graph advance
     // it without passing through this library); the host mirror follows it
     if (ctx->prefilled) { ctx->t = st.t; ctx->n = st.n; }

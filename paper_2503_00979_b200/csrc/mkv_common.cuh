@@ -101,7 +101,9 @@ constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32;
 // __syncthreads; warp-specialised kernels give each compute group its own id)
 __device__ __forceinline__ void group_sync(int bar_id, int nthr)
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthr) : "memory");
+    // barrier.sync without .aligned (bar.sync is the aligned form): the lanes of a warp may reach this
+    // point on different paths, e.g. straight after an `if (tid < k)` block, and each counts for itself
+    asm volatile("barrier.sync %0, %1;" ::"r"(bar_id), "r"(nthr) : "memory");
 }
 
 // Per-unit epilogue, run by the group of threads that finished a unit last (`tid` in

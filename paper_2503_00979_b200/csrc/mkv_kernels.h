@@ -24,8 +24,14 @@ cudaError_t launch_decode_tc(TcPlan *plan, const DecodeArgs &a, cudaStream_t str
 // Prompt phase: fills the arena (K, V, pos, ring) and the step state from a prompt of P
 // tokens.  `a` supplies the arena pointers and shape; q/k_new/v_new/out are ignored.
 // Allocates and frees its own temporary scratch.  *launches is advanced per kernel launched.
+// Device scratch of the prompt phase, owned by the context (allocated on first use, grown when a
+// longer prompt needs more, released with the context).
+struct PrefillScratch {
+    void *ptr;
+    size_t bytes;
+};
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
-                        int P, cudaStream_t stream, unsigned long long *launches);
+                        int P, cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch);
 
 // The same prompt phase with its scratch in a fixed device array of prefill_static_max_floats()
 // floats instead of a temporary allocation; cudaErrorInvalidConfiguration if one unit's

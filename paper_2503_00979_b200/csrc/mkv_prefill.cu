@@ -257,7 +257,7 @@ __global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, in
 
 template <typename T, int D>
 cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
-                          unsigned long long *launches)
+                          unsigned long long *launches, PrefillScratch *scratch)
 {
     const int U = a.U, G = a.G, R = a.R, C = a.C;
     const int Rw = P < R ? P : R, rows = Rw * G;
@@ -270,14 +270,24 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     if (ub < 1) ub = 1;
     if (ub > (size_t)U) ub = U;
     if (ub > 65535) ub = 65535;
-    float *S = nullptr;
-    cudaError_t e = cudaMalloc(&S, ub * per_unit);
-    if (e != cudaSuccess) return e;
+    // The scratch belongs to the context and is kept until the context is destroyed: it only grows.
+    // (Allocating and freeing it around every prompt put a cudaFree of up to 1 GiB right in front
+    // of the first decode launches.)
+    cudaError_t e = cudaSuccess;
+    if (scratch->bytes < ub * per_unit) {
+        if (scratch->ptr) cudaFree(scratch->ptr);
+        scratch->ptr = nullptr;
+        scratch->bytes = 0;
+        e = cudaMalloc(&scratch->ptr, ub * per_unit);
+        if (e != cudaSuccess) { scratch->ptr = nullptr; return e; }
+        scratch->bytes = ub * per_unit;
+    }
+    float *S = static_cast<float *>(scratch->ptr);
     float *Fp = S + ub * (size_t)rows * P;
 
     const size_t logits_smem = (size_t)(kPK * (D + 4) + kPR * (D + 4) + kPK * (kPR + 1)) * sizeof(float);
     e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
-    if (e != cudaSuccess) { cudaFree(S); return e; }
+    if (e != cudaSuccess) return e;
     const size_t init_n = max((size_t)U * a.cap, (size_t)U * R * G);
     init_arena_kernel<<<(unsigned)((init_n + 255) / 256), 256, 0, stream>>>(a);
     ++*launches;
@@ -305,7 +315,6 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     *launches += 3;
     e = cudaGetLastError();
     const cudaError_t e2 = cudaStreamSynchronize(stream);
-    cudaFree(S);
     return e != cudaSuccess ? e : e2;
 }
 
@@ -394,17 +403,17 @@ cudaError_t run_prefill_static_t(const DecodeArgs &a, const T *k, const T *v, co
 }  // namespace
 
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
-                        cudaStream_t stream, unsigned long long *launches)
+                        cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch)
 {
     if (f32) {
         auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
-        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches)
-                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches);
+        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches, scratch)
+                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches, scratch);
     }
     auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
          qq = static_cast<const __nv_bfloat16 *>(q_window);
-    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches)
-                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches);
+    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches, scratch)
+                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches, scratch);
 }
 
 }  // namespace mkv

@@ -112,8 +112,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Which wait gave up (recorded in the CTA's abort flag and reported to the host)
+enum WaitCode { kWaitQEmpty = 1, kWaitKEmpty, kWaitVEmpty, kWaitQFull, kWaitKFull, kWaitTEmpty, kWaitTFull, kWaitVFull,
+                kWaitPFree, kWaitUDone, kWaitDrain };
 // Bounded wait.  Gives up after kWaitCycles or as soon as another thread has raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort, int code)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -121,7 +124,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 0) {
             if (*abort) return false;
-            if (clock64() - t0 > kWaitCycles) { *abort = 1; return false; }
+            if (clock64() - t0 > kWaitCycles) { *abort = code; return false; }
         }
     }
 }
@@ -581,14 +584,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             bool ok = true;
             RingPos rk(0, SK);
             while (ok && w.next(x)) {
-                ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag);
+                ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag, kWaitQEmpty);
                 if (!ok) break;
                 mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
                 tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
                 tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
                 for (int j = 0; j < x.nk && ok; ++j, rk.step(1, SK)) {
                     const int T = w.T0 + j, s = rk.idx;
-                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(rk.lap ^ 1), abort_flag);
+                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(rk.lap ^ 1), abort_flag, kWaitKEmpty);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_kfull + 8 * s, kStageBytes);
@@ -601,7 +604,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             if (!ok) {   // give up: let the copies already in flight land before the CTA exits
                 int dummy = 0;
                 for (int T = max(0, issued - SK); T < issued; ++T)
-                    mbar_wait(bar_kfull + 8 * (T % SK), (uint32_t)((T / SK) & 1), &dummy);
+                    mbar_wait(bar_kfull + 8 * (T % SK), (uint32_t)((T / SK) & 1), &dummy, kWaitDrain);
             }
         }
     } else if (warp == 2) {
@@ -615,7 +618,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             while (ok && w.next(x)) {
                 for (int j = 0; j < x.nk && ok; ++j, rv.step(1, SV)) {
                     const int T = w.T0 + j, s = rv.idx;
-                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag);
+                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_vfull + 8 * s, kStageBytes);
@@ -628,7 +631,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             if (!ok) {
                 int dummy = 0;
                 for (int T = max(0, issued - SV); T < issued; ++T)
-                    mbar_wait(bar_vfull + 8 * (T % SV), (uint32_t)((T / SV) & 1), &dummy);
+                    mbar_wait(bar_vfull + 8 * (T % SV), (uint32_t)((T / SV) & 1), &dummy, kWaitDrain);
             }
         }
     } else if (warp == 1) {
@@ -647,7 +650,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i)
                     if (lane + 32 * i < G * 16) qv[i] = qsrc[lane + 32 * i];
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.nitems & 1), abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.nitems & 1), abort_flag, kWaitQFull));
                 if (!ok) break;
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i) {
@@ -663,8 +666,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             }
             for (int j = 0; j < x.nk; ++j, rk.step(1, SK), rb.step(1, NB)) {
                 const int s = rk.idx, b = rb.idx;
-                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)rk.lap, abort_flag);
-                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(rb.lap ^ 1), abort_flag);
+                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)rk.lap, abort_flag, kWaitKFull);
+                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(rb.lap ^ 1), abort_flag, kWaitTEmpty);
                 ok = __all_sync(0xffffffffu, k);
                 if (!ok) break;
                 tc_fence_after();
@@ -738,7 +741,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 const int j = Tn - w.T0;
                 const int buf = rb.idx;
                 // ---- scores of this warp's 32 keys (Eq. 4-6) and the new row's logits
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)rb.lap, abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)rb.lap, abort_flag, kWaitTFull));
                 if (!ok) break;
                 tc_fence_after();
                 const int key = (x.tile0 + j) * kTile + gtid;
@@ -789,7 +792,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 
                 // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys
                 const int s = rv.idx;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag, kWaitVFull));
                 if (!ok) break;
                 const uint32_t vbase = vst_addr + s * kStageBytes;
 #pragma unroll
@@ -836,7 +839,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             // ---- the item is done: leave this warp's partial for the epilogue group
             if (ok) {
                 // the previous partial must have been read before its buffer is overwritten
-                if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag));
+                if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag, kWaitPFree));
                 if (ok) {
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
@@ -883,7 +886,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         while (ok && w.next(x)) {
             {
                 const int u = x.unit;
-                if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag))) { ok = false; break; }
+                if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag, kWaitUDone))) { ok = false; break; }
                 // merge the compute warps' partials: common reference = max of theirs
                 if (etid < G) {
                     float m = -INFINITY;
@@ -953,7 +956,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)geo.tmem_cols);
     }
-    if (tid == 0 && *abort_flag) atomicExch(&a.st->err, (int)kErrBarrierTimeout);
+    if (tid == 0 && *abort_flag) atomicCAS(&a.st->err, 0, *abort_flag);      // the first wait that gave up
     finish_cta(a, t, n, evict);
 }
 
