@@ -154,8 +154,11 @@ mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const
 mkv_status mkv_decode_steps(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                             void *out, int n_steps, void *stream);
 
-/* One decode step with HOST buffers (pinned memory recommended): copies q, k_new, v_new to
- * the device, runs the step, copies `out` back, all on `stream`; does not synchronise. */
+/* One decode step with HOST buffers, in stream order on `stream`; does not synchronise.  If all four
+ * buffers are pinned (page-locked, hence mapped into the device's address space) and the context runs the
+ * tensor-core kernel, the kernel reads q, k_new, v_new and writes `out` directly in host memory; otherwise
+ * q, k_new, v_new are copied to the device, the step runs, and `out` is copied back.  Either way the
+ * inputs must stay unchanged, and `out` is complete, once the work enqueued on `stream` has finished. */
 mkv_status mkv_decode_step_host(mkv_ctx *ctx, const void *q_host, const void *k_new_host,
                                 const void *v_new_host, void *out_host, void *stream);
 

@@ -335,6 +335,21 @@ mkv_status mkv_decode_step_host(mkv_ctx *ctx, const void *q_host, const void *k_
     cudaStream_t s = (cudaStream_t)stream;
     const size_t qb = (size_t)ctx->s.U * ctx->s.G * ctx->s.D * ctx->s.es, kb = (size_t)ctx->s.U * ctx->s.D * ctx->s.es;
     char *b = ctx->base;
+    // Pinned host buffers are reachable from the device: the tensor-core kernel then reads q, k_new, v_new and
+    // writes `out` in place over the interconnect (a few hundred KB per step, read once or twice), which saves
+    // four copy launches per step.  Anything else goes through the staging buffers.
+    if (ctx->kind == kKindTc) {
+        const void *hp[4] = {q_host, k_new_host, v_new_host, out_host};
+        void *dp[4] = {nullptr, nullptr, nullptr, nullptr};
+        bool mapped = true;
+        for (int i = 0; i < 4 && mapped; ++i) {
+            cudaPointerAttributes at;
+            mapped = cudaPointerGetAttributes(&at, hp[i]) == cudaSuccess && at.type == cudaMemoryTypeHost &&
+                     cudaHostGetDevicePointer(&dp[i], const_cast<void *>(hp[i]), 0) == cudaSuccess && dp[i] != nullptr;
+        }
+        cudaGetLastError();     // a failed query of pageable memory is not an error of this call
+        if (mapped) return mkv_decode_step(ctx, dp[0], dp[1], dp[2], dp[3], stream);
+    }
     cudaError_t e = cudaMemcpyAsync(b + ctx->L.stage_q, q_host, qb, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(b + ctx->L.stage_k, k_new_host, kb, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(b + ctx->L.stage_v, v_new_host, kb, cudaMemcpyHostToDevice, s);

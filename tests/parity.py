@@ -53,7 +53,7 @@ def pick_units(w: synth.Workload, n: int, seed: int = 0):
 
 def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chunk: int = 32, kernel: str = "auto",
                splits: int = 0, check_F_every: int = 16, device: str = "cuda:0", use_steps_call: bool = False,
-               host_call_every: int = 0) -> ParityReport:
+               host_call_every: int = 0, host_pinned: bool = True) -> ParityReport:
     dev = torch.device(device)
     st = synth.Stream(w, dev)
     tdt = synth.torch_dtype(w.dtype)
@@ -122,8 +122,10 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
         else:
             for i in range(ns):
                 if host_call_every and (done + i) % host_call_every == 0:
-                    qh, kh, vh = qs[i].cpu().pin_memory(), ks[i].cpu().pin_memory(), vs[i].cpu().pin_memory()
-                    oh = torch.empty_like(qh).pin_memory()
+                    qh, kh, vh = qs[i].cpu(), ks[i].cpu(), vs[i].cpu()
+                    oh = torch.empty_like(qh)
+                    if host_pinned:
+                        qh, kh, vh, oh = qh.pin_memory(), kh.pin_memory(), vh.pin_memory(), oh.pin_memory()
                     mk.decode_step_host(qh, kh, vh, oh)
                     torch.cuda.current_stream().synchronize()
                     outs[i].copy_(oh)

@@ -207,6 +207,15 @@ def test_tc_item_counts_give_the_same_answer(ipu):
     assert rep.evictions > 0
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_tc_host_buffers_pinned_in_place_and_pageable_staged(pinned):
+    # pinned host buffers are read and written in place by the kernel, pageable ones go through staging copies
+    w = SMALL.replace(layers=2, C=300, R=32, prompt_len=400, steps=24)
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel="tc", host_call_every=2, host_pinned=pinned)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+
+
 def test_tc_fill_phase_warmup_and_single_tile():
     rep = run_parity(SMALL.replace(C=120, R=16, prompt_len=100, steps=80), steps=80, n_units=8, kernel="tc")
     _report(rep)
