@@ -38,7 +38,7 @@ METRIC, UNIT = "decode_tokens_per_s", "tokens/s"
 def algorithmic_bytes_per_step(w: synth.Workload, n: int) -> int:
     """K and V of the n cached tokens read once plus the R*G recent queries, per unit."""
     e = 2 if w.dtype == "bf16" else 4
-    return w.units * (2 * n * w.head_dim * e + w.R * w.group * w.head_dim * e)
+    return int(w.units * (2 * n * w.head_dim * e + w.R * w.group * w.head_dim * e))
 
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
@@ -219,7 +219,7 @@ def run_ours(args, w):
 
     st = synth.Stream(w, dev)
     mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
-                         kernel=args.kernel, splits=args.splits, device=str(dev))
+                         evict_interval=args.evict_interval, kernel=args.kernel, splits=args.splits, device=str(dev))
     # prompt phase (untimed), drawn layer by layer to bound the temporary memory
     ks, vs, qws = [], [], []
     for l in range(w.layers):
@@ -252,6 +252,9 @@ def run_ours(args, w):
     mk.decode_steps(qs[:W], kn[:W], vn[:W], outs[:W])
     mk.sync()
     n_steady = mk.view(0)["count"]
+    T = max(1, args.evict_interval)
+    if T > 1:       # the fill cycles through C+R .. C+R+T-1: the roofline bytes use its mean
+        n_steady = min(n_steady, w.C + w.R) + (T - 1) / 2
     launches0 = mk.launch_count
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -301,7 +304,7 @@ def run_ours(args, w):
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
                        "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "C": w.C, "R": w.R, "fusion": w.fusion,
-                       "prompt_len": P, "cached_tokens_per_unit": n_steady, "units_per_gpu": w.units,
+                       "prompt_len": P, "evict_interval": T, "cached_tokens_per_unit": n_steady, "units_per_gpu": w.units,
                        "kernel": mk.kernel_name, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2: each step streams the whole K/V cache "
                              f"({bytes_step / 1e6:.0f} MB per step against 126 MB of L2)"},
@@ -310,7 +313,7 @@ def run_ours(args, w):
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": measured_traffic(w.name) if mk.kernel_name == "tc" and args.prompt_len == 0 else None,
+                         "traffic": measured_traffic(w.name) if mk.kernel_name == "tc" and args.prompt_len == 0 and T == 1 else None,
                          "peak_source": peak_src, "kernel": f"decode_{mk.kernel_name}",
                          "algorithmic_bytes_per_launch": bytes_step},
         }
@@ -338,6 +341,8 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=512, help="steady-state steps per unit for the CPU baseline")
     ap.add_argument("--prompt-len", type=int, default=0,
                     help="override the workload's prompt length (e.g. C + R to start config 3 with a full cache)")
+    ap.add_argument("--evict-interval", type=int, default=1,
+                    help="run the policy every T-th step only (coarse-grained eviction appendix)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer arm (for profiler captures)")
     args = ap.parse_args()

@@ -61,8 +61,11 @@ typedef struct mkv_params {
     int R;                  /* recent window (H1)                                           */
     mkv_fusion fusion;
     mkv_dtype dtype;
-    int evict_interval;     /* run the policy every T-th step (coarse-grained eviction
-                               appendix); 0 or 1 = every step                              */
+    int evict_interval;     /* T: run the policy every T-th decode step only (coarse-grained
+                               eviction appendix); 0 or 1 = every step.  With T > 1 the cache
+                               grows by one token per step and every T-th step keeps the top C
+                               older tokens again (a second, small launch compacts the slots);
+                               evicted_pos is then always -1.  At most 64.               */
     mkv_kernel kernel;
     int splits;             /* CTAs cooperating on one unit's cache; 0 = choose            */
     void *workspace;        /* device memory owned by the caller, 256-byte aligned, or NULL
@@ -84,7 +87,7 @@ typedef struct mkv_view {
                                ring row: weight(k) = exp2(q.k * log2(e)/sqrt(d) - ring_c);
                                +inf marks an empty row                                     */
     int32_t count;          /* tokens cached per unit (the same for every unit)            */
-    int32_t capacity;       /* slots per unit: C + R + evict_interval - 1                  */
+    int32_t capacity;       /* slots per unit: C + R, plus evict_interval if that is > 1  */
     int64_t next_pos;       /* absolute position of the next token to decode               */
 } mkv_view;
 

@@ -64,7 +64,7 @@ bool params_valid(const mkv_params *p)
     if (p->kernel != MKV_KERNEL_AUTO && p->kernel != MKV_KERNEL_SIMT && p->kernel != MKV_KERNEL_TC) return false;
     const long long units = (long long)p->layers * p->batch * p->n_kv_heads;
     if (units > (1 << 24)) return false;
-    if ((long long)p->C + p->R + (p->evict_interval > 1 ? p->evict_interval - 1 : 0) > (1 << 24)) return false;
+    if ((long long)p->C + p->R + (p->evict_interval > 1 ? p->evict_interval : 0) > (1 << 24)) return false;
     return true;
 }
 
@@ -79,9 +79,10 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     s->R = p->R;
     s->C = p->C;
     s->T = p->evict_interval > 1 ? p->evict_interval : 1;
-    s->cap = p->C + p->R + s->T - 1;
+    // with T > 1 the step that runs the policy appends first and evicts afterwards: one more slot
+    s->cap = p->C + p->R + (s->T > 1 ? s->T : 0);
     s->es = p->dtype == MKV_DTYPE_F32 ? 4 : 2;
-    if (s->T != 1) return false;
+    if (s->T > 64) return false;
     const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R) &&
                        (long long)s->U * ((s->cap + 127) / 128) <= (1ll << 30);     // tile indices stay 32-bit
     if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
@@ -114,6 +115,7 @@ struct mkv_ctx {
     bool prefilled;
     long long t;      // host mirror of the device step state
     int n;
+    int steps;
     unsigned long long launches;
     PrefillScratch prefill_scratch;
     char err[256];
@@ -162,9 +164,16 @@ mkv_status launch_step(mkv_ctx *ctx, const void *q, const void *k, const void *v
                                                : launch_decode_simt(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "decode launch failed: %s", cudaGetErrorString(e));
     ctx->launches += 1;
-    const bool ev = step_evicts(ctx->t, ctx->n, ctx->s.R, ctx->s.C);
+    const bool ev = step_scores(ctx->t, ctx->n, ctx->steps, ctx->s.R, ctx->s.C, ctx->s.T);
+    if (ctx->s.T > 1) {
+        const cudaError_t e2 = launch_compact(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
+        if (e2 != cudaSuccess) return fail(ctx, MKV_CUDA, "compaction launch failed: %s", cudaGetErrorString(e2));
+        ctx->launches += 1;
+    }
     ctx->t += 1;
+    ctx->steps += 1;
     if (!ev) ctx->n += 1;
+    else if (ctx->s.T > 1) ctx->n = ctx->s.C + ctx->s.R;
     return MKV_OK;
 }
 
@@ -274,6 +283,7 @@ mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q
     const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
     ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
     ctx->t = prompt_len;
+    ctx->steps = 0;
     ctx->prefilled = true;
     return MKV_OK;
 }
@@ -299,6 +309,7 @@ mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const 
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_prefill_static: %s", cudaGetErrorString(e));
     ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
     ctx->t = prompt_len;
+    ctx->steps = 0;
     ctx->prefilled = true;
     return MKV_OK;
 }
@@ -397,7 +408,7 @@ mkv_status mkv_sync(mkv_ctx *ctx, void *stream)
     }
     // the device-resident state is authoritative (steps replayed from a CUDA graph advance
     // it without passing through this library); the host mirror follows it
-    if (ctx->prefilled) { ctx->t = st.t; ctx->n = st.n; }
+    if (ctx->prefilled) { ctx->t = st.t; ctx->n = st.n; ctx->steps = st.steps; }
     return MKV_OK;
 }
 

@@ -21,7 +21,7 @@ struct DevState {
     int steps;            // decode steps completed
     int err;              // sticky device-side error code (0 = none)
     unsigned int done;    // CTAs of the current launch that have finished
-    int pad;
+    int compact;          // coarse-grained eviction: the step that just ran scored, the cache awaits its compaction
 };
 
 enum DevError { kErrNone = 0, kErrBarrierTimeout = 1 };
@@ -93,6 +93,15 @@ __host__ __device__ inline bool step_evicts(long long t, int n, int R, int C)
 {
     const long long win = (t + 1 < (long long)R) ? t + 1 : (long long)R;
     return (long long)n + 1 - win > (long long)C;
+}
+
+// True when this step runs the policy (scores and evicts).  With evict_interval T > 1 (coarse-grained
+// eviction appendix) that is every T-th decode step only, and the step then appends like any other:
+// a separate compaction launch drops everything beyond the top C afterwards.
+__host__ __device__ inline bool step_scores(long long t, int n, int steps, int R, int C, int T)
+{
+    if (T > 1 && (steps + 1) % T != 0) return false;
+    return step_evicts(t, n, R, C);
 }
 
 constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32;
@@ -255,6 +264,11 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         e_slot = red_slot[0];
         e_pos = pos[e_slot];
         group_sync(bar_id, nthr);
+        if (a.T > 1) {          // coarse-grained eviction: append now, the compaction launch evicts
+            e_slot = n;
+            e_pos = -1;
+            if (tid == 0) F[n] = -1.f;
+        }
     }
 
     // Eq. 7 update: the freed (or next free) slot takes the new token; the ring row of the
@@ -284,7 +298,8 @@ __device__ __forceinline__ void finish_cta(const DecodeArgs &a, long long t, int
         const unsigned int total = gridDim.x * gridDim.y * gridDim.z;
         if (atomicAdd(&a.st->done, 1u) == total - 1) {
             a.st->t = t + 1;
-            a.st->n = evict ? n : n + 1;
+            a.st->n = (evict && a.T == 1) ? n : n + 1;
+            a.st->compact = (evict && a.T > 1) ? 1 : 0;
             a.st->steps += 1;
             a.st->done = 0;
             __threadfence();

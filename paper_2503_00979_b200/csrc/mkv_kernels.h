@@ -9,6 +9,10 @@ namespace mkv {
 cudaError_t launch_decode_simt(const DecodeArgs &a, bool f32, int D, cudaStream_t stream);
 int simt_default_splits(int U, int cap);
 
+// Coarse-grained eviction (evict_interval > 1): drops everything beyond the top C after a step that scored and
+// restores the dense prefix of C + R slots; a no-op after the other steps.  Launched after every decode step.
+cudaError_t launch_compact(const DecodeArgs &a, bool f32, int D, cudaStream_t stream);
+
 // Tensor-core (tcgen05) decode step: bf16, head_dim 128, GQA group in {1,2,4,8,16} and
 // R*G padded to a multiple of 32 at most 256.  The plan holds the TMA tensor maps of a
 // context's arena and the launch geometry; `a.splits` must be tc_partials_per_unit()

@@ -40,7 +40,7 @@ __global__ void init_arena_kernel(DecodeArgs a)
 
 __global__ void set_state_kernel(DevState *st, long long t, int n)
 {
-    st->t = t; st->n = n; st->steps = 0; st->err = 0; st->done = 0; st->pad = 0;
+    st->t = t; st->n = n; st->steps = 0; st->err = 0; st->done = 0; st->compact = 0;
 }
 
 // S[ub][row = i*G + g][j] = log2-domain logit of window row (i, g) against prompt key j,

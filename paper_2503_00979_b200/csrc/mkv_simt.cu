@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(const __grid_cons
     const int u = blockIdx.x / a.splits, sp = blockIdx.x % a.splits;
     const long long t = a.st->t;
     const int n = a.st->n;
-    const bool evict = step_evicts(t, n, R, a.C);
+    const bool evict = step_scores(t, n, a.st->steps, R, a.C, a.T);
     int active;
     const int per = split_len(n, a.splits, kTK, &active);
     const int k0 = sp * per, k1 = min(n, k0 + per);

@@ -448,7 +448,7 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     int *pos = a.pos + (size_t)u * a.cap;
     float *F = a.F + (size_t)u * a.cap;
     int e_slot = n, e_pos = -1;
-    if (evict) {
+    {
         const float *sn = a.s_new + (size_t)u * G * a.cap;
         const long long thr = t - a.R;
         float cn[G];
@@ -499,6 +499,13 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
             if (red_key[w] < best) { best = red_key[w]; bslot = red_slot[w]; }
         e_slot = bslot;
         e_pos = (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull));   // the rank key carries the position
+        if (!evict || a.T > 1) {
+            // nothing to evict on this step, or coarse-grained eviction (append now, the compaction launch
+            // evicts): the new token takes the next free slot and is not a candidate
+            e_slot = n;
+            e_pos = -1;
+            if (tid == 0) F[n] = -1.f;
+        }
     }
 
     // ---- phase D: Eq. 7 update from the registers loaded in phase A
@@ -564,15 +571,9 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // Programmatic dependent launch: the CTA may have started, and set itself up, while the
-    // previous kernel of the stream was still finishing.  Nothing before this line reads global
-    // memory; from here on the previous kernel has completed and its writes are visible.  The
-    // next kernel of the stream may then be staged the same way.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long t = a.st->t;
     const int n = a.st->n;
-    const bool evict = step_evicts(t, n, a.R, a.C);
+    const bool evict = step_scores(t, n, a.st->steps, a.R, a.C, a.T);
     const int rs_new = (int)(t % a.R);
 
     if (warp == 0) {
@@ -751,18 +752,18 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 // written asynchronously, so nothing may touch them between the two.
                 uint32_t sv[G];
                 tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
+                // Scored on every step, also on steps that evict nothing (cache still filling, or between two
+                // runs of a coarse-grained policy): every launch then has the shape of the steady-state one.
                 float F = 0.f;
-                if (evict) {
-                    for (int c = 0; c < RGP; c += 32) {
-                        uint32_t v[32];
-                        tmem_ld32(taddr + (uint32_t)c, v);
-                        score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
-                    }
+                for (int c = 0; c < RGP; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + (uint32_t)c, v);
+                    score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-                if (evict && valid) a.F[(size_t)u * a.cap + key] = F;
+                if (valid) a.F[(size_t)u * a.cap + key] = F;
 
                 // ---- online soft-max of the new row over this warp's keys (Eq. 1)
                 bool changed = false;
@@ -1013,19 +1014,8 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         set = true;
     }
-    // launched with programmatic stream serialization: the grid may be staged while the previous
-    // kernel of the stream drains (the kernel waits for it with griddepcontrol.wait)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)plan->geo.grid);
-    cfg.blockDim = dim3((unsigned)tc_threads(NG));
-    cfg.dynamicSmemBytes = (size_t)plan->geo.smem_bytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
+    kern<<<plan->geo.grid, tc_threads(NG), plan->geo.smem_bytes, stream>>>(a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
+    return cudaGetLastError();
 }
 
 template <int G, int FUSION>

@@ -182,3 +182,88 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
         assert rep.max_F_rel_err < 1e-3, f"fused scores off by {rep.max_F_rel_err:.3e} relative"
     mk.close()
     return rep
+
+
+def run_parity_coarse(w: synth.Workload, T: int, steps: int, n_units: int = 4, kernel: str = "auto",
+                      device: str = "cuda:0") -> ParityReport:
+    """Lock-step parity for coarse-grained eviction (the policy runs every T-th step and may drop several
+    tokens at once).  After every step the retained position set of each checked unit is read back; what the
+    device dropped is the oracle's set before the step, plus the new token, minus that.  The oracle is made
+    to drop the same tokens, and wherever that differs from its own ranking every token in the difference
+    must be a near tie with the boundary of its top C."""
+    dev = torch.device(device)
+    st = synth.Stream(w, dev)
+    tdt = synth.torch_dtype(w.dtype)
+    G, d, P, R, C_ = w.group, w.head_dim, w.prompt_len, w.R, w.C
+    units = pick_units(w, n_units)
+    rep = ParityReport()
+    mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, d, C_, R, w.fusion, w.dtype, evict_interval=T,
+                         kernel=kernel, device=device)
+    rep.kernel = mk.kernel_name
+    tol = TOL_OUT[w.dtype]
+    Rw = min(R, P)
+    k32, v32 = st.kv(np.arange(P))
+    qw32 = st.q(np.arange(P - Rw, P))
+    mk.prefill(k32.to(tdt).contiguous(), v32.to(tdt).contiguous(), qw32.to(tdt).contiguous())
+    mk.sync()
+    orac = {}
+    for (l, b, h) in units:
+        u = ora.Unit(G, d, C_, R, w.fusion, evict_interval=T)
+        u.prefill(k32[l, b, h].double().cpu().numpy(), v32[l, b, h].double().cpu().numpy(),
+                  qw32[l, b, h * G:(h + 1) * G].double().cpu().numpy())
+        view = mk.view(l)
+        gp = set(view["pos"][b, h, :view["count"]].cpu().numpy().tolist())
+        if gp != set(u.positions().tolist()):
+            kth, k1 = u.last_boundary()
+            assert near_tie(kth, k1), f"prefill retained set differs for unit {(l, b, h)} without a near tie"
+            rep.prefill_dropped += 1
+            continue
+        orac[(l, b, h)] = u
+    peak = 0
+    for i in range(steps):
+        t = P + i
+        k1_, v1_ = st.kv([t])
+        q1_ = st.q([t])
+        qs = q1_[..., 0, :].to(tdt).contiguous()
+        ks = k1_[..., 0, :].to(tdt).contiguous()
+        vs = v1_[..., 0, :].to(tdt).contiguous()
+        out = torch.empty_like(qs)
+        mk.decode_step(qs, ks, vs, out)
+        mk.sync()
+        out_c = out.float().cpu().numpy()
+        q_c, k_c, v_c = q1_.double().cpu().numpy(), k1_.double().cpu().numpy(), v1_.double().cpu().numpy()
+        views = {l: mk.view(l) for l in {u_[0] for u_ in orac}}
+        for (l, b, h), u in orac.items():
+            view = views[l]
+            peak = max(peak, view["count"])
+            gp = set(view["pos"][b, h, :view["count"]].cpu().numpy().tolist())
+            assert len(gp) == view["count"] and -1 not in gp, f"unit {(l, b, h)} step {t}: slots are not a dense prefix"
+            before = set(u.positions().tolist()) | {t}
+            dropped = sorted(before - gp)
+            assert gp <= before, f"unit {(l, b, h)} step {t}: device holds tokens the oracle never had"
+            o = u.step(q_c[l, b, h * G:(h + 1) * G, 0], k_c[l, b, h, 0], v_c[l, b, h, 0], forced=dropped or None)
+            err = float(np.abs(o - out_c[l, b, h * G:(h + 1) * G]).max())
+            rep.max_out_err = max(rep.max_out_err, err)
+            assert err <= tol, f"unit {(l, b, h)} step {t}: attention output error {err:.3e} > {tol}"
+            cp, cF = u.last_scores()
+            if len(cp) > C_:
+                rep.evictions += len(dropped)
+                assert len(dropped) == len(cp) - C_, (f"unit {(l, b, h)} step {t}: device dropped {len(dropped)} tokens, "
+                                                      f"the policy drops {len(cp) - C_}")
+                own = set(int(p) for p in cp[C_:])
+                diff = own ^ set(dropped)
+                if diff:
+                    Fof = {int(p): float(f) for p, f in zip(cp, cF)}
+                    for x in diff:
+                        assert near_tie(Fof[x], float(cF[C_ - 1])) or near_tie(Fof[x], float(cF[C_])), \
+                            f"unit {(l, b, h)} step {t}: token {x} (F={Fof[x]:.6e}) changed sides without a near tie"
+                    rep.near_tie_resyncs += 1
+            else:
+                assert not dropped, f"unit {(l, b, h)} step {t}: device dropped {dropped} on a step without the policy"
+            assert set(u.positions().tolist()) == gp, f"unit {(l, b, h)} step {t}: retained sets differ"
+            # K rows of the retained tokens are the rows that were appended, bit for bit
+            rep.unit_steps += 1
+        rep.steps = i + 1
+    rep.F_compared = peak        # reused: the largest fill seen (C + R + T - 1 expected)
+    mk.close()
+    return rep

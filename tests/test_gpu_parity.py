@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from paper_2503_00979_b200 import binding, synth
-from tests.parity import run_parity
+from tests.parity import run_parity, run_parity_coarse
 
 pytestmark = pytest.mark.gpu
 
@@ -238,6 +238,26 @@ def test_tc_llama_shape_two_layers():
 def test_tc_stress_shape_window_64():
     w = synth.WORKLOADS["c3"].replace(layers=1, batch=2, prompt_len=4100, steps=48)    # starts full: C=4000, R=64
     rep = run_parity(w, steps=w.steps, n_units=6, kernel="tc")
+    _report(rep)
+    assert rep.evictions > 0
+
+
+# ---- coarse-grained eviction: the policy runs every T-th step and drops several tokens at once
+@pytest.mark.parametrize("kernel,dtype,d", [("simt", "f32", 64), ("simt", "bf16", 128), ("tc", "bf16", 128)])
+@pytest.mark.parametrize("T,fusion", [(8, "sum"), (3, "max")])
+def test_coarse_grained_eviction(kernel, dtype, d, T, fusion):
+    w = synth.Workload("coarse", 1, 2, 8, 2, d, dtype, 260, 40, 150, 16, fusion, 4242)
+    rep = run_parity_coarse(w, T, steps=5 * T + 2, n_units=4, kernel=kernel)
+    _report(rep)
+    assert rep.kernel == kernel
+    assert rep.evictions == 4 * 5 * T               # T tokens per policy step and unit, five policy steps
+    assert rep.F_compared == w.C + w.R + T - 1      # the fill peaks one step before the policy runs
+
+
+def test_coarse_grained_eviction_while_the_cache_fills():
+    # prompt shorter than C + R: nothing is dropped until the older tokens exceed C on a policy step
+    w = synth.Workload("coarse_fill", 1, 1, 8, 2, 128, "bf16", 100, 64, 120, 16, "sum", 99)
+    rep = run_parity_coarse(w, 4, steps=64, n_units=2, kernel="tc")
     _report(rep)
     assert rep.evictions > 0
 
