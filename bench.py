@@ -43,7 +43,7 @@ def algorithmic_bytes_per_step(w: synth.Workload, n: int) -> int:
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
 # capture of a launch of that workload), valid only for the kernel sources it was taken with.
-_TRAFFIC = {"c1": {"bytes": 299.8e6, "sources_sha256": "81a235add8b9319f7e3b3cf64c5fcf21b70bff85ec2b8c25345ef8f6981d23a8"}}
+_TRAFFIC = {"c1": {"bytes": 298.6e6, "sources_sha256": "646a4652456151d13e10fd94c46bbfffabb984ff2d03877ee1f443a00f8c1a2b"}}
 
 
 def measured_traffic(workload: str):
