@@ -242,6 +242,59 @@ def test_tc_stress_shape_window_64():
     assert rep.evictions > 0
 
 
+def test_full_size_config1_fill_phase_launched_back_to_back():
+    # a prompt shorter than C + R: 96 steps that append without evicting, all launches enqueued without a
+    # synchronisation in between (the regime in which a kernel variant that skipped the scoring used to fault)
+    w = synth.WORKLOADS["c1"].replace(prompt_len=1500)
+    rep = run_parity(w, steps=96, n_units=6, kernel="auto", chunk=48, use_steps_call=True)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.unit_steps == 6 * 96
+
+
+def test_full_size_config1_coarse_grained_launched_back_to_back():
+    # T = 8 at the benchmark's size, 64 steps enqueued at once: the fill must cycle C+R .. C+R+T-1 and every
+    # unit must end with a dense prefix of distinct positions that contains the whole recent window
+    w = synth.WORKLOADS["c1"]
+    T, steps = 8, 64
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    P = w.prompt_len
+    mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
+                         evict_interval=T)
+    ks, vs, qs = [], [], []
+    for l in range(w.layers):
+        k, v = st.kv(np.arange(P), [l])
+        ks.append(k.bfloat16()); vs.append(v.bfloat16()); qs.append(st.q(np.arange(P - w.R, P), [l]).bfloat16())
+    mk.prefill(torch.cat(ks).contiguous(), torch.cat(vs).contiguous(), torch.cat(qs).contiguous())
+    pos = np.arange(P, P + steps)
+    kk, vv = st.kv(pos)
+    q = st.q(pos).permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    kn = kk.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    vn = vv.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    out = torch.empty_like(q)
+    mk.decode_steps(q, kn, vn, out)
+    mk.sync()
+    assert torch.isfinite(out.float()).all()
+    view = mk.view(w.layers - 1)
+    assert view["count"] == w.C + w.R                      # 64 = 8 policy steps: just compacted
+    p = view["pos"][:, :, :view["count"]].cpu().numpy()
+    for b in range(p.shape[0]):
+        for h in range(p.shape[1]):
+            row = p[b, h]
+            assert len(set(row.tolist())) == len(row) and row.min() >= 0
+            assert set(range(P + steps - w.R, P + steps)) <= set(row.tolist())
+    assert (view["pos"][:, :, view["count"]:].cpu().numpy() == -1).all()
+    mk.close()
+
+
+def test_longgenbench_shape_window_200_uses_the_cuda_core_kernel():
+    # R = 200 with a 4K budget (the LongGenBench setting): R*G = 800 rows do not fit the tensor-core kernel
+    w = synth.Workload("r200", 1, 1, 8, 2, 128, "bf16", 4200, 24, 3896, 200, "sum", 31)
+    rep = run_parity(w, steps=w.steps, n_units=2, kernel="auto", check_F_every=8)
+    _report(rep)
+    assert rep.kernel == "simt" and rep.evictions == 2 * 24
+
+
 # ---- coarse-grained eviction: the policy runs every T-th step and drops several tokens at once
 @pytest.mark.parametrize("kernel,dtype,d", [("simt", "f32", 64), ("simt", "bf16", 128), ("tc", "bf16", 128)])
 @pytest.mark.parametrize("T,fusion", [(8, "sum"), (3, "max")])
