@@ -74,3 +74,16 @@ def test_no_device_means_an_error_not_a_fallback(lib):
         pytest.skip("a device is present")
     st, h = binding.mkv_create(1, 1, 8, 2, 64, 16, 4, 0)
     assert st == binding.CUDA and h is None
+
+
+def test_coarse_grained_eviction_adds_its_interval_to_the_capacity(lib):
+    # evict_interval T > 1: the cache holds up to C + R + T tokens (the scoring step appends before it drops)
+    p = binding.mkv_default_params()
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 2, 1, 8, 2, 128, 1000, 32
+    base = binding.mkv_workspace_bytes(p)
+    p.evict_interval = 8
+    grown = binding.mkv_workspace_bytes(p)
+    units, row = 2 * 1 * 2, 128 * 2
+    assert grown - base >= 2 * units * 8 * row          # at least K and V rows of the 8 extra slots
+    p.evict_interval = 65                               # beyond what one compaction handles
+    assert binding.mkv_workspace_bytes(p) == 0
