@@ -138,6 +138,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 
+// brings a tensor map into the descriptor cache ahead of its first copy
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -554,6 +560,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const uint32_t bar_udone = smem_u32(bars + 44);                    // all compute warps have left their partial of a unit
     const uint32_t bar_pfree = smem_u32(bars + 48);                    // [8] a compute warp's partial has been read
 
+    // The step state (written by the previous launch) and the tensor maps are fetched while the
+    // barriers and TMEM are set up: both are on the way to the first tile.
+    const long long t = a.st->t;
+    const int n = a.st->n;
+    const int steps_done = a.st->steps;
+    if (tid == 0) { prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); }
+    if (tid == 64) prefetch_tensormap(&tmV);
+
     if (tid == 0) {
         for (int s = 0; s < SK; ++s) { mbar_init(bar_kfull + 8 * s, 1); mbar_init(bar_kempty + 8 * s, 1); }
         for (int s = 0; s < SV; ++s) { mbar_init(bar_vfull + 8 * s, 1); mbar_init(bar_vempty + 8 * s, 4); }
@@ -571,10 +585,21 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const long long t = a.st->t;
-    const int n = a.st->n;
-    const bool evict = step_scores(t, n, a.st->steps, a.R, a.C, a.T);
+    const bool evict = step_scores(t, n, steps_done, a.R, a.C, a.T);
     const int rs_new = (int)(t % a.R);
+    // Every thread of this CTA holds its copy of the step state (the barrier above orders their reads
+    // before this point), so the CTA can be counted now: the last CTA of the launch to get here advances
+    // the state for the next launch while the tiles stream, instead of at the tail of the kernel.
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(&a.st->done, 1u) == gridDim.x - 1) {
+            a.st->t = t + 1;
+            a.st->n = (evict && a.T == 1) ? n : n + 1;
+            a.st->compact = (evict && a.T > 1) ? 1 : 0;
+            a.st->steps = steps_done + 1;
+            a.st->done = 0;
+        }
+    }
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer: query ring and K tiles (one lane)
@@ -793,7 +818,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 
                 // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys
                 const int s = rv.idx;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag, kWaitVFull));
+                // A V stage is refilled for the two compute groups in turn whenever the ring has an odd number of
+                // stages, and a parity wait cannot tell "this load has landed" from "the load before the previous
+                // one has landed".  So first make sure the previous load of this stage has been consumed (the same
+                // wait the producer does before it refills the stage); only then is the parity of the full barrier
+                // unambiguous.
+                bool vok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty);
+                vok = vok && mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag, kWaitVFull);
+                ok = __all_sync(0xffffffffu, vok);
                 if (!ok) break;
                 const uint32_t vbase = vst_addr + s * kStageBytes;
 #pragma unroll
@@ -958,7 +990,6 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         tmem_dealloc(tmem_base, (uint32_t)geo.tmem_cols);
     }
     if (tid == 0 && *abort_flag) atomicCAS(&a.st->err, 0, *abort_flag);      // the first wait that gave up
-    finish_cta(a, t, n, evict);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
