@@ -818,11 +818,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 
                 // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys
                 const int s = rv.idx;
-                // A V stage is refilled for the two compute groups in turn whenever the ring has an odd number of
-                // stages, and a parity wait cannot tell "this load has landed" from "the load before the previous
-                // one has landed".  So first make sure the previous load of this stage has been consumed (the same
-                // wait the producer does before it refills the stage); only then is the parity of the full barrier
-                // unambiguous.
+                // A V stage serves the two compute groups in turn whenever the ring has an odd number of stages, and
+                // a parity wait cannot tell "this load has landed" from "the load before the previous one has
+                // landed".  The accumulator buffers keep the groups close enough for that never to matter; waiting
+                // for the previous load of the stage to be consumed first (the wait the producer does before it
+                // refills the stage) makes the full barrier's parity unambiguous without relying on that.
                 bool vok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty);
                 vok = vok && mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag, kWaitVFull);
                 ok = __all_sync(0xffffffffu, vok);
@@ -863,6 +863,12 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                         }
                     }
                 }
+                // The V tile was read through the generic proxy (ldmatrix); the producer refills the stage through the
+                // async proxy (TMA).  An mbarrier arrive/wait pair orders accesses of one proxy only, so every lane
+                // fences its reads against later async-proxy writes before the stage is handed back.  Without this
+                // fence a refill now and then overtook the last reads of a tile (one 16-column block of one warp's
+                // keys came out wrong, about ten times in 48 steps of 256 units).
+                fence_proxy_async();
                 __syncwarp();                               // every lane has read its rows of the V tile
                 if (lane == 0) mbar_arrive(bar_vempty + 8 * s);
                 ++seg_tiles;

@@ -374,6 +374,45 @@ def test_tc_matches_cuda_core_kernel_on_device():
     assert torch.allclose(res["simt"][2], res["tc"][2], rtol=0, atol=2e-4)
 
 
+@pytest.mark.parametrize("prompt_len,steps", [(4096, 48), (1500, 96)])
+def test_full_size_config1_every_unit_matches_cuda_core_kernel(prompt_len, steps):
+    # Every unit of config 1 on every step, launches enqueued back to back, repeated: the tensor-core kernel against
+    # the CUDA-core kernel (the oracle follows a handful of units only).  This is the test that shows a V stage being
+    # refilled under its last reads: one 16-column block of the output of a unit whose tiles end a CTA's range came
+    # out wrong about ten times per repetition before the readers fenced their reads against the refill.
+    w = synth.WORKLOADS["c1"].replace(prompt_len=prompt_len)
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    P, Rw = prompt_len, min(w.R, prompt_len)
+    ks, vs, qs = [], [], []
+    for l in range(w.layers):
+        k, v = st.kv(np.arange(P), [l])
+        ks.append(k.bfloat16()); vs.append(v.bfloat16()); qs.append(st.q(np.arange(P - Rw, P), [l]).bfloat16())
+    kp, vp, qp = torch.cat(ks).contiguous(), torch.cat(vs).contiguous(), torch.cat(qs).contiguous()
+    del ks, vs, qs
+    pos = np.arange(P, P + steps)
+    kk, vv = st.kv(pos)
+    qn = st.q(pos).permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    kn = kk.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    vn = vv.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+
+    def run(kernel):
+        mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
+                             kernel=kernel)
+        assert mk.kernel_name == kernel
+        mk.prefill(kp, vp, qp)
+        out = mk.decode_steps(qn, kn, vn)
+        mk.sync()
+        res = out.float()
+        mk.close()
+        return res
+
+    ref = run("simt")
+    for _ in range(5):
+        err = float((run("tc") - ref).abs().max())
+        assert err <= 2e-2, f"tensor-core and CUDA-core outputs differ by {err:.3e}"
+
+
 @pytest.mark.parametrize("ipu", [0, 1])
 def test_tc_runs_are_bitwise_reproducible(ipu):
     # static work assignment and fixed merge order: two runs on the same inputs agree bit for bit
