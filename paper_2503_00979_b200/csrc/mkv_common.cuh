@@ -13,8 +13,9 @@ constexpr int kMaxGroup = 16;     // largest supported GQA group size
 constexpr int kFusionSum = 0;
 constexpr int kFusionMax = 1;
 
-// Device-resident step state.  Kernels read it at entry; the last CTA of a launch to finish
-// advances it, so consecutive launches need no host-side step index.
+// Device-resident step state.  Kernels read it at entry and one CTA of each launch advances it
+// (the last one to finish in the CUDA-core kernel, the last one to have read it in the
+// tensor-core kernel), so consecutive launches need no host-side step index.
 struct DevState {
     long long t;          // absolute position of the token being decoded
     int n;                // tokens cached per unit before this step
