@@ -374,13 +374,16 @@ def test_tc_matches_cuda_core_kernel_on_device():
     assert torch.allclose(res["simt"][2], res["tc"][2], rtol=0, atol=2e-4)
 
 
-@pytest.mark.parametrize("prompt_len,steps", [(4096, 48), (1500, 96)])
-def test_full_size_config1_every_unit_matches_cuda_core_kernel(prompt_len, steps):
-    # Every unit of config 1 on every step, launches enqueued back to back, repeated: the tensor-core kernel against
-    # the CUDA-core kernel (the oracle follows a handful of units only).  This is the test that shows a V stage being
-    # refilled under its last reads: one 16-column block of the output of a unit whose tiles end a CTA's range came
-    # out wrong about ten times per repetition before the readers fenced their reads against the refill.
-    w = synth.WORKLOADS["c1"].replace(prompt_len=prompt_len)
+@pytest.mark.parametrize("name,prompt_len,steps,reps", [("c1", 4096, 48, 5), ("c1", 1500, 96, 5), ("c2", 2048, 10, 2),
+                                                        ("c3", 4100, 8, 2)])
+def test_full_size_every_unit_matches_cuda_core_kernel(name, prompt_len, steps, reps):
+    # Every unit of a benchmark configuration on every step, launches enqueued back to back, repeated: the
+    # tensor-core kernel against the CUDA-core kernel (the oracle follows a handful of units only).  This is the
+    # test that shows a V stage being refilled under its last reads: on config 1, one 16-column block of the output
+    # of a unit whose tiles end a CTA's range came out wrong about ten times per repetition before the readers
+    # fenced their reads against the refill.  Configs 2 and 3 run fewer steps: their CUDA-core reference takes
+    # tens of milliseconds per step.
+    w = synth.WORKLOADS[name].replace(prompt_len=prompt_len)
     dev = torch.device("cuda:0")
     st = synth.Stream(w, dev)
     P, Rw = prompt_len, min(w.R, prompt_len)
@@ -408,9 +411,11 @@ def test_full_size_config1_every_unit_matches_cuda_core_kernel(prompt_len, steps
         return res
 
     ref = run("simt")
-    for _ in range(5):
-        err = float((run("tc") - ref).abs().max())
-        assert err <= 2e-2, f"tensor-core and CUDA-core outputs differ by {err:.3e}"
+    for _ in range(reps):
+        # both outputs are rounded to bf16: allow the absolute tolerance of the parity tests plus one bf16 ulp of
+        # the value (config 2's attention sink gives outputs beyond 4, where one ulp is 2^-5)
+        excess = float(((run("tc") - ref).abs() - 2e-2 - ref.abs() * 2 ** -7).max())
+        assert excess <= 0, f"tensor-core and CUDA-core outputs differ by {excess:.3e} more than the tolerance"
 
 
 @pytest.mark.parametrize("ipu", [0, 1])
