@@ -560,11 +560,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const uint32_t bar_udone = smem_u32(bars + 44);                    // all compute warps have left their partial of a unit
     const uint32_t bar_pfree = smem_u32(bars + 48);                    // [8] a compute warp's partial has been read
 
-    // The step state (written by the previous launch) and the tensor maps are fetched while the
-    // barriers and TMEM are set up: both are on the way to the first tile.
-    const long long t = a.st->t;
-    const int n = a.st->n;
-    const int steps_done = a.st->steps;
+    // The tensor maps (kernel parameters) are fetched while the barriers and TMEM are set up.
     if (tid == 0) { prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); }
     if (tid == 64) prefetch_tensormap(&tmV);
 
@@ -584,6 +580,18 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+
+    // Programmatic dependent launch: this grid may have been started while the grid before it in the stream was
+    // still draining (a CTA gets an SM as soon as that grid's CTA there has exited), so everything above ran
+    // early.  Nothing that grid wrote - step state, cache rows, query ring - is read before this wait, which
+    // returns once that grid has completed and its memory operations are visible.  The next grid in the stream is
+    // released at once: it parks at the same wait.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const long long t = a.st->t;
+    const int n = a.st->n;
+    const int steps_done = a.st->steps;
+    __syncthreads();
 
     const bool evict = step_scores(t, n, steps_done, a.R, a.C, a.T);
     const int rs_new = (int)(t % a.R);
@@ -1051,8 +1059,19 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         set = true;
     }
-    kern<<<plan->geo.grid, tc_threads(NG), plan->geo.smem_bytes, stream>>>(a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
-    return cudaGetLastError();
+    // launched with programmatic stream serialisation: the kernel orders itself behind its predecessor with
+    // griddepcontrol.wait (see the kernel's prologue)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan->geo.grid);
+    cfg.blockDim = dim3(tc_threads(NG));
+    cfg.dynamicSmemBytes = plan->geo.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, a, plan->tmK, plan->tmV, plan->tmQ, plan->geo);
 }
 
 template <int G, int FUSION>
