@@ -56,12 +56,16 @@ class ShadowMorphKV:
     by a plain Python sort and also finds the best size-C subset by exhaustive enumeration.
     """
 
-    def __init__(self, G, d, C, R, fusion):
+    def __init__(self, G, d, C, R, fusion, evict_interval=1):
         self.G, self.d, self.C, self.R, self.fusion = G, d, C, R, fusion
+        # coarse-grained eviction (appendix): the policy runs on generation steps T, 2T, 3T, ... only
+        self.T = evict_interval
+        self.generated = 0
         self.keys, self.vals = {}, {}
         self.profile = {}  # position -> list over g of {pos: weight}
         self.cached = set()
         self.t = 0
+        self.last_F, self.last_ranked, self.last_dropped = None, None, []
 
     def prefill(self, k, v, qwin):
         P = k.shape[0]
@@ -91,12 +95,13 @@ class ShadowMorphKV:
 
     def _select(self):
         cand = self.cached - self._window()
-        self.last_F = None
+        self.last_F, self.last_dropped = None, []
         if len(cand) > self.C:
             F = self._fused(cand)
             ranked = sorted(cand, key=lambda p: (-F[p], p))
             self.last_F = F
             self.last_ranked = ranked
+            self.last_dropped = sorted(ranked[self.C:])
             self.cached -= set(ranked[self.C:])
 
     def step(self, q, k_new, v_new):
@@ -111,5 +116,8 @@ class ShadowMorphKV:
             out[g] = sum(wj * self.vals[j] for wj, j in zip(w, J))
         self.cached.add(t)
         self.t = t + 1
-        self._select()
+        self.generated += 1
+        self.last_F, self.last_dropped = None, []
+        if self.generated % self.T == 0:
+            self._select()
         return out

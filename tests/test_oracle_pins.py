@@ -292,6 +292,43 @@ def test_coarse_grained_eviction_bounds(oracle):
     assert sizes[T - 1::T] == [w.C + w.R] * (64 // T)
 
 
+@pytest.mark.parametrize("fusion", ["sum", "max"])
+@pytest.mark.parametrize("T", [2, 3, 8])
+@pytest.mark.parametrize("G,C,R,P", [(1, 3, 2, 4), (2, 4, 3, 9), (4, 5, 2, 12), (2, 2, 4, 3)])
+def test_coarse_grained_eviction_against_exhaustive_shadow(oracle, fusion, T, G, C, R, P):
+    """Which tokens a T-step policy drops, and on which steps: the dictionary shadow (plain sort over all
+    candidates, policy on generation steps T, 2T, ...) against the oracle, after every step."""
+    w = TINY.replace(n_q_heads=2 * G, prompt_len=P, steps=4 * T + 3, C=C, R=R, fusion=fusion, seed=500 + 7 * G + T)
+    q, k, v = unit_inputs(w, 0, 0, 1, np.arange(P + w.steps))
+    u = oracle.Unit(G, w.head_dim, C, R, fusion, evict_interval=T)
+    sh = ShadowMorphKV(G, w.head_dim, C, R, fusion, evict_interval=T)
+    Rw = min(R, P)
+    u.prefill(k[:P], v[:P], q[:, P - Rw:P])
+    sh.prefill(k[:P], v[:P], q[:, P - Rw:P])
+    assert set(u.positions().tolist()) == sh.cached
+    policy_steps, multi = [], 0
+    for s in range(w.steps):
+        t = P + s
+        o = u.step(q[:, t], k[t], v[t])
+        o2 = sh.step(q[:, t], k[t], v[t])
+        assert np.abs(o - o2).max() < 1e-12
+        assert set(u.positions().tolist()) == sh.cached, f"step {s + 1}: retained sets differ"
+        assert sorted(u.last_evicted().tolist()) == sh.last_dropped, f"step {s + 1}: different tokens dropped"
+        if (s + 1) % T != 0:
+            assert len(u.last_evicted()) == 0 and len(u.last_scores()[0]) == 0      # no policy between multiples of T
+        if sh.last_F is not None:
+            policy_steps.append(s + 1)
+            multi += len(sh.last_dropped) > 1
+            pos, F = u.last_scores()
+            assert pos.tolist() == sh.last_ranked                      # full ranking of ALL candidates
+            assert np.allclose(F, [sh.last_F[p] for p in pos], rtol=1e-12, atol=1e-300)
+            assert best_subset_by_enumeration(sh.last_F, C) == set(sh.last_ranked[:C])
+            assert len(sh.cached) == C + R                             # back to C + R after the policy
+        assert len(sh.cached) <= C + R + T - 1
+    assert policy_steps and all(p % T == 0 for p in policy_steps)
+    assert multi > 0                                                   # several tokens dropped at once was exercised
+
+
 def test_t1_is_default(oracle):
     w = synth.WORKLOADS["c0"].replace(steps=30)
     a, ua, _ = _run(oracle, w)
