@@ -82,49 +82,71 @@ def measured_peak_gbs():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """SM clock and throttle reasons of one GPU, read through NVML (the library nvidia-smi itself reads).
 
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    `during(done)` samples in the calling thread until `done()` turns true: it is called right after the timed
+    steps have been enqueued, so every sample falls inside the timed region however short that is, and no
+    query can sit between two kernel launches (a polling child process did: its queries take milliseconds and
+    held up the launches of a 1 ms region).  Without the NVML binding, one `nvidia-smi` query is made instead.
+    """
 
-    def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+    REASONS = (("sw_power_cap", 0x4), ("hw_slowdown", 0x8), ("sw_thermal_slowdown", 0x20), ("hw_thermal_slowdown", 0x40))
 
-    def __enter__(self):
+    def __init__(self, device: torch.device, period_s: float = 0.005):
+        self.period_s, self.sm, self.mx, self.reasons, self.nv, self.h = period_s, [], [], set(), None, None
+        self.index = device.index or 0
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
-                                         stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
-            self.thread.start()
-        except OSError:
-            self.proc = None
-        return self
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.nv = pynvml
+            self.sample()           # first call of each query pays one-time set-up costs: not a timed-region sample
+            self.sm, self.mx, self.reasons = [], [], set()
+        except Exception:
+            self.nv = None
 
-    def __exit__(self, *exc):
-        if self.proc:
-            time.sleep(0.15)
-            self.proc.terminate()
-            self.thread.join(timeout=2)
+    def sample(self):
+        nv = self.nv
+        if nv is None:
+            return self._sample_smi()
+        try:
+            self.sm.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+            self.mx.append(float(nv.nvmlDeviceGetMaxClockInfo(self.h, nv.NVML_CLOCK_SM)))
+            get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            mask = int(get(self.h))
+            self.reasons |= {name for name, bit in self.REASONS if mask & bit}
+        except Exception:
+            pass
+
+    def _sample_smi(self):
+        fields = ("clocks.sm,clocks.max.sm,clocks_event_reasons.sw_power_cap,clocks_event_reasons.hw_slowdown,"
+                  "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.hw_thermal_slowdown")
+        try:
+            out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={fields}",
+                                  "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10).stdout
+            parts = [p.strip() for p in out.strip().split("\n")[0].split(",")]
+            self.sm.append(float(parts[0])); self.mx.append(float(parts[1]))
+            self.reasons |= {name for (name, _), val in zip(self.REASONS, parts[2:6]) if val.lower().startswith("active")}
+        except Exception:
+            pass
+
+    def during(self, done):
+        """Samples until done() is true; at least once."""
+        while True:
+            self.sample()
+            if done():
+                break
+            time.sleep(self.period_s)
 
     def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [p.strip() for p in ln.split(",")]
-            if len(parts) < 6:
-                continue
-            try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, parts[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        if not sm:
+        if not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": float(max(self.mx)), "reasons": sorted(self.reasons),
+                "samples": len(self.sm), "source": "nvml" if self.nv else "nvidia-smi"}
 
 
 def oracle_throughput(w: synth.Workload, n_units: int, steps: int, warm: int = 2):
@@ -258,20 +280,28 @@ def run_ours(args, w):
         torch.cuda.synchronize()
 
     # ---- arm 1: inputs resident in HBM ----
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    clocks = ClockSampler(dev)
+    # the warm-up is bracketed by events like the timed steps: the first timing-event pair of a process costs the
+    # GPU some tens of microseconds that belong to no step
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0.record(stream)
     mk.decode_steps(qs[:W], kn[:W], vn[:W], outs[:W])
+    w1.record(stream)
+    w1.query()
     mk.sync()
+    w0.elapsed_time(w1)
     n_steady = mk.view(0)["count"]
     T = max(1, args.evict_interval)
     if T > 1:       # the fill cycles through C+R .. C+R+T-1: the roofline bytes use its mean
         n_steady = min(n_steady, w.C + w.R) + (T - 1) / 2
     launches0 = mk.launch_count
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    with ClockSampler(local) as clocks:
-        e0.record(stream)
-        mk.decode_steps(qs[W:W + K], kn[W:W + K], vn[W:W + K], outs[W:W + K])
-        e1.record(stream)
-        torch.cuda.synchronize()
+    e0.record(stream)
+    mk.decode_steps(qs[W:W + K], kn[W:W + K], vn[W:W + K], outs[W:W + K])
+    e1.record(stream)
+    clocks.during(e1.query)          # the steps are enqueued and running: sample until the last one is done
+    torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     launches = mk.launch_count - launches0
     mk.sync()

@@ -71,6 +71,12 @@ typedef struct mkv_params {
     void *workspace;        /* device memory owned by the caller, 256-byte aligned, or NULL
                                to let the library allocate it with cudaMalloc              */
     size_t workspace_bytes;
+    unsigned long long wait_limit_cycles;
+                            /* how long a device-side wait (on a copy, on the tensor cores, on another
+                               warp) may spin before the kernel gives up, in GPU clock ticks; 0 = the
+                               default of about two seconds.  A wait that runs out makes the kernel
+                               return early and mkv_sync report MKV_DEVICE_TIMEOUT.  Only tests have a
+                               reason to lower it.                                                   */
 } mkv_params;
 
 /* What one layer of the cache looks like.  Slot order inside a unit is unspecified: the

@@ -39,7 +39,9 @@
  * Pinned by tests/test_oracle_pins.py (full-attention special case against an
  * independent causal attention, the paper's worked 0.3/0.05 example, cache
  * invariants, brute-force ranking on tiny inputs, R=1 and G=1 reductions,
- * stored == recompute, shift / permutation / scaling metamorphic checks).
+ * stored == recompute, shift / permutation / scaling metamorphic checks, and
+ * for evict_interval > 1 which tokens are dropped on which steps against a
+ * dictionary restatement that ranks all candidates with a plain sort).
  * The readings themselves (window membership, stored weights, prefill
  * procedure) have no printed value in the paper to pin them: parity unpinned
  * for those choices.
@@ -210,9 +212,14 @@ static int score_and_select(ora_unit *u, const long *forced, int n_forced)
 
 /*
  * Prefill with P prompt tokens: k, v [P][d], q_window [G][Rw][d] (queries of
- * the last Rw = min(R, P) prompt positions, oldest first).
+ * the last Rw = min(R, P) prompt positions, oldest first).  `forced` /
+ * `n_forced`: optional list of the prompt positions to evict instead of the
+ * oracle's own choice (the harness uses it to follow a legitimate near-tie
+ * decision of the device); it must name exactly as many candidates as the
+ * policy evicts.  The ranking of all candidates is kept for ora_last_scores.
  */
-int ora_prefill(ora_unit *u, const double *k, const double *v, const double *q_window, int P)
+int ora_prefill_forced(ora_unit *u, const double *k, const double *v, const double *q_window, int P,
+                       const long *forced, int n_forced)
 {
     if (!u || P < 1 || u->t != 0) return -1;
     const int G = u->G, d = u->d, R = u->R;
@@ -252,7 +259,22 @@ int ora_prefill(ora_unit *u, const double *k, const double *v, const double *q_w
         }
         qsort(c, (size_t)ncand, sizeof(cand_t), cand_cmp);
         u->kth = c[u->C - 1].F; u->k1th = c[u->C].F;
-        for (int j = u->C; j < ncand; ++j) keep[c[j].pos] = 0;
+        /* the prompt may hold more candidates than the cache has slots: grow the read-back arrays */
+        if (ncand > u->cap) {
+            u->cand_pos = (long *)realloc(u->cand_pos, (size_t)ncand * sizeof(long));
+            u->cand_F = (double *)realloc(u->cand_F, (size_t)ncand * sizeof(double));
+        }
+        u->n_cand = ncand;
+        for (int j = 0; j < ncand; ++j) { u->cand_pos[j] = c[j].pos; u->cand_F[j] = c[j].F; }
+        if (n_forced > 0) {
+            int bad = n_forced != ncand - u->C;
+            for (int f = 0; f < n_forced && !bad; ++f) {
+                if (forced[f] < 0 || forced[f] >= ncand || !keep[forced[f]]) bad = 1; else keep[forced[f]] = 0;
+            }
+            if (bad) { free(c); free(Afull); free(m); free(l); free(keep); return -3; }
+        } else {
+            for (int j = u->C; j < ncand; ++j) keep[c[j].pos] = 0;
+        }
         free(c);
     }
     /* build the cache and the stored profile rows of the window */
@@ -280,6 +302,11 @@ int ora_prefill(ora_unit *u, const double *k, const double *v, const double *q_w
     u->t = P;
     free(Afull); free(m); free(l); free(keep);
     return 0;
+}
+
+int ora_prefill(ora_unit *u, const double *k, const double *v, const double *q_window, int P)
+{
+    return ora_prefill_forced(u, k, v, q_window, P, NULL, 0);
 }
 
 /*

@@ -42,6 +42,7 @@ def _load():
         lib.ora_create.argtypes = [C.c_int] * 7
         lib.ora_destroy.argtypes = [C.c_void_p]
         lib.ora_prefill.argtypes = [C.c_void_p, dp, dp, dp, C.c_int]
+        lib.ora_prefill_forced.argtypes = [C.c_void_p, dp, dp, dp, C.c_int, lp, C.c_int]
         lib.ora_step.argtypes = [C.c_void_p, dp, dp, dp, dp, lp, C.c_int]
         lib.ora_count.argtypes = [C.c_void_p]
         lib.ora_next_pos.argtypes = [C.c_void_p]
@@ -86,13 +87,19 @@ class Unit:
         if h:
             self.lib.ora_destroy(h)
 
-    def prefill(self, k, v, q_window) -> None:
-        """k, v [P,d]; q_window [G, min(R,P), d] (last prompt positions, oldest first)."""
+    def prefill(self, k, v, q_window, forced=None) -> None:
+        """k, v [P,d]; q_window [G, min(R,P), d] (last prompt positions, oldest first).  `forced`: the prompt
+        positions to evict instead of the oracle's own choice (harness resync after a near tie)."""
         k, v, qw = _f64(k), _f64(v), _f64(q_window)
         P = k.shape[0]
         assert k.shape == (P, self.d) and v.shape == (P, self.d)
         assert qw.shape == (self.G, min(self.R, P), self.d), qw.shape
-        rc = self.lib.ora_prefill(self.h, _dp(k), _dp(v), _dp(qw), P)
+        self._scores_cap = max(self.cap, P)
+        if forced is None or len(forced) == 0:
+            rc = self.lib.ora_prefill(self.h, _dp(k), _dp(v), _dp(qw), P)
+        else:
+            farr = np.ascontiguousarray(np.asarray(forced, dtype=np.int64))
+            rc = self.lib.ora_prefill_forced(self.h, _dp(k), _dp(v), _dp(qw), P, _lp(farr), len(farr))
         if rc:
             raise RuntimeError(f"ora_prefill failed ({rc})")
 
@@ -133,8 +140,9 @@ class Unit:
 
     def last_scores(self):
         """Candidates of the last selection as (positions, F), sorted (F desc, pos asc)."""
-        p = np.empty(self.cap, dtype=np.int64)
-        f = np.empty(self.cap, dtype=np.float64)
+        cap = max(self.cap, getattr(self, "_scores_cap", 0))      # a prompt can hold more candidates than slots
+        p = np.empty(cap, dtype=np.int64)
+        f = np.empty(cap, dtype=np.float64)
         n = self.lib.ora_last_scores(self.h, _lp(p), _dp(f))
         return p[:n].copy(), f[:n].copy()
 
@@ -167,11 +175,9 @@ def fuse_select(S, C_: int, fusion):
     return F, keep.astype(bool)
 
 
-def boundary_is_near_tie(kth: float, k1th: float, rel: float = 1e-3, floor: float = 1e-30) -> bool:
+def boundary_is_near_tie(kth: float, k1th: float, rel: float = 1e-3) -> bool:
     """True when the C-th and (C+1)-th fused scores are too close for the retained set to be unique:
-    relative gap <= ``rel``, or both below ``floor`` (under fp32's normal range after normalisation)."""
+    relative gap <= ``rel``."""
     if np.isnan(kth) or np.isnan(k1th):
         return False
-    if abs(kth) < floor and abs(k1th) < floor:
-        return True
     return abs(kth - k1th) <= rel * max(abs(kth), abs(k1th))

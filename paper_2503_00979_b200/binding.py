@@ -36,7 +36,7 @@ class mkv_params(C.Structure):
         ("layers", C.c_int), ("batch", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int),
         ("head_dim", C.c_int), ("C", C.c_int), ("R", C.c_int), ("fusion", C.c_int), ("dtype", C.c_int),
         ("evict_interval", C.c_int), ("kernel", C.c_int), ("splits", C.c_int),
-        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("wait_limit_cycles", C.c_ulonglong),
     ]
 
 
@@ -199,7 +199,7 @@ class MorphKV:
     """A context whose workspace is a torch tensor.  Methods mirror the C calls and raise on error."""
 
     def __init__(self, layers, batch, n_q_heads, n_kv_heads, head_dim, C_, R, fusion="sum", dtype="bf16",
-                 evict_interval=1, kernel="auto", splits=0, device="cuda:0"):
+                 evict_interval=1, kernel="auto", splits=0, device="cuda:0", wait_limit_cycles=0):
         self.device = torch.device(device)
         p = mkv_default_params()
         p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = layers, batch, n_q_heads, n_kv_heads, head_dim
@@ -207,6 +207,7 @@ class MorphKV:
         p.fusion = FUSION[fusion] if isinstance(fusion, str) else int(fusion)
         p.dtype = DTYPE[dtype] if isinstance(dtype, str) else int(dtype)
         p.evict_interval, p.kernel, p.splits = evict_interval, KERNEL[kernel], splits
+        p.wait_limit_cycles = wait_limit_cycles
         self.torch_dtype = torch.float32 if p.dtype == 1 else torch.bfloat16
         self.shape = dict(L=layers, B=batch, Hq=n_q_heads, Hkv=n_kv_heads, d=head_dim, C=C_, R=R,
                           G=n_q_heads // max(1, n_kv_heads))

@@ -165,7 +165,9 @@ mkv_status launch_step(mkv_ctx *ctx, const void *q, const void *k, const void *v
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "decode launch failed: %s", cudaGetErrorString(e));
     ctx->launches += 1;
     const bool ev = step_scores(ctx->t, ctx->n, ctx->steps, ctx->s.R, ctx->s.C, ctx->s.T);
-    if (ctx->s.T > 1) {
+    // coarse-grained eviction: the compaction follows the steps that ran the policy (the kernel itself checks the
+    // device state and does nothing if no compaction is pending)
+    if (ctx->s.T > 1 && ev) {
         const cudaError_t e2 = launch_compact(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
         if (e2 != cudaSuccess) return fail(ctx, MKV_CUDA, "compaction launch failed: %s", cudaGetErrorString(e2));
         ctx->launches += 1;
@@ -237,7 +239,7 @@ mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p)
     if (kind == kKindTc) {
         const DecodeArgs a = make_args(c, nullptr, nullptr, nullptr, nullptr);
         char msg[200] = "";
-        const cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, msg, sizeof(msg));
+        const cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, p->wait_limit_cycles, msg, sizeof(msg));
         if (e != cudaSuccess) {
             cudaGetLastError();
             if (c->owns_workspace) cudaFree(c->base);
@@ -401,6 +403,8 @@ mkv_status mkv_sync(mkv_ctx *ctx, void *stream)
     DevState st;
     e = cudaMemcpy(&st, ctx->base + ctx->L.state, sizeof(st), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e));
+    if (st.err == kErrCacheOverflow)
+        return fail(ctx, MKV_BAD_STATE, "a decode step found no free slot: coarse-grained eviction ran out of step%s");
     if (st.err != kErrNone) {
         char code[32];
         snprintf(code, sizeof(code), " (wait code %d)", st.err);

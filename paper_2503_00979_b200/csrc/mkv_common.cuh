@@ -25,7 +25,9 @@ struct DevState {
     int compact;          // coarse-grained eviction: the step that just ran scored, the cache awaits its compaction
 };
 
-enum DevError { kErrNone = 0, kErrBarrierTimeout = 1 };
+// 1..99: the code of the bounded wait that gave up; kErrCacheOverflow: a step found no free slot (only possible
+// when coarse-grained eviction was driven out of step, e.g. by replaying part of a period from a CUDA graph)
+enum DevError { kErrNone = 0, kErrBarrierTimeout = 1, kErrCacheOverflow = 100 };
 
 // Everything a decode kernel needs.  Passed by value as a __grid_constant__.
 struct DecodeArgs {
@@ -268,10 +270,14 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         if (a.T > 1) {          // coarse-grained eviction: append now, the compaction launch evicts
             e_slot = n;
             e_pos = -1;
-            if (tid == 0) F[n] = -1.f;
+            if (tid == 0 && n < a.cap) F[n] = -1.f;
         }
     }
 
+    if (e_slot >= a.cap) {      // no free slot: refuse to write beyond the unit's rows
+        if (tid == 0) { atomicCAS(&a.st->err, 0, (int)kErrCacheOverflow); a.ticket[u] = 0; }
+        return;
+    }
     // Eq. 7 update: the freed (or next free) slot takes the new token; the ring row of the
     // token that left the window takes the new query and its soft-max normaliser
     T *Kd = static_cast<T *>(a.K) + ((size_t)u * a.cap + e_slot) * D;

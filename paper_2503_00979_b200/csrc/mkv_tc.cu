@@ -50,7 +50,7 @@ constexpr int kMaxComputeWarps = 4 * kComputeGroups;
 __host__ __device__ constexpr int tc_threads(int ng) { return 32 * (3 + 4 * ng + 4); }
 constexpr int kFirstComputeWarp = 3;
 constexpr int kGroupThreads = 128;
-constexpr long long kWaitCycles = 4000000000ll;   // about two seconds
+constexpr long long kWaitCycles = 4000000000ll;   // default limit of a device-side wait: about two seconds
 constexpr int kFinFloats = 4 * kMaxGroup + 128 + 256 + 64 + 32 + 8;   // epilogue scratch of finalize_fast
 // epilogue group: finalize scratch, flag, merged (m, l), per-warp scale factors
 constexpr int kEpiFloats = kFinFloats + 8 + 2 * kMaxGroup + kMaxComputeWarps * kMaxGroup;
@@ -63,6 +63,7 @@ struct TcGeom {
     int tmem_cols;      // allocated TMEM columns (power of two)
     int grid;
     int smem_bytes;
+    long long wait_cycles;   // limit of every device-side wait, in clock64 ticks
 };
 
 struct SmemLayout {
@@ -115,27 +116,44 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Which wait gave up (recorded in the CTA's abort flag and reported to the host)
 enum WaitCode { kWaitQEmpty = 1, kWaitKEmpty, kWaitVEmpty, kWaitQFull, kWaitKFull, kWaitTEmpty, kWaitTFull, kWaitVFull,
                 kWaitPFree, kWaitUDone, kWaitDrain };
-// Bounded wait.  Gives up after kWaitCycles or as soon as another thread has raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort, int code)
+// Bounded wait.  Gives up after `limit` clock ticks or as soon as another thread has raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort, int code, long long limit)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0) {
+        if ((it & 15u) == 0) {
             if (*abort) return false;
-            if (clock64() - t0 > kWaitCycles) { *abort = code; return false; }
+            if (clock64() - t0 > limit) { *abort = code; return false; }
         }
     }
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
+// L2 eviction policies for the copies: the K/V tiles are read once per step and the whole cache is larger than
+// L2, so they are marked evict-first; the recent-query ring, the per-key scratch and the split partials are small
+// and re-read within a step or on the next one, so the ring is fetched evict-last and the rest keeps L2 to itself.
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar,
+                                            uint64_t policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy) : "memory");
 }
 
 // brings a tensor map into the descriptor cache ahead of its first copy
@@ -454,7 +472,11 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     int *pos = a.pos + (size_t)u * a.cap;
     float *F = a.F + (size_t)u * a.cap;
     int e_slot = n, e_pos = -1;
-    {
+    if (!evict) {
+        // no selection on this step (cache still filling, or between two runs of a coarse-grained policy):
+        // the new token takes the next free slot
+        if (tid == 0 && n < a.cap) F[n] = -1.f;
+    } else {
         const float *sn = a.s_new + (size_t)u * G * a.cap;
         const long long thr = t - a.R;
         float cn[G];
@@ -505,15 +527,19 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
             if (red_key[w] < best) { best = red_key[w]; bslot = red_slot[w]; }
         e_slot = bslot;
         e_pos = (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull));   // the rank key carries the position
-        if (!evict || a.T > 1) {
-            // nothing to evict on this step, or coarse-grained eviction (append now, the compaction launch
-            // evicts): the new token takes the next free slot and is not a candidate
+        if (a.T > 1) {
+            // coarse-grained eviction (append now, the compaction launch evicts): the new token takes the
+            // next free slot and is not a candidate
             e_slot = n;
             e_pos = -1;
-            if (tid == 0) F[n] = -1.f;
+            if (tid == 0 && n < a.cap) F[n] = -1.f;
         }
     }
 
+    if (e_slot >= a.cap) {      // no free slot: refuse to write beyond the unit's rows
+        if (tid == 0) { atomicCAS(&a.st->err, 0, (int)kErrCacheOverflow); a.ticket[u] = 0; }
+        return;
+    }
     // ---- phase D: Eq. 7 update from the registers loaded in phase A
     __nv_bfloat16 *Kd = static_cast<__nv_bfloat16 *>(a.K) + ((size_t)u * a.cap + e_slot) * kD;
     __nv_bfloat16 *Vd = static_cast<__nv_bfloat16 *>(a.V) + ((size_t)u * a.cap + e_slot) * kD;
@@ -548,6 +574,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const SmemLayout L = tc_smem_layout(geo, G);
     const int SK = geo.sk, SV = geo.sv, NB = geo.nb, RGP = geo.rgpad;
+    const long long WL = geo.wait_cycles;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t q_addr = sbase + L.q, kst_addr = sbase + L.kst, vst_addr = sbase + L.vst;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
@@ -614,23 +641,25 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         if (lane == 0) {
             Walk w(a.U, n);
             Item x;
-            int issued = 0;
+            int issued = 0, rings = 0;
             bool ok = true;
             RingPos rk(0, SK);
+            const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
             while (ok && w.next(x)) {
-                ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag, kWaitQEmpty);
+                ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag, kWaitQEmpty, WL);
                 if (!ok) break;
                 mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
-                tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull);
-                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull);
+                tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull, pol_keep);
+                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull, pol_keep);
+                ++rings;
                 for (int j = 0; j < x.nk && ok; ++j, rk.step(1, SK)) {
                     const int T = w.T0 + j, s = rk.idx;
-                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(rk.lap ^ 1), abort_flag, kWaitKEmpty);
+                    ok = mbar_wait(bar_kempty + 8 * s, (uint32_t)(rk.lap ^ 1), abort_flag, kWaitKEmpty, WL);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_kfull + 8 * s, kStageBytes);
-                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, x.unit, bar_kfull + 8 * s);
-                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, x.unit, bar_kfull + 8 * s);
+                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, x.unit, bar_kfull + 8 * s, pol_stream);
+                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, x.unit, bar_kfull + 8 * s, pol_stream);
                     issued = T + 1;
                 }
                 w.advance(x);
@@ -638,7 +667,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             if (!ok) {   // give up: let the copies already in flight land before the CTA exits
                 int dummy = 0;
                 for (int T = max(0, issued - SK); T < issued; ++T)
-                    mbar_wait(bar_kfull + 8 * (T % SK), (uint32_t)((T / SK) & 1), &dummy, kWaitDrain);
+                    mbar_wait(bar_kfull + 8 * (T % SK), (uint32_t)((T / SK) & 1), &dummy, kWaitDrain, kWaitCycles);
+                if (rings > 0) mbar_wait(bar_qfull, (uint32_t)((rings - 1) & 1), &dummy, kWaitDrain, kWaitCycles);
             }
         }
     } else if (warp == 2) {
@@ -649,15 +679,16 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             int issued = 0;
             bool ok = true;
             RingPos rv(0, SV);
+            const uint64_t pol_stream = l2_policy_evict_first();
             while (ok && w.next(x)) {
                 for (int j = 0; j < x.nk && ok; ++j, rv.step(1, SV)) {
                     const int T = w.T0 + j, s = rv.idx;
-                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty);
+                    ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty, WL);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_vfull + 8 * s, kStageBytes);
-                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, x.unit, bar_vfull + 8 * s);
-                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, x.unit, bar_vfull + 8 * s);
+                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, x.unit, bar_vfull + 8 * s, pol_stream);
+                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, x.unit, bar_vfull + 8 * s, pol_stream);
                     issued = T + 1;
                 }
                 w.advance(x);
@@ -665,7 +696,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             if (!ok) {
                 int dummy = 0;
                 for (int T = max(0, issued - SV); T < issued; ++T)
-                    mbar_wait(bar_vfull + 8 * (T % SV), (uint32_t)((T / SV) & 1), &dummy, kWaitDrain);
+                    mbar_wait(bar_vfull + 8 * (T % SV), (uint32_t)((T / SV) & 1), &dummy, kWaitDrain, kWaitCycles);
             }
         }
     } else if (warp == 1) {
@@ -674,6 +705,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         Item x;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RGP >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
         bool ok = true;
+        int n_mma = 0;                                  // tiles whose MMAs have been issued and committed
         RingPos rk(0, SK), rb(0, NB);
         while (ok && w.next(x)) {
             {
@@ -684,7 +716,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i)
                     if (lane + 32 * i < G * 16) qv[i] = qsrc[lane + 32 * i];
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.nitems & 1), abort_flag, kWaitQFull));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.nitems & 1), abort_flag, kWaitQFull, WL));
                 if (!ok) break;
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i) {
@@ -700,8 +732,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             }
             for (int j = 0; j < x.nk; ++j, rk.step(1, SK), rb.step(1, NB)) {
                 const int s = rk.idx, b = rb.idx;
-                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)rk.lap, abort_flag, kWaitKFull);
-                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(rb.lap ^ 1), abort_flag, kWaitTEmpty);
+                bool k = mbar_wait(bar_kfull + 8 * s, (uint32_t)rk.lap, abort_flag, kWaitKFull, WL);
+                k = k && mbar_wait(bar_tempty + 8 * b, (uint32_t)(rb.lap ^ 1), abort_flag, kWaitTEmpty, WL);
                 ok = __all_sync(0xffffffffu, k);
                 if (!ok) break;
                 tc_fence_after();
@@ -716,9 +748,24 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     umma_commit(bar_kempty + 8 * s);      // K tile consumed
                     umma_commit(bar_tfull + 8 * b);       // accumulators ready
                 }
+                ++n_mma;
                 __syncwarp();
             }
             w.advance(x);
+        }
+        // A tcgen05.commit arrives on its mbarrier asynchronously, when the MMAs before it have completed.  The
+        // arrivals on the K-empty barriers of the last tiles have no waiter left (the producer has issued its last
+        // load), and after a wait has given up the accumulator-full arrivals may have none either.  This warp
+        // observes every one of them before the CTA frees its TMEM and exits, so that no MMA is still running and
+        // no arrival can land in shared memory that by then belongs to a CTA of the next launch.
+        {
+            int dummy = 0;
+            for (int T = max(0, n_mma - SK); T < n_mma; ++T)
+                mbar_wait(bar_kempty + 8 * (T % SK), (uint32_t)((T / SK) & 1), &dummy, kWaitDrain, kWaitCycles);
+            if (!ok)
+                for (int T = max(0, n_mma - NB); T < n_mma; ++T)
+                    mbar_wait(bar_tfull + 8 * (T % NB), (uint32_t)((T / NB) & 1), &dummy, kWaitDrain, kWaitCycles);
+            __syncwarp();
         }
     } else if (warp < kFirstComputeWarp + 4 * NG) {
         // ------------------------------------------------ compute warps
@@ -775,7 +822,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 const int j = Tn - w.T0;
                 const int buf = rb.idx;
                 // ---- scores of this warp's 32 keys (Eq. 4-6) and the new row's logits
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)rb.lap, abort_flag, kWaitTFull));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)rb.lap, abort_flag, kWaitTFull, WL));
                 if (!ok) break;
                 tc_fence_after();
                 const int key = (x.tile0 + j) * kTile + gtid;
@@ -785,18 +832,6 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 // written asynchronously, so nothing may touch them between the two.
                 uint32_t sv[G];
                 tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
-                // Scored on every step, also on steps that evict nothing (cache still filling, or between two
-                // runs of a coarse-grained policy): every launch then has the shape of the steady-state one.
-                float F = 0.f;
-                for (int c = 0; c < RGP; c += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + (uint32_t)c, v);
-                    score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
-                if (valid) a.F[(size_t)u * a.cap + key] = F;
 
                 // ---- online soft-max of the new row over this warp's keys (Eq. 1)
                 bool changed = false;
@@ -804,7 +839,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 for (int g = 0; g < G; ++g) {
                     const float s2 = valid ? __uint_as_float(sv[g]) * a.scale2 : -INFINITY;
                     st_w[g * 32 + lane] = s2;
-                    if (valid) s_new[(size_t)g * a.cap + key] = s2;
+                    if (valid && evict) s_new[(size_t)g * a.cap + key] = s2;
                     const float mn = fmaxf(mrun[g], warp_max(s2));
                     // factor that brings what was accumulated under the old reference to the new one
                     const float f = mn == mrun[g] ? 1.f : ex2f(mrun[g] - mn);
@@ -824,15 +859,16 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     }
                 }
 
-                // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys
+                // ---- O^T[d][g] += V^T[d][keys] . P^T[keys][g] over this warp's 32 keys.  This runs before the scoring
+                // of the ring rows so that the V stage goes back to its producer as early as possible.
                 const int s = rv.idx;
                 // A V stage serves the two compute groups in turn whenever the ring has an odd number of stages, and
                 // a parity wait cannot tell "this load has landed" from "the load before the previous one has
                 // landed".  The accumulator buffers keep the groups close enough for that never to matter; waiting
                 // for the previous load of the stage to be consumed first (the wait the producer does before it
                 // refills the stage) makes the full barrier's parity unambiguous without relying on that.
-                bool vok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty);
-                vok = vok && mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag, kWaitVFull);
+                bool vok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty, WL);
+                vok = vok && mbar_wait(bar_vfull + 8 * s, (uint32_t)rv.lap, abort_flag, kWaitVFull, WL);
                 ok = __all_sync(0xffffffffu, vok);
                 if (!ok) break;
                 const uint32_t vbase = vst_addr + s * kStageBytes;
@@ -879,6 +915,23 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 fence_proxy_async();
                 __syncwarp();                               // every lane has read its rows of the V tile
                 if (lane == 0) mbar_arrive(bar_vempty + 8 * s);
+                __syncwarp();                               // converged again in front of the .aligned TMEM loads
+
+                // ---- fused scores of this warp's 32 keys over the ring rows (Eq. 4-6): only on steps that run the
+                // policy.  While the cache is still filling, and between two runs of a coarse-grained policy, nothing
+                // is evicted and the accumulator buffer goes back as soon as the new row's logits have been read.
+                if (evict) {
+                    float F = 0.f;
+                    for (int c = 0; c < RGP; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + (uint32_t)c, v);
+                        score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
+                    }
+                    if (valid) a.F[(size_t)u * a.cap + key] = F;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
                 ++seg_tiles;
             }
 
@@ -886,7 +939,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             // ---- the item is done: leave this warp's partial for the epilogue group
             if (ok) {
                 // the previous partial must have been read before its buffer is overwritten
-                if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag, kWaitPFree));
+                if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag, kWaitPFree, WL));
                 if (ok) {
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
@@ -904,9 +957,12 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                             if (gc + 1 < G) { wbuf[(gc + 1) * kD + db * 16 + gid] = acc[nt][db][1]; wbuf[(gc + 1) * kD + db * 16 + gid + 8] = acc[nt][db][3]; }
                         }
                     }
-                    // fused scores / new-row logits of this warp's keys are read by the epilogue group of
-                    // this CTA, or of another CTA when the unit is shared
-                    if (w.unit_is_local(u)) __threadfence_block(); else __threadfence();
+                    // Fused scores / new-row logits of this warp's keys are read by the epilogue group of this CTA,
+                    // or of another CTA when the unit is shared.  The arrive releases this warp's writes at CTA
+                    // scope; for a shared unit the epilogue thread that takes the unit's ticket fences at device
+                    // scope after it has observed the arrivals, which carries these writes along (release
+                    // sequences are cumulative), so no device-scope fence is paid here.
+                    __threadfence_block();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_udone);
                     ++npub;
@@ -933,7 +989,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         while (ok && w.next(x)) {
             {
                 const int u = x.unit;
-                if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag, kWaitUDone))) { ok = false; break; }
+                if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag, kWaitUDone, WL))) { ok = false; break; }
                 // merge the compute warps' partials: common reference = max of theirs
                 if (etid < G) {
                     float m = -INFINITY;
@@ -965,14 +1021,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     finalize_fast<G, true>(a, u, t, n, 1, evict, fin_sm, etid, kEpiBar, o, cml);
                 } else {
                     // the unit is shared: publish this CTA's partial; the last CTA to do so finishes the unit.
-                    // Writers fence their own writes; after the barrier the ticket thread fences again
-                    // (cumulative over what the barrier made it observe) and then takes the ticket.
+                    // The group barrier orders every thread's writes (and, through the mbarrier above, the compute
+                    // warps' writes) before the ticket thread's device-scope fence, which releases them all; the
+                    // fence after the ticket is the acquire side, and the data is then read past L1 (ld.global.cg).
                     float *pml = a.part_ml + ((size_t)u * a.splits + my_index) * G * 2;
                     float *po = a.part_o + ((size_t)u * a.splits + my_index) * G * kD;
 #pragma unroll
                     for (int g = 0; g < G; ++g) po[g * kD + etid] = o[g];
                     if (etid < 2 * G) pml[etid] = cml[etid];
-                    __threadfence();
                     group_sync(kEpiBar, kGroupThreads);
                     if (etid == 0) {
                         __threadfence();
@@ -982,7 +1038,6 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     }
                     group_sync(kEpiBar, kGroupThreads);
                     if (*flag) {
-                        __threadfence();
                         if (ncta <= 8 && ncta * G * 2 <= 256)
                             finalize_fast<G, false>(a, u, t, n, ncta, evict, fin_sm, etid, kEpiBar, o, nullptr);
                         else
@@ -1128,7 +1183,8 @@ int tc_partials_per_unit(int U, int cap, int grid)
     return worst;
 }
 
-cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, char *err, size_t err_len)
+cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned long long wait_limit_cycles, char *err,
+                           size_t err_len)
 {
     *out = nullptr;
     TcPlan *p = new (std::nothrow) TcPlan;
@@ -1147,6 +1203,7 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, char *er
     g.tmem_cols = 32;
     while (g.tmem_cols < g.nb * g.rgpad) g.tmem_cols *= 2;
     g.grid = grid;
+    g.wait_cycles = wait_limit_cycles > 0 ? (long long)wait_limit_cycles : kWaitCycles;
     // as many 32 KB stages as fit, split between the K ring (short-lived tiles) and the V ring
     int total_stages = 0;
     for (int st = 9; st >= 2; --st) {
