@@ -3,13 +3,20 @@
 Both sides receive the same materialised tensors.  Per decode step and per checked unit the
 harness compares the attention output (max abs error) and the evicted position.  Where the
 device evicts a different token than the oracle ranks last, the choice is accepted only if
-the oracle's own fused scores of the two tokens are a near tie (relative gap <= 1e-3, or
-both below 1e-30); the oracle is then made to follow the device so later steps stay
-comparable.  Anything else is a failure.
+the oracle's own fused scores of the two tokens are a near tie (relative gap <= 1e-3); the
+oracle is then made to follow the device so later steps stay comparable.  Anything else is a
+failure.  The same rule covers the prompt phase: a retained set that differs from the
+oracle's must differ only in tokens whose fused scores tie with the boundary of the top C,
+and the oracle then starts from the device's set.
+
+The oracle units are independent, so their steps run on a thread pool (the C calls release
+the interpreter lock); only the sampled units' inputs are converted to float64.
 """
 from __future__ import annotations
 
 import dataclasses
+import os
+from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
 import torch
@@ -19,26 +26,30 @@ from paper_2503_00979_b200 import binding, synth
 
 TOL_OUT = {"bf16": 2e-2, "f32": 1e-4}     # max abs error of attention outputs, per step
 TIE_REL = 1e-3
-TIE_FLOOR = 1e-30
 
 
 @dataclasses.dataclass
 class ParityReport:
     steps: int = 0
     unit_steps: int = 0
+    units: int = 0
     max_out_err: float = 0.0
     evictions: int = 0
-    near_tie_resyncs: int = 0
+    near_tie_resyncs: int = 0           # decode steps on which the device's choice differed within the tie rule
+    prefill_resyncs: int = 0            # units whose prompt-phase set differed within the tie rule
+    min_rel_gap: float = float("inf")   # smallest relative gap between the oracle's C-th and (C+1)-th score
     max_F_rel_err: float = 0.0
     F_compared: int = 0
-    prefill_dropped: int = 0
     kernel: str = ""
 
 
 def near_tie(a: float, b: float) -> bool:
-    if abs(a) < TIE_FLOOR and abs(b) < TIE_FLOOR:
-        return True
     return abs(a - b) <= TIE_REL * max(abs(a), abs(b))
+
+
+def rel_gap(a: float, b: float) -> float:
+    m = max(abs(a), abs(b))
+    return abs(a - b) / m if m > 0 else 0.0
 
 
 def pick_units(w: synth.Workload, n: int, seed: int = 0):
@@ -51,57 +62,120 @@ def pick_units(w: synth.Workload, n: int, seed: int = 0):
     return [all_units[i] for i in sorted(idx)][:max(n, 2)]
 
 
+def _workers() -> int:
+    return max(1, min(32, len(os.sched_getaffinity(0))))
+
+
+def _f64(t: torch.Tensor) -> np.ndarray:
+    return t.double().cpu().numpy()
+
+
+class _DeviceStream:
+    """synth.Stream whose draws are made on one device and delivered on another."""
+
+    def __init__(self, w, draw_on, deliver_on):
+        self.st, self.to = synth.Stream(w, draw_on), torch.device(deliver_on)
+
+    def kv(self, *a, **k):
+        x, y = self.st.kv(*a, **k)
+        return x.to(self.to), y.to(self.to)
+
+    def q(self, *a, **k):
+        return self.st.q(*a, **k).to(self.to)
+
+
+def oracle_unit_following(make_unit, k, v, qw, device_positions, where: str):
+    """A prefilled oracle unit (from `make_unit()`) whose retained set equals the device's.  If the oracle's own
+    choice differs, every token that changed sides must tie with the boundary of its top C, and the oracle is
+    prefilled again with the device's evictions forced.  Returns (unit, resynced)."""
+    u = make_unit()
+    u.prefill(k, v, qw)
+    dev = set(int(p) for p in device_positions)
+    own = set(u.positions().tolist())
+    if dev == own:
+        return u, False
+    cp, cF = u.last_scores()
+    assert len(cp) > u.C, f"{where}: prompt-phase sets differ although nothing had to be evicted"
+    Fof = {int(p): float(f) for p, f in zip(cp, cF)}
+    kth, k1 = float(cF[u.C - 1]), float(cF[u.C])
+    for p in dev ^ own:
+        assert p in Fof, f"{where}: prompt position {p} is not a candidate"
+        assert near_tie(Fof[p], kth) or near_tie(Fof[p], k1), \
+            f"{where}: prompt token {p} (F={Fof[p]:.6e}) changed sides without a near tie (boundary {kth:.6e} / {k1:.6e})"
+    u2 = make_unit()
+    u2.prefill(k, v, qw, forced=sorted(set(int(p) for p in cp) - dev))
+    assert set(u2.positions().tolist()) == dev
+    return u2, True
+
+
 def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chunk: int = 32, kernel: str = "auto",
                splits: int = 0, check_F_every: int = 16, device: str = "cuda:0", use_steps_call: bool = False,
-               host_call_every: int = 0, host_pinned: bool = True) -> ParityReport:
+               host_call_every: int = 0, host_pinned: bool = True, synth_device=None, **ctx_kwargs) -> ParityReport:
+    """Prefill + `steps` decode steps of workload `w` on the device, followed by the oracle on `units`.
+
+    The steps of a chunk are enqueued without a synchronisation in between (the evicted positions of the
+    checked units are gathered on the stream and read back once per chunk).
+    use_steps_call   one mkv_decode_steps call per chunk (no per-step evicted positions: outputs are compared on
+                     every step, retained sets at the end of each chunk unless the oracle saw a near tie in it).
+    synth_device     where the inputs are drawn ("cpu" keeps the drawing's many small kernels off the GPU).
+    """
     dev = torch.device(device)
-    st = synth.Stream(w, dev)
+    st = _DeviceStream(w, synth_device or dev, dev)
     tdt = synth.torch_dtype(w.dtype)
     G, d, P, R, C_ = w.group, w.head_dim, w.prompt_len, w.R, w.C
     units = units or pick_units(w, n_units)
     rep = ParityReport()
     mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, d, C_, R, w.fusion, w.dtype, kernel=kernel,
-                         splits=splits, device=device)
+                         splits=splits, device=device, **ctx_kwargs)
     rep.kernel = mk.kernel_name
     tol = TOL_OUT[w.dtype]
     Rw = min(R, P)
+    pool = ThreadPoolExecutor(max_workers=_workers())
 
     # ---- prefill: inputs are drawn layer by layer so that full-size workloads fit in memory ----
     Hkv, Hq = w.n_kv_heads, w.n_q_heads
     k_all = torch.empty((w.layers, w.batch, Hkv, P, d), dtype=tdt, device=dev)
     v_all = torch.empty_like(k_all)
     qw_all = torch.empty((w.layers, w.batch, Hq, Rw, d), dtype=tdt, device=dev)
+    by_layer = {}
+    for (l, b, h) in units:
+        by_layer.setdefault(l, []).append((b, h))
     prompt = {}
     for l in range(w.layers):
         k32, v32 = st.kv(np.arange(P), [l])
         qw32 = st.q(np.arange(P - Rw, P), [l])
         k_all[l], v_all[l], qw_all[l] = k32[0].to(tdt), v32[0].to(tdt), qw32[0].to(tdt)
-        for (ul, b, h) in units:
-            if ul == l:
-                prompt[(ul, b, h)] = (k32[0, b, h].double().cpu().numpy(), v32[0, b, h].double().cpu().numpy(),
-                                      qw32[0, b, h * G:(h + 1) * G].double().cpu().numpy(), k32[0, b, h].clone())
+        for (b, h) in by_layer.get(l, []):
+            prompt[(l, b, h)] = (_f64(k32[0, b, h]), _f64(v32[0, b, h]), _f64(qw32[0, b, h * G:(h + 1) * G]))
         del k32, v32, qw32
     mk.prefill(k_all, v_all, qw_all)
     mk.sync()
-    del k_all, v_all, qw_all
+    views = {l: mk.view(l) for l in by_layer}
+    count0 = views[units[0][0]]["count"]
+    dev_pos = {(l, b, h): views[l]["pos"][b, h, :count0].cpu().numpy() for (l, b, h) in units}
+
+    def prefill_unit(key):
+        kp, vp, qp = prompt[key]
+        u, resync = oracle_unit_following(lambda: ora.Unit(G, d, C_, R, w.fusion), kp, vp, qp, dev_pos[key], f"unit {key}")
+        assert count0 == u.count, (count0, u.count)
+        return key, u, resync
+
     orac = {}
+    for key, u, resync in pool.map(prefill_unit, units):
+        orac[key] = u
+        rep.prefill_resyncs += int(resync)
+    # K rows must be the prompt rows of those positions, bit for bit
     for (l, b, h) in units:
-        kp, vp, qp, k_dev = prompt[(l, b, h)]
-        u = ora.Unit(G, d, C_, R, w.fusion)
-        u.prefill(kp, vp, qp)
-        view = mk.view(l)
-        gp = view["pos"][b, h, :view["count"]].cpu().numpy()
-        assert view["count"] == u.count, (view["count"], u.count)
-        if set(gp.tolist()) != set(u.positions().tolist()):
-            kth, k1 = u.last_boundary()
-            assert near_tie(kth, k1), f"prefill retained set differs for unit {(l, b, h)} without a near tie"
-            rep.prefill_dropped += 1
-            continue
-        # K/V rows must be the prompt rows of those positions, bit for bit
-        kk = view["K"][b, h, :view["count"]].float().cpu()
-        assert torch.equal(kk, k_dev[torch.from_numpy(gp).long().to(dev)].cpu())
-        orac[(l, b, h)] = u
-    del prompt
+        gp = torch.from_numpy(dev_pos[(l, b, h)]).long().to(dev)
+        assert torch.equal(views[l]["K"][b, h, :count0], k_all[l, b, h][gp]), f"unit {(l, b, h)}: K rows differ from the prompt's"
+        assert torch.equal(views[l]["V"][b, h, :count0], v_all[l, b, h][gp]), f"unit {(l, b, h)}: V rows differ from the prompt's"
+    del k_all, v_all, qw_all, prompt
+    rep.units = len(orac)
+    layers_checked = sorted(by_layer)
+    li = torch.tensor([l for (l, b, h) in units], device=dev)
+    bi = torch.tensor([b for (l, b, h) in units], device=dev)
+    hi = torch.tensor([h for (l, b, h) in units], device=dev)
+    lidx = torch.tensor([layers_checked.index(l) for (l, b, h) in units], device=dev)
 
     # ---- decode in chunks ----
     done = 0
@@ -114,7 +188,7 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
         ks = k32.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
         vs = v32.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
         outs = torch.empty_like(qs)
-        evh = torch.empty((ns, w.layers, w.batch, w.n_kv_heads), dtype=torch.int32, device=dev)
+        evh = torch.empty((ns, len(units)), dtype=torch.int32, device=dev)
         Fsnap = {}
         if use_steps_call:
             mk.decode_steps(qs, ks, vs, outs)
@@ -131,38 +205,50 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
                     outs[i].copy_(oh)
                 else:
                     mk.decode_step(qs[i], ks[i], vs[i], outs[i])
-                for l in sorted({u[0] for u in orac}):
-                    evh[i, l].copy_(mk.view(l)["evicted_pos"])
+                # evicted positions of the checked units, gathered on the stream
+                ev_all = torch.stack([views[l]["evicted_pos"] for l in layers_checked])      # [layers checked, B, Hkv]
+                evh[i] = ev_all[lidx, bi, hi]
                 if check_F_every and (done + i) % check_F_every == check_F_every - 1:
-                    Fsnap[i] = {l: (mk.view(l)["F"].clone(), mk.view(l)["pos"].clone()) for l in {u[0] for u in orac}}
+                    Fsnap[i] = {l: (views[l]["F"].clone(), views[l]["pos"].clone()) for l in layers_checked}
         mk.sync()
-        outs_c = outs.float().cpu().numpy()
-        q_c, k_c, v_c = q32.double().cpu().numpy(), k32.double().cpu().numpy(), v32.double().cpu().numpy()
+        # only the checked units cross to the host
+        q_u = _f64(q32.view(w.layers, w.batch, Hkv, G, ns, d)[li, bi, hi])        # [units, G, ns, d]
+        k_u, v_u = _f64(k32[li, bi, hi]), _f64(v32[li, bi, hi])                     # [units, ns, d]
+        o_u = outs.view(ns, w.layers, w.batch, Hkv, G, d)[:, li, bi, hi].float().cpu().numpy()   # [ns, units, G, d]
         ev_c = evh.cpu().numpy() if evh is not None else None
-        for (l, b, h), u in orac.items():
+        del q32, k32, v32, qs, ks, vs, outs
+        t0 = P + done
+
+        def follow(ui):
+            key = units[ui]
+            u = orac[key]
+            r = dict(err=0.0, evictions=0, resyncs=0, Fmax=0.0, Fcmp=0, gap=float("inf"))
             for i in range(ns):
-                t = P + done + i
-                e_g = int(ev_c[i, l, b, h]) if ev_c is not None else None
+                t = t0 + i
+                e_g = int(ev_c[i, ui]) if ev_c is not None else None
                 forced = [e_g] if (e_g is not None and e_g >= 0) else None
-                o = u.step(q_c[l, b, h * G:(h + 1) * G, i], k_c[l, b, h, i], v_c[l, b, h, i], forced=forced)
-                err = float(np.abs(o - outs_c[i, l, b, h * G:(h + 1) * G]).max())
-                rep.max_out_err = max(rep.max_out_err, err)
-                assert err <= tol, f"unit {(l, b, h)} step {t}: attention output error {err:.3e} > {tol}"
+                o = u.step(np.ascontiguousarray(q_u[ui, :, i]), k_u[ui, i], v_u[ui, i], forced=forced)
+                err = float(np.abs(o - o_u[i, ui]).max())
+                r["err"] = max(r["err"], err)
+                assert err <= tol, f"unit {key} step {t}: attention output error {err:.3e} > {tol}"
                 cp, cF = u.last_scores()
+                if len(cp) > C_:
+                    r["gap"] = min(r["gap"], rel_gap(float(cF[C_ - 1]), float(cF[C_])))
                 if ev_c is not None:
                     if len(cp) > C_:
-                        rep.evictions += 1
-                        assert e_g >= 0, f"unit {(l, b, h)} step {t}: device did not evict"
+                        r["evictions"] += 1
+                        assert e_g >= 0, f"unit {key} step {t}: device did not evict"
                         own = int(cp[C_])
                         if e_g != own:
                             Fg = float(cF[np.nonzero(cp == e_g)[0][0]])
                             assert near_tie(Fg, float(cF[C_])), \
-                                (f"unit {(l, b, h)} step {t}: device evicted {e_g} (F={Fg:.6e}) but the oracle ranks "
+                                (f"unit {key} step {t}: device evicted {e_g} (F={Fg:.6e}) but the oracle ranks "
                                  f"{own} last (F={cF[C_]:.6e}), no near tie")
-                            rep.near_tie_resyncs += 1
+                            r["resyncs"] += 1
                     else:
-                        assert e_g == -1, f"unit {(l, b, h)} step {t}: device evicted {e_g} but the cache is not full"
+                        assert e_g == -1, f"unit {key} step {t}: device evicted {e_g} but the cache is not full"
                 if i in Fsnap and len(cp) > C_:
+                    l, b, h = key
                     Fg_all, pos_all = Fsnap[i][l]
                     Fg_u = Fg_all[b, h].cpu().numpy()
                     # the snapshot is taken after the step: the evicted slot now holds position t
@@ -170,29 +256,45 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
                     lut = {int(p): float(f) for p, f in zip(pos_u, Fg_u)}
                     for p, f in zip(cp, cF):
                         if int(p) in lut and lut[int(p)] >= 0 and f > 1e-20:
-                            rep.max_F_rel_err = max(rep.max_F_rel_err, abs(lut[int(p)] - f) / f)
-                            rep.F_compared += 1
-                rep.unit_steps += 1
-            gpos = mk.view(l)["pos"][b, h, :mk.view(l)["count"]].cpu().numpy()
+                            r["Fmax"] = max(r["Fmax"], abs(lut[int(p)] - f) / f)
+                            r["Fcmp"] += 1
+            return r
+
+        results = list(pool.map(follow, range(len(units))))
+        gpos = {l: views[l]["pos"][:, :, :mk.view(l)["count"]].cpu().numpy() for l in layers_checked}
+        for ui, r in enumerate(results):
+            l, b, h = units[ui]
+            rep.max_out_err = max(rep.max_out_err, r["err"])
+            rep.evictions += r["evictions"]
+            rep.near_tie_resyncs += r["resyncs"]
+            rep.max_F_rel_err = max(rep.max_F_rel_err, r["Fmax"])
+            rep.F_compared += r["Fcmp"]
+            rep.min_rel_gap = min(rep.min_rel_gap, r["gap"])
+            rep.unit_steps += ns
+            same = set(gpos[l][b, h].tolist()) == set(orac[(l, b, h)].positions().tolist())
             if ev_c is not None:
-                assert set(gpos.tolist()) == set(u.positions().tolist()), f"unit {(l, b, h)}: retained sets differ"
+                assert same, f"unit {(l, b, h)}: retained sets differ"
+            elif r["gap"] > TIE_REL:
+                # no per-step resync in this mode: without a near tie in the chunk the sets must still agree
+                assert same, f"unit {(l, b, h)}: retained sets differ after a chunk without a near tie"
         done += ns
         rep.steps = done
     if rep.F_compared:
         assert rep.max_F_rel_err < 1e-3, f"fused scores off by {rep.max_F_rel_err:.3e} relative"
+    pool.shutdown()
     mk.close()
     return rep
 
 
 def run_parity_coarse(w: synth.Workload, T: int, steps: int, n_units: int = 4, kernel: str = "auto",
-                      device: str = "cuda:0") -> ParityReport:
+                      device: str = "cuda:0", synth_device=None) -> ParityReport:
     """Lock-step parity for coarse-grained eviction (the policy runs every T-th step and may drop several
     tokens at once).  After every step the retained position set of each checked unit is read back; what the
     device dropped is the oracle's set before the step, plus the new token, minus that.  The oracle is made
     to drop the same tokens, and wherever that differs from its own ranking every token in the difference
     must be a near tie with the boundary of its top C."""
     dev = torch.device(device)
-    st = synth.Stream(w, dev)
+    st = _DeviceStream(w, synth_device or dev, dev)
     tdt = synth.torch_dtype(w.dtype)
     G, d, P, R, C_ = w.group, w.head_dim, w.prompt_len, w.R, w.C
     units = pick_units(w, n_units)
@@ -208,17 +310,13 @@ def run_parity_coarse(w: synth.Workload, T: int, steps: int, n_units: int = 4, k
     mk.sync()
     orac = {}
     for (l, b, h) in units:
-        u = ora.Unit(G, d, C_, R, w.fusion, evict_interval=T)
-        u.prefill(k32[l, b, h].double().cpu().numpy(), v32[l, b, h].double().cpu().numpy(),
-                  qw32[l, b, h * G:(h + 1) * G].double().cpu().numpy())
         view = mk.view(l)
-        gp = set(view["pos"][b, h, :view["count"]].cpu().numpy().tolist())
-        if gp != set(u.positions().tolist()):
-            kth, k1 = u.last_boundary()
-            assert near_tie(kth, k1), f"prefill retained set differs for unit {(l, b, h)} without a near tie"
-            rep.prefill_dropped += 1
-            continue
+        gp = view["pos"][b, h, :view["count"]].cpu().numpy()
+        u, resync = oracle_unit_following(lambda: ora.Unit(G, d, C_, R, w.fusion, evict_interval=T), _f64(k32[l, b, h]),
+                                          _f64(v32[l, b, h]), _f64(qw32[l, b, h * G:(h + 1) * G]), gp, f"unit {(l, b, h)}")
+        rep.prefill_resyncs += int(resync)
         orac[(l, b, h)] = u
+    rep.units = len(orac)
     peak = 0
     for i in range(steps):
         t = P + i
@@ -261,7 +359,6 @@ def run_parity_coarse(w: synth.Workload, T: int, steps: int, n_units: int = 4, k
             else:
                 assert not dropped, f"unit {(l, b, h)} step {t}: device dropped {dropped} on a step without the policy"
             assert set(u.positions().tolist()) == gp, f"unit {(l, b, h)} step {t}: retained sets differ"
-            # K rows of the retained tokens are the rows that were appended, bit for bit
             rep.unit_steps += 1
         rep.steps = i + 1
     rep.F_compared = peak        # reused: the largest fill seen (C + R + T - 1 expected)

@@ -14,7 +14,7 @@ SMALL = synth.Workload("small", 2, 2, 8, 2, 128, "bf16", 300, 96, 200, 16, "sum"
 def _report(rep):
     print(f"\n[parity] kernel={rep.kernel} steps={rep.steps} unit_steps={rep.unit_steps} max_out_err={rep.max_out_err:.3e} "
           f"evictions={rep.evictions} near_tie_resyncs={rep.near_tie_resyncs} max_F_rel_err={rep.max_F_rel_err:.3e} "
-          f"(F compared {rep.F_compared}) prefill_dropped={rep.prefill_dropped}")
+          f"(F compared {rep.F_compared}) prefill_resyncs={rep.prefill_resyncs} min_rel_gap={rep.min_rel_gap:.2e}")
 
 
 @pytest.mark.parametrize("seed_off", [0, 100, 200])
@@ -22,7 +22,7 @@ def test_config0_every_unit_every_step(seed_off):
     w = synth.WORKLOADS["c0"]
     rep = run_parity(w.replace(seed=w.seed + seed_off), steps=w.steps, n_units=w.units, chunk=128)
     _report(rep)
-    assert rep.unit_steps == (w.units - rep.prefill_dropped) * w.steps and rep.evictions > 0
+    assert rep.unit_steps == w.units * w.steps and rep.evictions > 0
     assert rep.near_tie_resyncs <= 0.01 * rep.evictions + 2
 
 
@@ -346,6 +346,45 @@ def test_full_size_config4_sampled_units(name):
     rep = run_parity(w, steps=steps, n_units=6, kernel="auto", check_F_every=8)
     _report(rep)
     assert rep.kernel == "tc" and rep.evictions >= 5 * steps
+
+
+# ---- the configurations over their whole length: every generated step of a seeded sample of units (first and
+# last layer / batch row included) is followed by the oracle; all other units run on the device beside them
+def test_full_length_config1_every_generated_step():
+    w = synth.WORKLOADS["c1"]
+    rep = run_parity(w, steps=w.steps, n_units=8, chunk=256, check_F_every=1024)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.steps == 8192 and rep.units == 8
+    assert rep.evictions == 8 * 8192 and rep.near_tie_resyncs <= 0.002 * rep.evictions + 2
+
+
+def test_full_length_config2_every_generated_step():
+    w = synth.WORKLOADS["c2"]
+    rep = run_parity(w, steps=w.steps, n_units=8, chunk=64, check_F_every=512)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.steps == 4096 and rep.units == 8
+    assert rep.evictions == 8 * 4096 and rep.near_tie_resyncs <= 0.002 * rep.evictions + 2
+
+
+def test_config3_from_its_real_prompt_through_the_fill_into_eviction():
+    # 512-token prompt: 3552 steps that only append, then the cache is full (C + R = 4064) and every step evicts
+    w = synth.WORKLOADS["c3"]
+    fill = w.C + w.R - w.prompt_len
+    steps = fill + 544
+    rep = run_parity(w, steps=steps, n_units=4, chunk=128, check_F_every=128)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.units == 4
+    assert rep.evictions == 4 * 544 and rep.F_compared > 0
+
+
+def test_config1_all_units_prompt_phase_and_first_steps_against_the_oracle():
+    # every one of the 256 units: retained set after the prompt phase (near-tie rule), K/V rows bit for bit, then
+    # 16 decode steps with outputs and evictions compared
+    w = synth.WORKLOADS["c1"]
+    rep = run_parity(w, steps=16, n_units=w.units, chunk=16, check_F_every=16)
+    _report(rep)
+    assert rep.units == 256 and rep.unit_steps == 256 * 16 and rep.evictions == 256 * 16
+    assert rep.prefill_resyncs <= 2
 
 
 def test_tc_matches_cuda_core_kernel_on_device():
