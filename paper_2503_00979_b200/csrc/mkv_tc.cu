@@ -51,6 +51,7 @@ __host__ __device__ constexpr int tc_threads(int ng) { return 32 * (3 + 4 * ng +
 constexpr int kFirstComputeWarp = 3;
 constexpr int kGroupThreads = 128;
 constexpr long long kWaitCycles = 4000000000ll;   // default limit of a device-side wait: about two seconds
+constexpr long long kShortWaitCycles = 1000000ll; // limits below this are polled (see mbar_wait)
 constexpr int kFinFloats = 4 * kMaxGroup + 128 + 256 + 64 + 32 + 8;   // epilogue scratch of finalize_fast
 // epilogue group: finalize scratch, flag, merged (m, l), per-warp scale factors
 constexpr int kEpiFloats = kFinFloats + 8 + 2 * kMaxGroup + kMaxComputeWarps * kMaxGroup;
@@ -113,14 +114,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Which wait gave up (recorded in the CTA's abort flag and reported to the host)
 enum WaitCode { kWaitQEmpty = 1, kWaitKEmpty, kWaitVEmpty, kWaitQFull, kWaitKFull, kWaitTEmpty, kWaitTFull, kWaitVFull,
                 kWaitPFree, kWaitUDone, kWaitDrain };
-// Bounded wait.  Gives up after `limit` clock ticks or as soon as another thread has raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort, int code, long long limit)
+// Bounded wait.  Gives up after `limit` clock ticks or as soon as another thread has raised `abort`.  The common
+// case - the phase has completed, or completes within the time the hardware lets try_wait block - is inlined; the
+// rest is a function call, which keeps the callers' loops small.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort, int code, long long limit)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
+    if (limit < kShortWaitCycles) {
+        // try_wait may itself block for a while before it answers; a short limit (tests lower it to make a wait run
+        // out on purpose) is honoured by polling with the non-blocking form
+        while (!mbar_test_wait(bar, parity)) {
+            if (*abort) return false;
+            if (clock64() - t0 > limit) { *abort = code; return false; }
+        }
+        return true;
+    }
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 0) {
@@ -128,6 +147,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (clock64() - t0 > limit) { *abort = code; return false; }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort, int code, long long limit)
+{
+    if (limit >= kShortWaitCycles && mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort, code, limit);
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -671,6 +695,9 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 if (rings > 0) mbar_wait(bar_qfull, (uint32_t)((rings - 1) & 1), &dummy, kWaitDrain, kWaitCycles);
             }
         }
+        // lanes 1-31 skipped the loop: the warp must be whole again before it reaches the CTA barrier of the tail
+        // (bar.sync is an aligned instruction; lanes of one warp arriving at different times is undefined)
+        __syncwarp();
     } else if (warp == 2) {
         // ------------------------------------------------ TMA producer: V tiles (one lane)
         if (lane == 0) {
@@ -699,6 +726,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     mbar_wait(bar_vfull + 8 * (T % SV), (uint32_t)((T / SV) & 1), &dummy, kWaitDrain, kWaitCycles);
             }
         }
+        __syncwarp();       // see the K producer
     } else if (warp == 1) {
         // ------------------------------------------------ new-query substitution + MMA issue
         Walk w(a.U, n);
