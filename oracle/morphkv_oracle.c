@@ -34,7 +34,11 @@
  *   - prefill: one application of Algorithm 1 with the whole prompt as G_i and
  *     the last min(R,P) prompt tokens (full causal profiles) as the window;
  *   - evict_interval T > 1 (coarse-grained eviction appendix): the policy runs
- *     on every T-th decode step only; the cache peaks at C + R + T - 1.
+ *     on every T-th decode step only; the cache peaks at C + R + T - 1;
+ *   - norm_mode CURRENT (the other reading of Eq. 4's AW_r): each window row's
+ *     stored weights are renormalised over the tokens that are still cached
+ *     when the scores are taken (a row never saw tokens newer than itself, so
+ *     this is causal inside the window); the default FROZEN uses them as stored.
  *
  * Pinned by tests/test_oracle_pins.py (full-attention special case against an
  * independent causal attention, the paper's worked 0.3/0.05 example, cache
@@ -54,6 +58,7 @@ enum { ORA_SUM = 0, ORA_MAX = 1 };
 
 typedef struct ora_unit {
     int G, d, C, R, fusion, T, recompute;
+    int norm_current; /* 1: renormalise each window row over the tokens still cached (see header) */
     int cap;        /* physical slots: C + R + T (one transient slot for the new token) */
     int n;          /* occupied slots */
     long t;         /* position of the next token to decode */
@@ -109,6 +114,9 @@ void ora_destroy(ora_unit *u)
     free(u);
 }
 
+/* 0 = FROZEN (default), 1 = CURRENT */
+void ora_set_norm_mode(ora_unit *u, int current) { if (u) u->norm_current = current != 0; }
+
 static int free_slot(const ora_unit *u)
 {
     for (int s = 0; s < u->cap; ++s) if (u->pos[s] < 0) return s;
@@ -134,9 +142,11 @@ static double dot(const double *a, const double *b, int d)
     return s;
 }
 
-/* AW_r^g[k]: the weight window row `r` (head g) assigned to the token in `slot`. */
+/* AW_r^g[k]: the weight window row `r` (head g) assigned to the token in `slot`
+ * when r was generated (0 for a token newer than r: it was not there). */
 static double profile_weight(const ora_unit *u, int r, int g, int slot)
 {
+    if (u->pos[slot] > u->wpos[r]) return 0.0;
     if (!u->recompute) return u->A[((size_t)r * u->G + g) * u->cap + slot];
     const double *q = u->Q + ((size_t)r * u->G + g) * u->d;
     double s = dot(q, u->K + (size_t)slot * u->d, u->d) / sqrt((double)u->d);
@@ -175,6 +185,17 @@ static int score_and_select(ora_unit *u, const long *forced, int n_forced)
 {
     cand_t *c = (cand_t *)malloc((size_t)u->cap * sizeof(cand_t));
     int nc = 0;
+    /* CURRENT: what is left of each row's weight mass on the tokens still cached (1 under FROZEN) */
+    double *mass = (double *)malloc((size_t)(u->R + 1) * u->G * sizeof(double));
+    for (int r = 0; r <= u->R; ++r)
+        for (int g = 0; g < u->G; ++g) {
+            double m = 1.0;
+            if (u->norm_current && u->wpos[r] >= 0) {
+                m = 0.0;
+                for (int s = 0; s < u->cap; ++s) if (u->pos[s] >= 0) m += profile_weight(u, r, g, s);
+            }
+            mass[r * u->G + g] = m;
+        }
     for (int s = 0; s < u->cap; ++s) {
         if (u->pos[s] < 0 || in_window(u, u->pos[s])) continue;
         double F = 0.0;
@@ -182,13 +203,14 @@ static int score_and_select(ora_unit *u, const long *forced, int n_forced)
         for (int r = 0; r <= u->R; ++r) {
             if (u->wpos[r] < 0) continue;
             double S = 0.0;                                   /* GQA aggregate */
-            for (int g = 0; g < u->G; ++g) S += profile_weight(u, r, g, s);
+            for (int g = 0; g < u->G; ++g) S += profile_weight(u, r, g, s) / mass[r * u->G + g];
             if (u->fusion == ORA_SUM) F += S;                 /* Eq. 5 */
             else if (first || S > F) F = S;                   /* Eq. 6 */
             first = 0;
         }
         c[nc].F = F; c[nc].pos = u->pos[s]; c[nc].slot = s; ++nc;
     }
+    free(mass);
     qsort(c, (size_t)nc, sizeof(cand_t), cand_cmp);
     u->n_cand = nc;
     for (int i = 0; i < nc; ++i) { u->cand_pos[i] = c[i].pos; u->cand_F[i] = c[i].F; }

@@ -41,6 +41,8 @@ def _load():
         lib.ora_create.restype = C.c_void_p
         lib.ora_create.argtypes = [C.c_int] * 7
         lib.ora_destroy.argtypes = [C.c_void_p]
+        lib.ora_set_norm_mode.argtypes = [C.c_void_p, C.c_int]
+        lib.ora_set_norm_mode.restype = None
         lib.ora_prefill.argtypes = [C.c_void_p, dp, dp, dp, C.c_int]
         lib.ora_prefill_forced.argtypes = [C.c_void_p, dp, dp, dp, C.c_int, lp, C.c_int]
         lib.ora_step.argtypes = [C.c_void_p, dp, dp, dp, dp, lp, C.c_int]
@@ -73,13 +75,17 @@ def _f64(a) -> np.ndarray:
 class Unit:
     """One MorphKV unit: a (layer, batch row, KV head) cache serving G query heads."""
 
-    def __init__(self, G: int, d: int, C_: int, R: int, fusion, evict_interval: int = 1, recompute: bool = False):
+    def __init__(self, G: int, d: int, C_: int, R: int, fusion, evict_interval: int = 1, recompute: bool = False,
+                 norm: str = "frozen"):
         self.lib = _load()
         self.G, self.d, self.C, self.R, self.T = G, d, C_, R, evict_interval
         fusion = FUSION[fusion] if isinstance(fusion, str) else int(fusion)
         self.h = self.lib.ora_create(G, d, C_, R, fusion, evict_interval, int(recompute))
         if not self.h:
             raise ValueError("ora_create rejected the parameters")
+        if norm not in ("frozen", "current"):
+            raise ValueError(norm)
+        self.lib.ora_set_norm_mode(self.h, int(norm == "current"))
         self.cap = C_ + R + evict_interval
 
     def __del__(self):

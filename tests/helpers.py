@@ -56,8 +56,10 @@ class ShadowMorphKV:
     by a plain Python sort and also finds the best size-C subset by exhaustive enumeration.
     """
 
-    def __init__(self, G, d, C, R, fusion, evict_interval=1):
+    def __init__(self, G, d, C, R, fusion, evict_interval=1, norm="frozen"):
         self.G, self.d, self.C, self.R, self.fusion = G, d, C, R, fusion
+        # "current": a window row's weights are divided by what is left of its mass on the tokens still cached
+        self.norm = norm
         # coarse-grained eviction (appendix): the policy runs on generation steps T, 2T, 3T, ... only
         self.T = evict_interval
         self.generated = 0
@@ -88,8 +90,10 @@ class ShadowMorphKV:
     def _fused(self, cand):
         win = sorted(self._window())
         F = {}
+        left = {(r, g): (sum(wt for p, wt in self.profile[r][g].items() if p in self.cached) if self.norm == "current" else 1.0)
+                for r in win for g in range(self.G)}
         for c in cand:
-            per_row = [sum(self.profile[r][g][c] for g in range(self.G)) for r in win]
+            per_row = [sum(self.profile[r][g][c] / left[(r, g)] for g in range(self.G)) for r in win]
             F[c] = sum(per_row) if self.fusion == "sum" else max(per_row)
         return F
 

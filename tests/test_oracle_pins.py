@@ -329,6 +329,83 @@ def test_coarse_grained_eviction_against_exhaustive_shadow(oracle, fusion, T, G,
     assert multi > 0                                                   # several tokens dropped at once was exercised
 
 
+# ---- the other reading of Eq. 4: window rows renormalised over the tokens still cached ("current") ----
+@pytest.mark.parametrize("fusion", ["sum", "max"])
+@pytest.mark.parametrize("recompute", [False, True])
+@pytest.mark.parametrize("G,C,R,P", [(1, 3, 2, 5), (2, 4, 3, 9), (4, 5, 4, 12)])
+def test_current_normalisation_against_exhaustive_shadow(oracle, fusion, recompute, G, C, R, P):
+    w = TINY.replace(n_q_heads=2 * G, prompt_len=P, steps=16, C=C, R=R, fusion=fusion, seed=900 + G)
+    q, k, v = unit_inputs(w, 0, 0, 1, np.arange(P + w.steps))
+    u = oracle.Unit(G, w.head_dim, C, R, fusion, recompute=recompute, norm="current")
+    sh = ShadowMorphKV(G, w.head_dim, C, R, fusion, norm="current")
+    Rw = min(R, P)
+    for x in (u, sh):
+        x.prefill(k[:P], v[:P], q[:, P - Rw:P])
+    assert set(u.positions().tolist()) == sh.cached
+    n_sel, rescaled = 0, False
+    for s in range(w.steps):
+        t = P + s
+        o = u.step(q[:, t], k[t], v[t])
+        o2 = sh.step(q[:, t], k[t], v[t])
+        assert np.abs(o - o2).max() < 1e-12
+        assert set(u.positions().tolist()) == sh.cached
+        if sh.last_F is not None:
+            n_sel += 1
+            pos, F = u.last_scores()
+            assert pos.tolist() == sh.last_ranked
+            assert np.allclose(F, [sh.last_F[p] for p in pos], rtol=1e-11, atol=1e-300)
+            # every window row's weights sum to 1 over what the row can still see, so a fused score under "current"
+            # is never below the stored-weights score of the same state, and is above it once mass was evicted
+            Ffrozen = ShadowMorphKV._fused(_with_norm(sh, "frozen"), set(pos.tolist()))
+            assert all(sh.last_F[p] >= Ffrozen[p] * (1 - 1e-12) for p in pos)
+            rescaled |= any(sh.last_F[p] > Ffrozen[p] * (1 + 1e-9) for p in pos)
+    assert n_sel > 0 and rescaled
+
+
+def _with_norm(shadow, norm):
+    """A view of a shadow's state that scores under the other normalisation (state before the last selection is not
+    needed: only weights of tokens still cached plus the just-dropped ones enter, which `profile` still holds)."""
+    import copy
+    other = copy.copy(shadow)
+    other.norm = norm
+    # scores are taken before the selection drops anything: restore the candidates of that moment
+    other.cached = set(shadow.cached) | set(shadow.last_dropped)
+    return other
+
+
+@pytest.mark.parametrize("fusion", ["sum", "max"])
+def test_current_equals_frozen_for_a_window_of_one(oracle, fusion):
+    # R = 1: the only window row was generated on this very step, nothing it saw has been evicted since
+    w = synth.WORKLOADS["c0"].replace(steps=60)
+    a, ua, _ = _run(oracle, w, R=1, fusion=fusion)
+    q, k, v = unit_inputs(w, 0, 0, 0, np.arange(w.prompt_len + 60))
+    u = oracle.Unit(w.group, w.head_dim, w.C, 1, fusion, norm="current")
+    u.prefill(k[:w.prompt_len], v[:w.prompt_len], q[:, w.prompt_len - 1:w.prompt_len])
+    b = np.array([u.step(q[:, w.prompt_len + s], k[w.prompt_len + s], v[w.prompt_len + s]) for s in range(60)])
+    assert np.array_equal(a, b) and np.array_equal(ua.positions(), u.positions())
+
+
+def test_current_scales_surviving_weights_by_the_evicted_mass(oracle):
+    # one window row (G = 1, R = 2 so that the older row has lived through one eviction): its weight on a survivor
+    # is the stored weight divided by 1 - (mass it had on the token evicted meanwhile)
+    w = TINY.replace(n_q_heads=2, n_kv_heads=2, prompt_len=6, steps=3, C=3, R=2)
+    q, k, v = unit_inputs(w, 0, 0, 0, np.arange(9))
+    sh = ShadowMorphKV(1, w.head_dim, 3, 2, "sum", norm="current")
+    u = oracle.Unit(1, w.head_dim, 3, 2, "sum", norm="current")
+    for x in (u, sh):
+        x.prefill(k[:6], v[:6], q[:, 4:6])
+    for t in (6, 7):
+        u.step(q[:, t], k[t], v[t]); sh.step(q[:, t], k[t], v[t])
+    pos, F = u.last_scores()
+    older, newer = 6, 7                       # window rows at the selection of step 7
+    gone = [p for p in sh.profile[older][0] if p not in sh.cached and p not in sh.last_dropped and p <= older]
+    assert gone                               # the older row did see a token that has been evicted since
+    lost = sum(sh.profile[older][0][p] for p in gone)
+    for p, f in zip(pos, F):
+        want = sh.profile[older][0][p] / (1.0 - lost) + sh.profile[newer][0][p]
+        assert abs(f - want) < 1e-13
+
+
 def test_t1_is_default(oracle):
     w = synth.WORKLOADS["c0"].replace(steps=30)
     a, ua, _ = _run(oracle, w)
