@@ -230,6 +230,75 @@ def replica_workload(w: synth.Workload, rank: int) -> synth.Workload:
     return w.replace(seed=w.seed + 1000 * rank)
 
 
+def secondary_record(w: synth.Workload, W: int, K: int, dev, per_layer: bool = False, kernel: str = "auto"):
+    """A second, smaller measurement in the same process (own context, device-resident inputs, same timing rules):
+    either K whole-stack steps of another workload, or K steps made of per-layer calls (one call per layer, the way
+    a model that runs its layers in sequence would use the library)."""
+    from paper_2503_00979_b200 import binding
+    tdt = synth.torch_dtype(w.dtype)
+    P, Rw = w.prompt_len, min(w.R, w.prompt_len)
+    st = synth.Stream(w, dev)
+    mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
+                         kernel=kernel, device=str(dev))
+    ks, vs, qws = [], [], []
+    for l in range(w.layers):
+        k, v = st.kv(np.arange(P), [l])
+        ks.append(k.to(tdt)); vs.append(v.to(tdt))
+        qws.append(st.q(np.arange(P - Rw, P), [l]).to(tdt))
+    k, v, qw = torch.cat(ks), torch.cat(vs), torch.cat(qws)
+    del ks, vs, qws
+    mk.prefill(k.contiguous(), v.contiguous(), qw.contiguous())
+    del k, v, qw
+    pos = np.arange(P, P + W + K)
+    kk, vv = st.kv(pos)
+    qs = st.q(pos).permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+    kn = kk.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+    vn = vv.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+    del kk, vv
+    outs = torch.empty_like(qs)
+    stream = torch.cuda.current_stream()
+
+    def run(lo, hi):
+        if not per_layer:
+            mk.decode_steps(qs[lo:hi], kn[lo:hi], vn[lo:hi], outs[lo:hi])
+            return
+        for i in range(lo, hi):
+            for l in range(w.layers):
+                mk.decode_step_layer(l, qs[i, l], kn[i, l], vn[i, l], outs[i, l])
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    clocks = ClockSampler(dev)
+    run(0, W)
+    mk.sync()
+    n_steady = mk.view(0)["count"]
+    launches0 = mk.launch_count
+    torch.cuda.synchronize()
+    e0.record(stream)
+    run(W, W + K)
+    e1.record(stream)
+    clocks.during(e1.query)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    mk.sync()
+    assert torch.isfinite(outs[W:].float()).all()
+    bytes_step = algorithmic_bytes_per_step(w, n_steady)
+    peak, _ = measured_peak_gbs()
+    achieved = bytes_step / (ms / K * 1e-3) / 1e9
+    rec = {"workload": w.name, "prompt_len": P, "cached_tokens_per_unit": n_steady, "steps": K, "warmup": W,
+           "ms_per_step": ms / K, "tokens_per_s": w.batch * K / (ms * 1e-3), "kernel": mk.kernel_name,
+           "gpu_launches": int(mk.launch_count - launches0),
+           "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                        "algorithmic_bytes_per_launch": bytes_step if not per_layer else bytes_step // w.layers},
+           "clocks": clocks.summary()}
+    if per_layer:
+        rec["calls"] = "one mkv_decode_step_layer call per layer"
+        rec["us_per_layer_call"] = 1e3 * ms / (K * w.layers)
+    mk.close()
+    del qs, kn, vn, outs
+    torch.cuda.empty_cache()
+    return rec
+
+
 def run_ours(args, w):
     import torch.distributed as dist
     from paper_2503_00979_b200 import binding
@@ -356,6 +425,17 @@ def run_ours(args, w):
                          "peak_source": peak_src, "kernel": f"decode_{mk.kernel_name}",
                          "algorithmic_bytes_per_launch": bytes_step},
         }
+        if world == 1 and args.also and w.name == "c1" and args.prompt_len == 0 and T == 1:
+            # second target configuration (started with a full cache so that every timed step evicts) and the
+            # per-layer calling pattern, measured in the same run
+            mk.close()
+            del qs, kn, vn, outs
+            torch.cuda.empty_cache()
+            c3 = synth.WORKLOADS["c3"]
+            line["also"] = [
+                secondary_record(c3.replace(prompt_len=c3.C + c3.R), W, min(K, 64), dev),
+                secondary_record(w, W, min(K, 32), dev, per_layer=True),
+            ]
         if world == 1 and not args.no_cpu_baseline:
             cores = len(os.sched_getaffinity(0))
             n_units = max(1, min(cores, w.units))
@@ -383,6 +463,8 @@ def main():
     ap.add_argument("--evict-interval", type=int, default=1,
                     help="run the policy every T-th step only (coarse-grained eviction appendix)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", dest="also", action="store_false",
+                    help="skip the secondary records (config 3 with a full cache; per-layer calls on config 1)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer arm (for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -71,6 +71,12 @@ typedef struct mkv_params {
     void *workspace;        /* device memory owned by the caller, 256-byte aligned, or NULL
                                to let the library allocate it with cudaMalloc              */
     size_t workspace_bytes;
+    int full_layers;        /* layer-aware variant (the appendix on selective layer retention): MorphKV is
+                               switched off for the first full_layers layers, which keep every token; the
+                               other layers run MorphKV as usual.  0 = none.                           */
+    int max_tokens;         /* with full_layers > 0: the cache of those layers holds this many tokens (prompt
+                               plus generated; > R).  While the sequence stays within it nothing is evicted
+                               there; beyond it those layers fall back to MorphKV with that capacity.    */
     unsigned long long wait_limit_cycles;
                             /* how long a device-side wait (on a copy, on the tensor cores, on another
                                warp) may spin before the kernel gives up, in GPU clock ticks; 0 = the
@@ -92,8 +98,9 @@ typedef struct mkv_view {
     float *ring_c;          /* [batch][n_kv_heads][R][G] log2-domain soft-max normaliser of a
                                ring row: weight(k) = exp2(q.k * log2(e)/sqrt(d) - ring_c);
                                +inf marks an empty row                                     */
-    int32_t count;          /* tokens cached per unit (the same for every unit)            */
-    int32_t capacity;       /* slots per unit: C + R, plus evict_interval if that is > 1  */
+    int32_t count;          /* tokens cached per unit of this layer (the same for every unit of it) */
+    int32_t capacity;       /* slots per unit: C + R, plus evict_interval if that is > 1; max_tokens
+                               for a layer that keeps every token                          */
     int64_t next_pos;       /* absolute position of the next token to decode               */
 } mkv_view;
 
@@ -158,6 +165,15 @@ mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const 
  * index, so a sequence of calls can be recorded into a CUDA graph. */
 mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                            void *out, void *stream);
+
+/* One layer of a decode step, for a model that runs its layers one after the other (the paper's implementation
+ * hooks MorphKV into each layer's attention call; "Implementation" paragraph): q, out
+ * [batch][n_q_heads][head_dim]; k_new, v_new [batch][n_kv_heads][head_dim] of layer `layer`.  The layers of a step
+ * must be called in order 0, 1, ..., layers - 1 (MKV_BAD_STATE otherwise); the step is complete after the last one.
+ * The results equal those of mkv_decode_step on the stacked tensors; a step may not mix the two calls.
+ * Asynchronous on `stream`. */
+mkv_status mkv_decode_step_layer(mkv_ctx *ctx, int layer, const void *q, const void *k_new,
+                                 const void *v_new, void *out, void *stream);
 
 /* n_steps consecutive decode steps; every tensor has a leading [n_steps] dimension. */
 mkv_status mkv_decode_steps(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new,

@@ -26,7 +26,7 @@ KERNEL = {"auto": 0, "simt": 1, "tc": 2}
 EXPORTS = [
     "mkv_default_params", "mkv_workspace_bytes", "mkv_create", "mkv_create_ex", "mkv_destroy", "mkv_prefill",
     "mkv_prefill_static",
-    "mkv_decode_step", "mkv_decode_steps", "mkv_decode_step_host", "mkv_cache_view", "mkv_sync", "mkv_last_error",
+    "mkv_decode_step", "mkv_decode_step_layer", "mkv_decode_steps", "mkv_decode_step_host", "mkv_cache_view", "mkv_sync", "mkv_last_error",
     "mkv_launch_count", "mkv_kernel_name",
 ]
 
@@ -36,7 +36,8 @@ class mkv_params(C.Structure):
         ("layers", C.c_int), ("batch", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int),
         ("head_dim", C.c_int), ("C", C.c_int), ("R", C.c_int), ("fusion", C.c_int), ("dtype", C.c_int),
         ("evict_interval", C.c_int), ("kernel", C.c_int), ("splits", C.c_int),
-        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("wait_limit_cycles", C.c_ulonglong),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("full_layers", C.c_int), ("max_tokens", C.c_int),
+        ("wait_limit_cycles", C.c_ulonglong),
     ]
 
 
@@ -77,6 +78,7 @@ def lib() -> C.CDLL:
         L.mkv_prefill.argtypes = [vp, vp, vp, vp, ip, vp]
         L.mkv_prefill_static.argtypes = [vp, vp, vp, vp, ip, vp]
         L.mkv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.mkv_decode_step_layer.argtypes = [vp, ip, vp, vp, vp, vp, vp]
         L.mkv_decode_steps.argtypes = [vp, vp, vp, vp, vp, ip, vp]
         L.mkv_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
         L.mkv_cache_view.argtypes = [vp, ip, C.POINTER(mkv_view)]
@@ -145,6 +147,10 @@ def mkv_decode_step(ctx, q, k_new, v_new, out, stream=None) -> int:
     return lib().mkv_decode_step(ctx, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream))
 
 
+def mkv_decode_step_layer(ctx, layer, q, k_new, v_new, out, stream=None) -> int:
+    return lib().mkv_decode_step_layer(ctx, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _stream(stream))
+
+
 def mkv_decode_steps(ctx, q, k_new, v_new, out, n_steps, stream=None) -> int:
     return lib().mkv_decode_steps(ctx, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), n_steps, _stream(stream))
 
@@ -199,7 +205,8 @@ class MorphKV:
     """A context whose workspace is a torch tensor.  Methods mirror the C calls and raise on error."""
 
     def __init__(self, layers, batch, n_q_heads, n_kv_heads, head_dim, C_, R, fusion="sum", dtype="bf16",
-                 evict_interval=1, kernel="auto", splits=0, device="cuda:0", wait_limit_cycles=0):
+                 evict_interval=1, kernel="auto", splits=0, device="cuda:0", wait_limit_cycles=0,
+                 full_layers=0, max_tokens=0):
         self.device = torch.device(device)
         p = mkv_default_params()
         p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = layers, batch, n_q_heads, n_kv_heads, head_dim
@@ -208,6 +215,7 @@ class MorphKV:
         p.dtype = DTYPE[dtype] if isinstance(dtype, str) else int(dtype)
         p.evict_interval, p.kernel, p.splits = evict_interval, KERNEL[kernel], splits
         p.wait_limit_cycles = wait_limit_cycles
+        p.full_layers, p.max_tokens = full_layers, max_tokens
         self.torch_dtype = torch.float32 if p.dtype == 1 else torch.bfloat16
         self.shape = dict(L=layers, B=batch, Hq=n_q_heads, Hkv=n_kv_heads, d=head_dim, C=C_, R=R,
                           G=n_q_heads // max(1, n_kv_heads))
@@ -248,6 +256,12 @@ class MorphKV:
         if out is None:
             out = torch.empty_like(q)
         self._check(mkv_decode_step(self.ctx, q, k_new, v_new, out, stream), "mkv_decode_step")
+        return out
+
+    def decode_step_layer(self, layer, q, k_new, v_new, out=None, stream=None):
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(mkv_decode_step_layer(self.ctx, layer, q, k_new, v_new, out, stream), "mkv_decode_step_layer")
         return out
 
     def decode_steps(self, q, k_new, v_new, out=None, stream=None):

@@ -21,7 +21,9 @@ struct Layout {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Shape {
-    int U, G, D, R, C, cap, splits, T, tc_grid_size;
+    int layers;             // layers served by this context's own arena
+    int upl;                // units per layer = batch * n_kv_heads
+    int U, G, D, R, C, cap, splits, T, tc_grid_size, tc_grid_layer;
     size_t es;
 };
 
@@ -42,7 +44,7 @@ Layout make_layout(const Shape &s)
     L.part_o = take(U * sp * G * D * 4);
     L.ticket = take(U * 4);
     L.evicted = take(U * 4);
-    L.state = take(sizeof(DevState));
+    L.state = take(sizeof(DevState) * (1 + (size_t)s.layers));     // whole-stack state, then one per layer
     L.stage_q = take(U * G * D * s.es);
     L.stage_k = take(U * D * s.es);
     L.stage_v = take(U * D * s.es);
@@ -62,6 +64,8 @@ bool params_valid(const mkv_params *p)
     if (p->dtype != MKV_DTYPE_BF16 && p->dtype != MKV_DTYPE_F32) return false;
     if (p->evict_interval < 0 || p->splits < 0) return false;
     if (p->kernel != MKV_KERNEL_AUTO && p->kernel != MKV_KERNEL_SIMT && p->kernel != MKV_KERNEL_TC) return false;
+    if (p->full_layers < 0 || p->full_layers >= p->layers) return false;
+    if (p->full_layers > 0 && p->max_tokens <= p->R) return false;
     const long long units = (long long)p->layers * p->batch * p->n_kv_heads;
     if (units > (1 << 24)) return false;
     if ((long long)p->C + p->R + (p->evict_interval > 1 ? p->evict_interval : 0) > (1 << 24)) return false;
@@ -73,7 +77,9 @@ enum KernelKind { kKindSimt = 0, kKindTc = 1 };
 // kernel choice and split count implied by the parameters; returns false if unsupported
 bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
 {
-    s->U = p->layers * p->batch * p->n_kv_heads;
+    s->layers = p->layers - p->full_layers;
+    s->upl = p->batch * p->n_kv_heads;
+    s->U = s->layers * s->upl;
     s->G = p->n_q_heads / p->n_kv_heads;
     s->D = p->head_dim;
     s->R = p->R;
@@ -90,7 +96,12 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
         *kind = kKindTc;
         // the persistent grid (148 SMs on B200; correctness does not depend on the count)
         s->tc_grid_size = tc_grid(s->U, s->cap, p->splits, 148);
-        s->splits = tc_partials_per_unit(s->U, s->cap, s->tc_grid_size);
+        // a per-layer call sees only a layer's units: ranges of about an eighth of a unit's tiles, so that a layer
+        // of few units still spreads over the SMs while a unit stays within eight CTAs
+        s->tc_grid_layer = tc_grid(s->upl, s->cap, p->splits > 0 ? p->splits : 8, 148);
+        const int sp_all = tc_partials_per_unit(s->U, s->cap, s->tc_grid_size);
+        const int sp_layer = tc_partials_per_unit(s->upl, s->cap, s->tc_grid_layer);
+        s->splits = sp_all > sp_layer ? sp_all : sp_layer;
         return true;
     }
     *kind = kKindSimt;
@@ -99,23 +110,29 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     if (sp > max_splits) sp = max_splits;
     s->splits = sp;
     s->tc_grid_size = 0;
+    s->tc_grid_layer = 0;
     return true;
 }
 
 }  // namespace
 
 struct mkv_ctx {
-    mkv_params p;
+    mkv_params p;     // as given; p.layers counts every layer, s.layers those in this context's own arena
     Shape s;
     Layout L;
     KernelKind kind;
-    TcPlan *plan;
+    TcPlan *plan, *plan_layer;
+    mkv_ctx *full;    // layer-aware variant: the context of the first p.full_layers layers, which keep every token
     char *base;
+    int device;       // the CUDA device the context was created on
     bool owns_workspace;
     bool prefilled;
     long long t;      // host mirror of the device step state
     int n;
     int steps;
+    int next_layer;   // per-layer calls: the layer (of this context's own) expected next; 0 at a step boundary
+    int cursor;       // per-layer calls: the layer of the whole model expected next (kept by the outer context)
+    int state_ahead;  // 0: whole-stack and per-layer device states level, 1: whole-stack ahead, 2: per-layer ahead
     unsigned long long launches;
     PrefillScratch prefill_scratch;
     char err[256];
@@ -140,6 +157,7 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.part_ml = (float *)(b + c->L.part_ml); a.part_o = (float *)(b + c->L.part_o);
     a.ticket = (int *)(b + c->L.ticket); a.evicted_pos = (int *)(b + c->L.evicted);
     a.st = (DevState *)(b + c->L.state);
+    a.u0 = 0;
     a.U = c->s.U; a.G = c->s.G; a.R = c->s.R; a.C = c->s.C; a.cap = c->s.cap; a.splits = c->s.splits;
     a.fusion = c->p.fusion == MKV_FUSION_SUM ? kFusionSum : kFusionMax;
     a.T = c->s.T;
@@ -157,10 +175,46 @@ bool clear_arena(mkv_ctx *c, cudaStream_t stream)
            cudaMemsetAsync(c->base + c->L.ring_q, 0, rq, stream) == cudaSuccess;
 }
 
-mkv_status launch_step(mkv_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream)
+// Arguments of a launch that covers one layer of the context's own: every arena pointer is moved to the layer's
+// first unit, the inputs and `out` are that layer's tensors, and the layer's own step state is used.
+DecodeArgs make_args_layer(const mkv_ctx *c, int layer, const void *q, const void *k, const void *v, void *out)
 {
-    const DecodeArgs a = make_args(ctx, q, k, v, out);
-    const cudaError_t e = ctx->kind == kKindTc ? launch_decode_tc(ctx->plan, a, stream)
+    DecodeArgs a = make_args(c, q, k, v, out);
+    const Shape &s = c->s;
+    const size_t u0 = (size_t)layer * s.upl;
+    a.K = (char *)a.K + u0 * s.cap * s.D * s.es; a.V = (char *)a.V + u0 * s.cap * s.D * s.es;
+    a.pos += u0 * s.cap;
+    a.ring_q = (char *)a.ring_q + u0 * s.R * s.G * s.D * s.es; a.ring_c += u0 * s.R * s.G;
+    a.s_new += u0 * s.G * s.cap; a.F += u0 * s.cap;
+    a.part_ml += u0 * s.splits * s.G * 2; a.part_o += u0 * s.splits * s.G * s.D;
+    a.ticket += u0; a.evicted_pos += u0;
+    a.st = a.st + 1 + layer;
+    a.u0 = (int)u0;
+    a.U = s.upl;
+    return a;
+}
+
+// Brings the whole-stack state and the per-layer states level before a call of the other kind (only at a step
+// boundary: every layer has taken the same number of steps then).
+mkv_status level_states(mkv_ctx *ctx, int want, cudaStream_t stream)
+{
+    if (ctx->state_ahead == 0 || ctx->state_ahead == want) return MKV_OK;
+    DevState *st = (DevState *)(ctx->base + ctx->L.state);
+    const cudaError_t e = ctx->state_ahead == 1 ? launch_copy_state(st + 1, ctx->s.layers, st, stream)
+                                                : launch_copy_state(st, 1, st + 1, stream);
+    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "state copy launch failed: %s", cudaGetErrorString(e));
+    ctx->launches += 1;
+    ctx->state_ahead = 0;
+    return MKV_OK;
+}
+
+// One decode step of the whole stack (layer < 0) or of one layer of this context's own.
+mkv_status launch_step(mkv_ctx *ctx, int layer, const void *q, const void *k, const void *v, void *out, cudaStream_t stream)
+{
+    const mkv_status ls = level_states(ctx, layer < 0 ? 1 : 2, stream);
+    if (ls != MKV_OK) return ls;
+    const DecodeArgs a = layer < 0 ? make_args(ctx, q, k, v, out) : make_args_layer(ctx, layer, q, k, v, out);
+    const cudaError_t e = ctx->kind == kKindTc ? launch_decode_tc(layer < 0 ? ctx->plan : ctx->plan_layer, a, stream)
                                                : launch_decode_simt(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "decode launch failed: %s", cudaGetErrorString(e));
     ctx->launches += 1;
@@ -172,12 +226,162 @@ mkv_status launch_step(mkv_ctx *ctx, const void *q, const void *k, const void *v
         if (e2 != cudaSuccess) return fail(ctx, MKV_CUDA, "compaction launch failed: %s", cudaGetErrorString(e2));
         ctx->launches += 1;
     }
+    if (layer >= 0) {
+        ctx->state_ahead = 2;
+        ctx->next_layer = layer + 1 < ctx->s.layers ? layer + 1 : 0;
+        if (ctx->next_layer != 0) return MKV_OK;          // the step is complete once its last layer has run
+    } else {
+        ctx->state_ahead = 1;
+    }
     ctx->t += 1;
     ctx->steps += 1;
     if (!ev) ctx->n += 1;
     else if (ctx->s.T > 1) ctx->n = ctx->s.C + ctx->s.R;
     return MKV_OK;
 }
+
+// ---- the calls on one context's own layers ------------------------------------------------------------------
+mkv_status core_create(mkv_ctx **out, const mkv_params *p, void *workspace, size_t workspace_bytes)
+{
+    *out = nullptr;
+    Shape s;
+    KernelKind kind;
+    if (!resolve(p, &s, &kind)) return MKV_UNSUPPORTED;
+    const Layout L = make_layout(s);
+    if (workspace && workspace_bytes < L.total) return MKV_OOM;
+    mkv_ctx *c = new (std::nothrow) mkv_ctx;
+    if (!c) return MKV_OOM;
+    memset(c, 0, sizeof(*c));
+    c->p = *p; c->s = s; c->L = L; c->kind = kind;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); delete c; return MKV_CUDA; }
+    if (workspace) {
+        c->base = (char *)workspace;
+    } else {
+        void *mem = nullptr;
+        if (cudaMalloc(&mem, L.total) != cudaSuccess) {
+            cudaGetLastError();
+            delete c;
+            return MKV_OOM;
+        }
+        c->base = (char *)mem;
+        c->owns_workspace = true;
+    }
+    if (kind == kKindTc) {
+        const DecodeArgs a = make_args(c, nullptr, nullptr, nullptr, nullptr);
+        char msg[200] = "";
+        cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, p->wait_limit_cycles, msg, sizeof(msg));
+        if (e == cudaSuccess) e = tc_plan_create(&c->plan_layer, a, s.tc_grid_layer, p->wait_limit_cycles, msg, sizeof(msg));
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            if (c->plan) tc_plan_destroy(c->plan);
+            if (c->owns_workspace) cudaFree(c->base);
+            delete c;
+            return e == cudaErrorMemoryAllocation ? MKV_OOM : MKV_CUDA;
+        }
+    }
+    *out = c;
+    return MKV_OK;
+}
+
+void core_destroy(mkv_ctx *ctx)
+{
+    if (!ctx) return;
+    if (ctx->plan) tc_plan_destroy(ctx->plan);
+    if (ctx->plan_layer) tc_plan_destroy(ctx->plan_layer);
+    if (ctx->prefill_scratch.ptr) cudaFree(ctx->prefill_scratch.ptr);
+    if (ctx->owns_workspace && ctx->base) cudaFree(ctx->base);
+    delete ctx;
+}
+
+// use_static: scratch in the library's fixed device array instead of an allocation
+mkv_status core_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, cudaStream_t stream,
+                        bool use_static, const char *who)
+{
+    char where[64];
+    snprintf(where, sizeof(where), "%s", who);
+    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "%s: context already holds a sequence", where);
+    const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
+    if (use_static) {
+        const size_t need = ((size_t)Rw * ctx->s.G + 1) * (size_t)prompt_len;
+        if (need > prefill_static_max_floats()) {
+            snprintf(ctx->err, sizeof(ctx->err),
+                     "mkv_prefill_static: one unit needs (min(R,P)*G + 1) * prompt_len = %zu floats of scratch, the fixed "
+                     "array holds %zu; use mkv_prefill for this prompt", need, prefill_static_max_floats());
+            return MKV_UNSUPPORTED;
+        }
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device)
+            return fail(ctx, MKV_INVALID_ARG, "%s: the current CUDA device is not the one the context was created on", where);
+    }
+    const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
+    if (!clear_arena(ctx, stream)) return fail(ctx, MKV_CUDA, "%s: clearing the arena failed", where);
+    const bool f32 = ctx->p.dtype == MKV_DTYPE_F32;
+    const int n_states = 1 + ctx->s.layers;
+    const cudaError_t e = use_static
+        ? run_prefill_static(a, f32, ctx->s.D, k, v, q_window, prompt_len, stream, &ctx->launches, ctx->device, n_states)
+        : run_prefill(a, f32, ctx->s.D, k, v, q_window, prompt_len, stream, &ctx->launches, &ctx->prefill_scratch, n_states);
+    if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(ctx, MKV_OOM, "%s: no memory for scratch", where); }
+    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase: %s", cudaGetErrorString(e));
+    ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
+    ctx->t = prompt_len;
+    ctx->steps = 0;
+    ctx->next_layer = 0;
+    ctx->state_ahead = 0;
+    ctx->prefilled = true;
+    return MKV_OK;
+}
+
+mkv_status core_sync(mkv_ctx *ctx, cudaStream_t stream)
+{
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e));
+    // whole-stack state first, then the per-layer states
+    const int ns = 1 + ctx->s.layers;
+    DevState *st = new (std::nothrow) DevState[ns];
+    if (!st) return fail(ctx, MKV_OOM, "mkv_sync: out of host memory%s");
+    e = cudaMemcpy(st, ctx->base + ctx->L.state, sizeof(DevState) * ns, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { delete[] st; return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e)); }
+    int err = kErrNone;
+    for (int i = 0; i < ns && err == kErrNone; ++i) err = st[i].err;
+    const DevState cur = st[ctx->state_ahead == 2 ? 1 : 0];
+    delete[] st;
+    if (err == kErrCacheOverflow)
+        return fail(ctx, MKV_BAD_STATE, "a decode step found no free slot: coarse-grained eviction ran out of step%s");
+    if (err != kErrNone) {
+        char code[32];
+        snprintf(code, sizeof(code), " (wait code %d)", err);
+        return fail(ctx, MKV_DEVICE_TIMEOUT, "a device-side wait ran out of iterations%s", code);
+    }
+    // the device-resident state is authoritative (steps replayed from a CUDA graph advance
+    // it without passing through this library); the host mirror follows it at a step boundary
+    if (ctx->prefilled && ctx->next_layer == 0) { ctx->t = cur.t; ctx->n = cur.n; ctx->steps = cur.steps; }
+    return MKV_OK;
+}
+
+void core_view(mkv_ctx *ctx, int layer, mkv_view *view)
+{
+    const size_t u0 = (size_t)ctx->s.upl * layer;
+    const Shape &s = ctx->s;
+    char *b = ctx->base;
+    view->K = b + ctx->L.K + u0 * s.cap * s.D * s.es;
+    view->V = b + ctx->L.V + u0 * s.cap * s.D * s.es;
+    view->pos = (int32_t *)(b + ctx->L.pos) + u0 * s.cap;
+    view->F = (float *)(b + ctx->L.F) + u0 * s.cap;
+    view->evicted_pos = (int32_t *)(b + ctx->L.evicted) + u0;
+    view->ring_q = b + ctx->L.ring_q + u0 * s.R * s.G * s.D * s.es;
+    view->ring_c = (float *)(b + ctx->L.ring_c) + u0 * s.R * s.G;
+    // between the per-layer calls of a step the layers below next_layer have taken the step already
+    const bool ahead = layer < ctx->next_layer;
+    const bool ev = step_scores(ctx->t, ctx->n, ctx->steps, s.R, s.C, s.T);
+    view->count = !ahead ? ctx->n : (!ev ? ctx->n + 1 : (s.T > 1 ? s.C + s.R : ctx->n));
+    view->capacity = s.cap;
+    view->next_pos = ctx->t + (ahead ? 1 : 0);
+}
+
+// byte offsets of the first own layer inside whole-model tensors
+size_t q_bytes_per_layer(const mkv_ctx *c) { return (size_t)c->p.batch * c->p.n_q_heads * c->s.D * c->s.es; }
+size_t kv_bytes_per_layer(const mkv_ctx *c) { return (size_t)c->p.batch * c->p.n_kv_heads * c->s.D * c->s.es; }
+const char *off(const void *p, size_t bytes) { return (const char *)p + bytes; }
 
 }  // namespace
 
@@ -193,13 +397,33 @@ void mkv_default_params(mkv_params *p)
     p->kernel = MKV_KERNEL_AUTO;
 }
 
+// the parameters of the context that serves the first full_layers layers: a cache that holds max_tokens
+static mkv_params full_layer_params(const mkv_params *p)
+{
+    mkv_params c = *p;
+    c.layers = p->full_layers;
+    c.full_layers = 0;
+    c.max_tokens = 0;
+    c.C = p->max_tokens - p->R;
+    c.evict_interval = 1;
+    c.workspace = nullptr;
+    c.workspace_bytes = 0;
+    return c;
+}
+
 size_t mkv_workspace_bytes(const mkv_params *p)
 {
     if (!params_valid(p)) return 0;
     Shape s;
     KernelKind kind;
     if (!resolve(p, &s, &kind)) return 0;
-    return make_layout(s).total;
+    size_t total = align256(make_layout(s).total);
+    if (p->full_layers > 0) {
+        const mkv_params c = full_layer_params(p);
+        if (!params_valid(&c) || !resolve(&c, &s, &kind)) return 0;
+        total += align256(make_layout(s).total);
+    }
+    return total;
 }
 
 mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p)
@@ -207,45 +431,27 @@ mkv_status mkv_create_ex(mkv_ctx **out, const mkv_params *p)
     if (!out) return MKV_INVALID_ARG;
     *out = nullptr;
     if (!params_valid(p)) return MKV_INVALID_ARG;
-    Shape s;
-    KernelKind kind;
-    if (!resolve(p, &s, &kind)) return MKV_UNSUPPORTED;
-    const Layout L = make_layout(s);
-    if (p->workspace) {
-        if (((uintptr_t)p->workspace & 255) != 0) return MKV_INVALID_ARG;
-        if (p->workspace_bytes < L.total) return MKV_OOM;
-    }
+    if (p->workspace && ((uintptr_t)p->workspace & 255) != 0) return MKV_INVALID_ARG;
+    const size_t need = mkv_workspace_bytes(p);
+    if (need == 0) return MKV_UNSUPPORTED;
+    if (p->workspace && p->workspace_bytes < need) return MKV_OOM;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
         cudaGetLastError();
         return MKV_CUDA;
     }
-    mkv_ctx *c = new (std::nothrow) mkv_ctx;
-    if (!c) return MKV_OOM;
-    memset(c, 0, sizeof(*c));
-    c->p = *p; c->s = s; c->L = L; c->kind = kind;
-    if (p->workspace) {
-        c->base = (char *)p->workspace;
-    } else {
-        void *mem = nullptr;
-        if (cudaMalloc(&mem, L.total) != cudaSuccess) {
-            cudaGetLastError();
-            delete c;
-            return MKV_OOM;
-        }
-        c->base = (char *)mem;
-        c->owns_workspace = true;
-    }
-    if (kind == kKindTc) {
-        const DecodeArgs a = make_args(c, nullptr, nullptr, nullptr, nullptr);
-        char msg[200] = "";
-        const cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, p->wait_limit_cycles, msg, sizeof(msg));
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            if (c->owns_workspace) cudaFree(c->base);
-            delete c;
-            return e == cudaErrorMemoryAllocation ? MKV_OOM : MKV_CUDA;
-        }
+    Shape s;
+    KernelKind kind;
+    resolve(p, &s, &kind);
+    const size_t own_bytes = align256(make_layout(s).total);
+    mkv_ctx *c = nullptr;
+    mkv_status st = core_create(&c, p, p->workspace, p->workspace ? own_bytes : 0);
+    if (st != MKV_OK) return st;
+    if (p->full_layers > 0) {
+        const mkv_params cp = full_layer_params(p);
+        st = core_create(&c->full, &cp, p->workspace ? (char *)p->workspace + own_bytes : nullptr,
+                         p->workspace ? need - own_bytes : 0);
+        if (st != MKV_OK) { core_destroy(c); return st; }
     }
     *out = c;
     return MKV_OK;
@@ -264,56 +470,37 @@ mkv_status mkv_create(mkv_ctx **out, int layers, int batch, int n_q_heads, int n
 void mkv_destroy(mkv_ctx *ctx)
 {
     if (!ctx) return;
-    if (ctx->plan) tc_plan_destroy(ctx->plan);
-    if (ctx->prefill_scratch.ptr) cudaFree(ctx->prefill_scratch.ptr);
-    if (ctx->owns_workspace && ctx->base) cudaFree(ctx->base);
-    delete ctx;
+    core_destroy(ctx->full);
+    core_destroy(ctx);
+}
+
+static mkv_status prefill_any(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, void *stream,
+                              bool use_static, const char *who)
+{
+    if (!ctx) return MKV_INVALID_ARG;
+    if (!k || !v || !q_window) return fail(ctx, MKV_INVALID_ARG, "%s: NULL tensor", who);
+    if (prompt_len < 1 || prompt_len > (1 << 24)) return fail(ctx, MKV_INVALID_ARG, "%s: prompt_len out of range", who);
+    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "%s: context already holds a sequence", who);
+    const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
+    size_t off_kv = 0, off_q = 0;
+    if (ctx->full) {
+        if (prompt_len > ctx->p.max_tokens) return fail(ctx, MKV_INVALID_ARG, "%s: the prompt is longer than max_tokens", who);
+        const mkv_status st = core_prefill(ctx->full, k, v, q_window, prompt_len, (cudaStream_t)stream, use_static, who);
+        if (st != MKV_OK) { snprintf(ctx->err, sizeof(ctx->err), "%s", ctx->full->err); return st; }
+        off_kv = kv_bytes_per_layer(ctx) * prompt_len * ctx->p.full_layers;
+        off_q = q_bytes_per_layer(ctx) * Rw * ctx->p.full_layers;
+    }
+    return core_prefill(ctx, off(k, off_kv), off(v, off_kv), off(q_window, off_q), prompt_len, (cudaStream_t)stream, use_static, who);
 }
 
 mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, void *stream)
 {
-    if (!ctx) return MKV_INVALID_ARG;
-    if (!k || !v || !q_window) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill: NULL tensor%s");
-    if (prompt_len < 1 || prompt_len > (1 << 24)) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill: prompt_len out of range%s");
-    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill: context already holds a sequence%s");
-    const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
-    if (!clear_arena(ctx, (cudaStream_t)stream)) return fail(ctx, MKV_CUDA, "mkv_prefill: clearing the arena failed%s");
-    const cudaError_t e = run_prefill(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, k, v, q_window, prompt_len,
-                                      (cudaStream_t)stream, &ctx->launches, &ctx->prefill_scratch);
-    if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(ctx, MKV_OOM, "mkv_prefill: no memory for scratch%s"); }
-    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_prefill: %s", cudaGetErrorString(e));
-    const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
-    ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
-    ctx->t = prompt_len;
-    ctx->steps = 0;
-    ctx->prefilled = true;
-    return MKV_OK;
+    return prefill_any(ctx, k, v, q_window, prompt_len, stream, false, "mkv_prefill");
 }
 
 mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, void *stream)
 {
-    if (!ctx) return MKV_INVALID_ARG;
-    if (!k || !v || !q_window) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_static: NULL tensor%s");
-    if (prompt_len < 1 || prompt_len > (1 << 24)) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_static: prompt_len out of range%s");
-    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill_static: context already holds a sequence%s");
-    const int Rw = prompt_len < ctx->s.R ? prompt_len : ctx->s.R;
-    const size_t need = ((size_t)Rw * ctx->s.G + 1) * (size_t)prompt_len;
-    if (need > prefill_static_max_floats()) {
-        snprintf(ctx->err, sizeof(ctx->err),
-                 "mkv_prefill_static: one unit needs (min(R,P)*G + 1) * prompt_len = %zu floats of scratch, the fixed "
-                 "array holds %zu; use mkv_prefill for this prompt", need, prefill_static_max_floats());
-        return MKV_UNSUPPORTED;
-    }
-    const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
-    if (!clear_arena(ctx, (cudaStream_t)stream)) return fail(ctx, MKV_CUDA, "mkv_prefill_static: clearing the arena failed%s");
-    const cudaError_t e = run_prefill_static(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, k, v, q_window, prompt_len,
-                                             (cudaStream_t)stream, &ctx->launches);
-    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_prefill_static: %s", cudaGetErrorString(e));
-    ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
-    ctx->t = prompt_len;
-    ctx->steps = 0;
-    ctx->prefilled = true;
-    return MKV_OK;
+    return prefill_any(ctx, k, v, q_window, prompt_len, stream, true, "mkv_prefill_static");
 }
 
 mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *out, void *stream)
@@ -321,8 +508,39 @@ mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const
     if (!ctx) return MKV_INVALID_ARG;
     if (!q || !k_new || !v_new || !out) return fail(ctx, MKV_INVALID_ARG, "mkv_decode_step: NULL tensor%s");
     if (!ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_decode_step: call mkv_prefill first%s");
+    if (ctx->cursor != 0)
+        return fail(ctx, MKV_BAD_STATE, "mkv_decode_step: a step begun with mkv_decode_step_layer has layers left%s");
     if (ctx->t >= 0x7fffffffLL) return fail(ctx, MKV_UNSUPPORTED, "mkv_decode_step: position exceeds int32%s");
-    return launch_step(ctx, q, k_new, v_new, out, (cudaStream_t)stream);
+    size_t oq = 0, okv = 0;
+    if (ctx->full) {
+        const mkv_status st = launch_step(ctx->full, -1, q, k_new, v_new, out, (cudaStream_t)stream);
+        if (st != MKV_OK) { snprintf(ctx->err, sizeof(ctx->err), "%s", ctx->full->err); return st; }
+        oq = q_bytes_per_layer(ctx) * ctx->p.full_layers;
+        okv = kv_bytes_per_layer(ctx) * ctx->p.full_layers;
+    }
+    return launch_step(ctx, -1, off(q, oq), off(k_new, okv), off(v_new, okv), (char *)out + oq, (cudaStream_t)stream);
+}
+
+mkv_status mkv_decode_step_layer(mkv_ctx *ctx, int layer, const void *q, const void *k_new, const void *v_new, void *out,
+                                 void *stream)
+{
+    if (!ctx) return MKV_INVALID_ARG;
+    if (!q || !k_new || !v_new || !out) return fail(ctx, MKV_INVALID_ARG, "mkv_decode_step_layer: NULL tensor%s");
+    if (!ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_decode_step_layer: call mkv_prefill first%s");
+    if (layer < 0 || layer >= ctx->p.layers) return fail(ctx, MKV_INVALID_ARG, "mkv_decode_step_layer: layer out of range%s");
+    if (ctx->t >= 0x7fffffffLL) return fail(ctx, MKV_UNSUPPORTED, "mkv_decode_step_layer: position exceeds int32%s");
+    // the layers of a step come in order 0, 1, ..., layers - 1
+    const int fl = ctx->p.full_layers;
+    if (layer != ctx->cursor) return fail(ctx, MKV_BAD_STATE, "mkv_decode_step_layer: layers must be called in order within a step%s");
+    mkv_status st;
+    if (layer < fl) {
+        st = launch_step(ctx->full, layer, q, k_new, v_new, out, (cudaStream_t)stream);
+        if (st != MKV_OK) snprintf(ctx->err, sizeof(ctx->err), "%s", ctx->full->err);
+    } else {
+        st = launch_step(ctx, layer - fl, q, k_new, v_new, out, (cudaStream_t)stream);
+    }
+    if (st == MKV_OK) ctx->cursor = layer + 1 < ctx->p.layers ? layer + 1 : 0;
+    return st;
 }
 
 mkv_status mkv_decode_steps(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *out, int n_steps,
@@ -330,7 +548,7 @@ mkv_status mkv_decode_steps(mkv_ctx *ctx, const void *q, const void *k_new, cons
 {
     if (!ctx) return MKV_INVALID_ARG;
     if (n_steps < 0) return fail(ctx, MKV_INVALID_ARG, "mkv_decode_steps: negative n_steps%s");
-    const size_t qb = (size_t)ctx->s.U * ctx->s.G * ctx->s.D * ctx->s.es, kb = (size_t)ctx->s.U * ctx->s.D * ctx->s.es;
+    const size_t qb = q_bytes_per_layer(ctx) * ctx->p.layers, kb = kv_bytes_per_layer(ctx) * ctx->p.layers;
     for (int i = 0; i < n_steps; ++i) {
         const mkv_status st = mkv_decode_step(ctx, (const char *)q + i * qb, (const char *)k_new + i * kb,
                                               (const char *)v_new + i * kb, (char *)out + i * qb, stream);
@@ -345,6 +563,7 @@ mkv_status mkv_decode_step_host(mkv_ctx *ctx, const void *q_host, const void *k_
     if (!ctx) return MKV_INVALID_ARG;
     if (!q_host || !k_new_host || !v_new_host || !out_host) return fail(ctx, MKV_INVALID_ARG, "mkv_decode_step_host: NULL buffer%s");
     if (!ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_decode_step_host: call mkv_prefill first%s");
+    if (ctx->full) return fail(ctx, MKV_UNSUPPORTED, "mkv_decode_step_host: not available with full_layers; copy the inputs and call mkv_decode_step%s");
     cudaStream_t s = (cudaStream_t)stream;
     const size_t qb = (size_t)ctx->s.U * ctx->s.G * ctx->s.D * ctx->s.es, kb = (size_t)ctx->s.U * ctx->s.D * ctx->s.es;
     char *b = ctx->base;
@@ -379,46 +598,24 @@ mkv_status mkv_cache_view(mkv_ctx *ctx, int layer, mkv_view *view)
 {
     if (!ctx || !view) return MKV_INVALID_ARG;
     if (layer < 0 || layer >= ctx->p.layers) return fail(ctx, MKV_INVALID_ARG, "mkv_cache_view: layer out of range%s");
-    const size_t upl = (size_t)ctx->p.batch * ctx->p.n_kv_heads, u0 = upl * layer;
-    const Shape &s = ctx->s;
-    char *b = ctx->base;
-    view->K = b + ctx->L.K + u0 * s.cap * s.D * s.es;
-    view->V = b + ctx->L.V + u0 * s.cap * s.D * s.es;
-    view->pos = (int32_t *)(b + ctx->L.pos) + u0 * s.cap;
-    view->F = (float *)(b + ctx->L.F) + u0 * s.cap;
-    view->evicted_pos = (int32_t *)(b + ctx->L.evicted) + u0;
-    view->ring_q = b + ctx->L.ring_q + u0 * s.R * s.G * s.D * s.es;
-    view->ring_c = (float *)(b + ctx->L.ring_c) + u0 * s.R * s.G;
-    view->count = ctx->n;
-    view->capacity = s.cap;
-    view->next_pos = ctx->t;
+    if (layer < ctx->p.full_layers) core_view(ctx->full, layer, view);
+    else core_view(ctx, layer - ctx->p.full_layers, view);
     return MKV_OK;
 }
 
 mkv_status mkv_sync(mkv_ctx *ctx, void *stream)
 {
     if (!ctx) return MKV_INVALID_ARG;
-    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
-    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e));
-    DevState st;
-    e = cudaMemcpy(&st, ctx->base + ctx->L.state, sizeof(st), cudaMemcpyDeviceToHost);
-    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e));
-    if (st.err == kErrCacheOverflow)
-        return fail(ctx, MKV_BAD_STATE, "a decode step found no free slot: coarse-grained eviction ran out of step%s");
-    if (st.err != kErrNone) {
-        char code[32];
-        snprintf(code, sizeof(code), " (wait code %d)", st.err);
-        return fail(ctx, MKV_DEVICE_TIMEOUT, "a device-side wait ran out of iterations%s", code);
+    if (ctx->full) {
+        const mkv_status st = core_sync(ctx->full, (cudaStream_t)stream);
+        if (st != MKV_OK) { snprintf(ctx->err, sizeof(ctx->err), "%s", ctx->full->err); return st; }
     }
-    // the device-resident state is authoritative (steps replayed from a CUDA graph advance
-    // it without passing through this library); the host mirror follows it
-    if (ctx->prefilled) { ctx->t = st.t; ctx->n = st.n; ctx->steps = st.steps; }
-    return MKV_OK;
+    return core_sync(ctx, (cudaStream_t)stream);
 }
 
 const char *mkv_last_error(const mkv_ctx *ctx) { return ctx ? ctx->err : ""; }
 
-uint64_t mkv_launch_count(const mkv_ctx *ctx) { return ctx ? ctx->launches : 0; }
+uint64_t mkv_launch_count(const mkv_ctx *ctx) { return ctx ? ctx->launches + (ctx->full ? ctx->full->launches : 0) : 0; }
 
 const char *mkv_kernel_name(const mkv_ctx *ctx) { return (ctx && ctx->kind == kKindTc) ? "tc" : "simt"; }
 

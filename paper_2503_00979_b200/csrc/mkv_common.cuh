@@ -43,7 +43,9 @@ struct DecodeArgs {
     float *part_o;             // [U][splits][G][D]  un-normalised split outputs
     int *ticket;               // [U]
     int *evicted_pos;          // [U]
-    DevState *st;
+    DevState *st;              // the step state this launch reads and advances
+    int u0;                    // index of this launch's first unit in the context's arena (per-layer launches): the
+                               // pointers above are already offset by it, tensor-map coordinates are not
     int U, G, R, C, cap, splits, fusion, T;
     float scale2;              // log2(e) / sqrt(D)
 };

@@ -26,9 +26,9 @@ cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int grid, unsigne
 void tc_plan_destroy(TcPlan *plan);
 cudaError_t launch_decode_tc(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream);
 
-// Prompt phase: fills the arena (K, V, pos, ring) and the step state from a prompt of P
+// Prompt phase: fills the arena (K, V, pos, ring) and the n_states step states at a.st from a prompt of P
 // tokens.  `a` supplies the arena pointers and shape; q/k_new/v_new/out are ignored.
-// Allocates and frees its own temporary scratch.  *launches is advanced per kernel launched.
+// *launches is advanced per kernel launched.
 // Device scratch of the prompt phase, owned by the context (allocated on first use, grown when a
 // longer prompt needs more, released with the context).
 struct PrefillScratch {
@@ -36,13 +36,17 @@ struct PrefillScratch {
     size_t bytes;
 };
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
-                        int P, cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch);
+                        int P, cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states);
 
 // The same prompt phase with its scratch in a fixed device array of prefill_static_max_floats()
 // floats instead of a temporary allocation; cudaErrorInvalidConfiguration if one unit's
 // (R*G + 1) * P floats do not fit.
 size_t prefill_static_max_floats();
 cudaError_t run_prefill_static(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
-                               int P, cudaStream_t stream, unsigned long long *launches);
+                               int P, cudaStream_t stream, unsigned long long *launches, int device, int n_states);
+
+// Copies one step state over n_dst others (the whole-stack state and the per-layer states are brought level when
+// a context switches between whole-stack and per-layer calls).
+cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream);
 
 }  // namespace mkv

@@ -6,6 +6,8 @@
 // older prompt token gets the fused score of Eq. 4-6 (group sum first), and the C best are
 // kept beside the window (Eq. 7).  The selection is a block-wide radix select over
 // (score, position) keys, so ties keep the lower position deterministically.
+#include <mutex>
+
 #include "mkv_common.cuh"
 #include "mkv_kernels.h"
 
@@ -38,9 +40,12 @@ __global__ void init_arena_kernel(DecodeArgs a)
     if (i < (size_t)a.U) { a.ticket[i] = 0; a.evicted_pos[i] = -1; }
 }
 
-__global__ void set_state_kernel(DevState *st, long long t, int n)
+// the whole-stack state and one state per layer (per-layer calls advance their own)
+__global__ void set_state_kernel(DevState *st, int n_states, long long t, int n)
 {
-    st->t = t; st->n = n; st->steps = 0; st->err = 0; st->done = 0; st->compact = 0;
+    for (int i = threadIdx.x; i < n_states; i += blockDim.x) {
+        st[i].t = t; st[i].n = n; st[i].steps = 0; st[i].err = 0; st[i].done = 0; st[i].compact = 0;
+    }
 }
 
 // S[ub][row = i*G + g][j] = log2-domain logit of window row (i, g) against prompt key j,
@@ -255,38 +260,27 @@ __global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, in
     }
 }
 
+// The prompt phase on a scratch area of `scratch_floats` floats (the window-row logits S and the fused scores of
+// as many units as fit go through it, batch after batch).  Every element a kernel reads was written earlier in the
+// same batch, so what the area held before never matters.
 template <typename T, int D>
 cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
-                          unsigned long long *launches, PrefillScratch *scratch)
+                          unsigned long long *launches, float *S, size_t scratch_floats, int n_states)
 {
     const int U = a.U, G = a.G, R = a.R, C = a.C;
     const int Rw = P < R ? P : R, rows = Rw * G;
     const bool select = P - Rw > C;
     const int n = select ? C + Rw : P;
     if (n > a.cap) return cudaErrorInvalidValue;
-
-    const size_t per_unit = ((size_t)rows * P + P) * sizeof(float);
-    size_t ub = ((size_t)1 << 30) / per_unit;
-    if (ub < 1) ub = 1;
+    const size_t per_unit = (size_t)rows * P + P;            // floats
+    if (per_unit > scratch_floats) return cudaErrorInvalidConfiguration;
+    size_t ub = scratch_floats / per_unit;
     if (ub > (size_t)U) ub = U;
     if (ub > 65535) ub = 65535;
-    // The scratch belongs to the context and is kept until the context is destroyed: it only grows.
-    // (Allocating and freeing it around every prompt put a cudaFree of up to 1 GiB right in front
-    // of the first decode launches.)
-    cudaError_t e = cudaSuccess;
-    if (scratch->bytes < ub * per_unit) {
-        if (scratch->ptr) cudaFree(scratch->ptr);
-        scratch->ptr = nullptr;
-        scratch->bytes = 0;
-        e = cudaMalloc(&scratch->ptr, ub * per_unit);
-        if (e != cudaSuccess) { scratch->ptr = nullptr; return e; }
-        scratch->bytes = ub * per_unit;
-    }
-    float *S = static_cast<float *>(scratch->ptr);
     float *Fp = S + ub * (size_t)rows * P;
 
     const size_t logits_smem = (size_t)(kPK * (D + 4) + kPR * (D + 4) + kPK * (kPR + 1)) * sizeof(float);
-    e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
+    cudaError_t e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
     if (e != cudaSuccess) return e;
     const size_t init_n = max((size_t)U * a.cap, (size_t)U * R * G);
     init_arena_kernel<<<(unsigned)((init_n + 255) / 256), 256, 0, stream>>>(a);
@@ -311,32 +305,47 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     constexpr int CH = D * sizeof(T) / 16;
     prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
     prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
-    set_state_kernel<<<1, 1, 0, stream>>>(a.st, (long long)P, n);
+    set_state_kernel<<<1, 32, 0, stream>>>(a.st, n_states, (long long)P, n);
     *launches += 3;
     e = cudaGetLastError();
     const cudaError_t e2 = cudaStreamSynchronize(stream);
     return e != cudaSuccess ? e : e2;
 }
 
+cudaError_t dispatch_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
+                             cudaStream_t stream, unsigned long long *launches, float *S, size_t scratch_floats, int n_states)
+{
+    if (f32) {
+        auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
+        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states)
+                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states);
+    }
+    auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
+         qq = static_cast<const __nv_bfloat16 *>(q_window);
+    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states)
+                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states);
+}
 
-// ---- prompt phase without any allocation ---------------------------------------------------
-// Scratch for the logits table S and the fused scores lives in a fixed device array that every
-// GPU loading this library holds until the process exits.  16 MiB: one unit of a 4096-token
-// prompt with R*G = 128 window rows needs 2.1 MB, so the units go through it a few at a time.
+// ---- scratch of mkv_prefill_static -------------------------------------------------------------------------
+// A fixed device array that every GPU loading this library holds until the process exits.  16 MiB: one unit of a
+// 4096-token prompt with R*G = 128 window rows needs 2.1 MB, so the units go through it a few at a time.
 constexpr size_t kStaticScratchFloats = (size_t)4 << 20;
 static __device__ __align__(256) float g_prefill_scratch[kStaticScratchFloats];
 
 constexpr int kMaxDevices = 64;
 static float *g_scratch_addr[kMaxDevices];   // device address of the array, per device ordinal
+static std::mutex g_scratch_mutex;
 
-// The array's name is only a host-side handle here; a kernel needs its device address, which
-// the runtime hands out per device.  Looked up once per device, with that device current.
-cudaError_t static_scratch_address(float **out)
+// The array's name is only a host-side handle here; a kernel needs its device address, which the runtime hands out
+// per device.  Looked up once per device, with that device current.
+cudaError_t static_scratch_address(int device, float **out)
 {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (dev != device) return cudaErrorInvalidDevice;          // the context lives on another device than the current one
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
     if (!g_scratch_addr[dev]) {
         float *ptr = nullptr;
         e = cudaGetSymbolAddress((void **)&ptr, g_prefill_scratch);
@@ -347,93 +356,56 @@ cudaError_t static_scratch_address(float **out)
     return cudaSuccess;
 }
 
-template <typename T, int D>
-cudaError_t run_prefill_static_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
-                                 unsigned long long *launches)
-{
-    const int U = a.U, G = a.G, R = a.R, C = a.C;
-    const int Rw = P < R ? P : R, rows = Rw * G;
-    const bool select = P - Rw > C;
-    const int n = select ? C + Rw : P;
-    if (n > a.cap) return cudaErrorInvalidValue;
-    const size_t per_unit = (size_t)rows * P + P;            // floats
-    if (per_unit > kStaticScratchFloats) return cudaErrorInvalidConfiguration;
-    size_t ub = kStaticScratchFloats / per_unit;
-    if (ub > (size_t)U) ub = U;
-    if (ub > 65535) ub = 65535;
-    float *S = nullptr;
-    cudaError_t e = static_scratch_address(&S);
-    if (e != cudaSuccess) return e;
-    // every element of S and Fp that a kernel reads was written earlier in the same batch,
-    // so what an earlier call left in the array never matters and nothing has to be cleared
-    float *Fp = S + ub * (size_t)rows * P;
-    const size_t logits_smem = (size_t)(kPK * (D + 4) + kPR * (D + 4) + kPK * (kPR + 1)) * sizeof(float);
-    e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
-    if (e != cudaSuccess) return e;
-    const size_t init_n = max((size_t)U * a.cap, (size_t)U * R * G);
-    init_arena_kernel<<<(unsigned)((init_n + 255) / 256), 256, 0, stream>>>(a);
-    ++*launches;
-    for (int ub0 = 0; ub0 < U; ub0 += (int)ub) {
-        const int nb = min((int)ub, U - ub0);
-        prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw, G,
-                                                                                             a.scale2);
-        prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, G, R);
-        *launches += 2;
-        if (select) {
-            prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
-                S, a.ring_c, Fp, ub0, P, Rw, G, R, a.fusion);
-            prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
-            *launches += 2;
-        }
-    }
-    if (!select) {
-        prefill_identity_pos_kernel<<<(unsigned)(((size_t)U * n + 255) / 256), 256, 0, stream>>>(a.pos, U, n, a.cap);
-        ++*launches;
-    }
-    constexpr int CH = D * sizeof(T) / 16;
-    prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
-    prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
-    set_state_kernel<<<1, 1, 0, stream>>>(a.st, (long long)P, n);
-    *launches += 3;
-    e = cudaGetLastError();
-    const cudaError_t e2 = cudaStreamSynchronize(stream);
-    return e != cudaSuccess ? e : e2;
-}
-
 }  // namespace
 
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
-                        cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch)
+                        cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states)
 {
-    if (f32) {
-        auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
-        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches, scratch)
-                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches, scratch);
+    const int Rw = P < a.R ? P : a.R;
+    const size_t per_unit = ((size_t)Rw * a.G * P + P) * sizeof(float);
+    size_t ub = ((size_t)1 << 30) / per_unit;
+    if (ub < 1) ub = 1;
+    if (ub > (size_t)a.U) ub = a.U;
+    if (ub > 65535) ub = 65535;
+    // The scratch belongs to the context and is kept until the context is destroyed: it only grows.
+    // (Allocating and freeing it around every prompt put a cudaFree of up to 1 GiB right in front
+    // of the first decode launches.)
+    if (scratch->bytes < ub * per_unit) {
+        if (scratch->ptr) cudaFree(scratch->ptr);
+        scratch->ptr = nullptr;
+        scratch->bytes = 0;
+        const cudaError_t e = cudaMalloc(&scratch->ptr, ub * per_unit);
+        if (e != cudaSuccess) { scratch->ptr = nullptr; return e; }
+        scratch->bytes = ub * per_unit;
     }
-    auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
-         qq = static_cast<const __nv_bfloat16 *>(q_window);
-    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches, scratch)
-                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches, scratch);
+    return dispatch_prefill(a, f32, D, k, v, q_window, P, stream, launches, static_cast<float *>(scratch->ptr),
+                            scratch->bytes / sizeof(float), n_states);
 }
 
-}  // namespace mkv
+namespace {
+__global__ void copy_state_kernel(DevState *dst, int n_dst, const DevState *src)
+{
+    const DevState s = *src;
+    __syncthreads();            // src may be one of the destinations
+    for (int i = threadIdx.x; i < n_dst; i += blockDim.x) { dst[i] = s; dst[i].done = 0; }
+}
+}  // namespace
 
-namespace mkv {
+cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream)
+{
+    copy_state_kernel<<<1, 64, 0, stream>>>(dst, n_dst, src);
+    return cudaGetLastError();
+}
 
 size_t prefill_static_max_floats() { return kStaticScratchFloats; }
 
 cudaError_t run_prefill_static(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
-                               int P, cudaStream_t stream, unsigned long long *launches)
+                               int P, cudaStream_t stream, unsigned long long *launches, int device, int n_states)
 {
-    if (f32) {
-        auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
-        return D == 64 ? run_prefill_static_t<float, 64>(a, kk, vv, qq, P, stream, launches)
-                       : run_prefill_static_t<float, 128>(a, kk, vv, qq, P, stream, launches);
-    }
-    auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
-         qq = static_cast<const __nv_bfloat16 *>(q_window);
-    return D == 64 ? run_prefill_static_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches)
-                   : run_prefill_static_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches);
+    float *S = nullptr;
+    const cudaError_t e = static_scratch_address(device, &S);
+    if (e != cudaSuccess) return e;
+    return dispatch_prefill(a, f32, D, k, v, q_window, P, stream, launches, S, kStaticScratchFloats, n_states);
 }
 
 }  // namespace mkv

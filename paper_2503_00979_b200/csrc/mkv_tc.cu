@@ -673,8 +673,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag, kWaitQEmpty, WL);
                 if (!ok) break;
                 mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
-                tma_load_3d(q_addr, &tmQ, 0, 0, x.unit, bar_qfull, pol_keep);
-                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, x.unit, bar_qfull, pol_keep);
+                tma_load_3d(q_addr, &tmQ, 0, 0, a.u0 + x.unit, bar_qfull, pol_keep);
+                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, a.u0 + x.unit, bar_qfull, pol_keep);
                 ++rings;
                 for (int j = 0; j < x.nk && ok; ++j, rk.step(1, SK)) {
                     const int T = w.T0 + j, s = rk.idx;
@@ -682,8 +682,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_kfull + 8 * s, kStageBytes);
-                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, x.unit, bar_kfull + 8 * s, pol_stream);
-                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, x.unit, bar_kfull + 8 * s, pol_stream);
+                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, a.u0 + x.unit, bar_kfull + 8 * s, pol_stream);
+                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, a.u0 + x.unit, bar_kfull + 8 * s, pol_stream);
                     issued = T + 1;
                 }
                 w.advance(x);
@@ -714,8 +714,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_vfull + 8 * s, kStageBytes);
-                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, x.unit, bar_vfull + 8 * s, pol_stream);
-                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, x.unit, bar_vfull + 8 * s, pol_stream);
+                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, a.u0 + x.unit, bar_vfull + 8 * s, pol_stream);
+                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, a.u0 + x.unit, bar_vfull + 8 * s, pol_stream);
                     issued = T + 1;
                 }
                 w.advance(x);

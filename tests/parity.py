@@ -110,7 +110,8 @@ def oracle_unit_following(make_unit, k, v, qw, device_positions, where: str):
 
 def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chunk: int = 32, kernel: str = "auto",
                splits: int = 0, check_F_every: int = 16, device: str = "cuda:0", use_steps_call: bool = False,
-               host_call_every: int = 0, host_pinned: bool = True, synth_device=None, **ctx_kwargs) -> ParityReport:
+               host_call_every: int = 0, host_pinned: bool = True, synth_device=None, per_layer: int = 0,
+               full_layers: int = 0, max_tokens: int = 0, **ctx_kwargs) -> ParityReport:
     """Prefill + `steps` decode steps of workload `w` on the device, followed by the oracle on `units`.
 
     The steps of a chunk are enqueued without a synchronisation in between (the evicted positions of the
@@ -118,6 +119,10 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     use_steps_call   one mkv_decode_steps call per chunk (no per-step evicted positions: outputs are compared on
                      every step, retained sets at the end of each chunk unless the oracle saw a near tie in it).
     synth_device     where the inputs are drawn ("cpu" keeps the drawing's many small kernels off the GPU).
+    per_layer        1: every step is made of mkv_decode_step_layer calls, layer by layer; 2: steps alternate between
+                     one whole-stack call and per-layer calls.
+    full_layers, max_tokens   layer-aware variant: the first full_layers layers keep every token (the oracle units of
+                     those layers get C = max_tokens - R, so they never evict within max_tokens).
     """
     dev = torch.device(device)
     st = _DeviceStream(w, synth_device or dev, dev)
@@ -126,8 +131,9 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     units = units or pick_units(w, n_units)
     rep = ParityReport()
     mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, d, C_, R, w.fusion, w.dtype, kernel=kernel,
-                         splits=splits, device=device, **ctx_kwargs)
+                         splits=splits, device=device, full_layers=full_layers, max_tokens=max_tokens, **ctx_kwargs)
     rep.kernel = mk.kernel_name
+    C_of = {l: (max_tokens - R if l < full_layers else C_) for l in range(w.layers)}     # distant tokens kept per layer
     tol = TOL_OUT[w.dtype]
     Rw = min(R, P)
     pool = ThreadPoolExecutor(max_workers=_workers())
@@ -151,13 +157,13 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     mk.prefill(k_all, v_all, qw_all)
     mk.sync()
     views = {l: mk.view(l) for l in by_layer}
-    count0 = views[units[0][0]]["count"]
-    dev_pos = {(l, b, h): views[l]["pos"][b, h, :count0].cpu().numpy() for (l, b, h) in units}
+    count0 = {l: views[l]["count"] for l in by_layer}
+    dev_pos = {(l, b, h): views[l]["pos"][b, h, :count0[l]].cpu().numpy() for (l, b, h) in units}
 
     def prefill_unit(key):
         kp, vp, qp = prompt[key]
-        u, resync = oracle_unit_following(lambda: ora.Unit(G, d, C_, R, w.fusion), kp, vp, qp, dev_pos[key], f"unit {key}")
-        assert count0 == u.count, (count0, u.count)
+        u, resync = oracle_unit_following(lambda: ora.Unit(G, d, C_of[key[0]], R, w.fusion), kp, vp, qp, dev_pos[key], f"unit {key}")
+        assert count0[key[0]] == u.count, (count0[key[0]], u.count)
         return key, u, resync
 
     orac = {}
@@ -167,8 +173,8 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     # K rows must be the prompt rows of those positions, bit for bit
     for (l, b, h) in units:
         gp = torch.from_numpy(dev_pos[(l, b, h)]).long().to(dev)
-        assert torch.equal(views[l]["K"][b, h, :count0], k_all[l, b, h][gp]), f"unit {(l, b, h)}: K rows differ from the prompt's"
-        assert torch.equal(views[l]["V"][b, h, :count0], v_all[l, b, h][gp]), f"unit {(l, b, h)}: V rows differ from the prompt's"
+        assert torch.equal(views[l]["K"][b, h, :count0[l]], k_all[l, b, h][gp]), f"unit {(l, b, h)}: K rows differ from the prompt's"
+        assert torch.equal(views[l]["V"][b, h, :count0[l]], v_all[l, b, h][gp]), f"unit {(l, b, h)}: V rows differ from the prompt's"
     del k_all, v_all, qw_all, prompt
     rep.units = len(orac)
     layers_checked = sorted(by_layer)
@@ -203,6 +209,9 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
                     mk.decode_step_host(qh, kh, vh, oh)
                     torch.cuda.current_stream().synchronize()
                     outs[i].copy_(oh)
+                elif per_layer == 1 or (per_layer == 2 and (done + i) % 2 == 1):
+                    for l in range(w.layers):
+                        mk.decode_step_layer(l, qs[i, l], ks[i, l], vs[i, l], outs[i, l])
                 else:
                     mk.decode_step(qs[i], ks[i], vs[i], outs[i])
                 # evicted positions of the checked units, gathered on the stream
@@ -222,6 +231,7 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
         def follow(ui):
             key = units[ui]
             u = orac[key]
+            C_ = C_of[key[0]]
             r = dict(err=0.0, evictions=0, resyncs=0, Fmax=0.0, Fcmp=0, gap=float("inf"))
             for i in range(ns):
                 t = t0 + i

@@ -387,6 +387,89 @@ def test_config1_all_units_prompt_phase_and_first_steps_against_the_oracle():
     assert rep.prefill_resyncs <= 2
 
 
+# ---- per-layer entry (a model that runs its layers one after the other) and the layer-aware variant
+@pytest.mark.parametrize("kernel,dtype,d", [("tc", "bf16", 128), ("simt", "f32", 64)])
+@pytest.mark.parametrize("mode", [1, 2])
+def test_per_layer_calls_against_the_oracle(kernel, dtype, d, mode):
+    # mode 1: every step layer by layer; mode 2: whole-stack and per-layer steps alternate in one context
+    w = SMALL.replace(layers=3, batch=2, head_dim=d, dtype=dtype, C=600, R=16, prompt_len=700, steps=40, fusion="max")
+    rep = run_parity(w, steps=w.steps, n_units=6, kernel=kernel, per_layer=mode)
+    _report(rep)
+    assert rep.kernel == kernel and rep.evictions == 6 * 40 and rep.F_compared > 0
+
+
+def test_per_layer_calls_give_the_whole_stack_results():
+    # config 1's shape on four layers: a step made of per-layer calls against the same step as one call.  The two
+    # cut a unit's tiles into different ranges, so outputs agree to rounding, evictions exactly.
+    w = synth.WORKLOADS["c1"].replace(layers=4, steps=24)
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    P = w.prompt_len
+    k, v = st.kv(np.arange(P))
+    qw = st.q(np.arange(P - w.R, P))
+    pos = np.arange(P, P + w.steps)
+    kk, vv = st.kv(pos)
+    qn = st.q(pos).permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    kn = kk.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    vn = vv.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    res = []
+    for per_layer in (False, True):
+        mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype)
+        mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+        out = torch.empty_like(qn)
+        ev = []
+        for i in range(w.steps):
+            if per_layer:
+                for l in range(w.layers):
+                    mk.decode_step_layer(l, qn[i, l], kn[i, l], vn[i, l], out[i, l])
+            else:
+                mk.decode_step(qn[i], kn[i], vn[i], out[i])
+            ev.append(torch.stack([mk.view(l)["evicted_pos"].clone() for l in range(w.layers)]))
+        mk.sync()
+        assert mk.view(0)["next_pos"] == P + w.steps
+        res.append((out.float(), torch.stack(ev), torch.stack([torch.sort(mk.view(l)["pos"], dim=-1).values for l in range(w.layers)])))
+        mk.close()
+    assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+    assert ((res[0][0] - res[1][0]).abs() <= 2 ** -7 * res[0][0].abs() + 1e-3).all()
+
+
+def test_per_layer_calls_must_come_in_order():
+    w = SMALL.replace(layers=3, batch=1, steps=1)
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    k, v = st.kv(np.arange(w.prompt_len))
+    qw = st.q(np.arange(w.prompt_len - w.R, w.prompt_len))
+    mk = binding.MorphKV(3, 1, 8, 2, 128, w.C, w.R, w.fusion, "bf16")
+    mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+    q = torch.zeros(1, 8, 128, dtype=torch.bfloat16, device=dev)
+    kv = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device=dev)
+    qa = torch.zeros(3, 1, 8, 128, dtype=torch.bfloat16, device=dev)
+    kva = torch.zeros(3, 1, 2, 128, dtype=torch.bfloat16, device=dev)
+    assert binding.mkv_decode_step_layer(mk.ctx, 1, q, kv, kv, q) == binding.BAD_STATE          # layer 0 comes first
+    assert binding.mkv_decode_step_layer(mk.ctx, 3, q, kv, kv, q) == binding.INVALID_ARG
+    assert binding.mkv_decode_step_layer(mk.ctx, 0, q, kv, kv, q) == binding.OK
+    assert binding.mkv_decode_step(mk.ctx, qa, kva, kva, qa) == binding.BAD_STATE                # the step has layers left
+    assert binding.mkv_decode_step_layer(mk.ctx, 0, q, kv, kv, q) == binding.BAD_STATE
+    assert binding.mkv_decode_step_layer(mk.ctx, 1, q, kv, kv, q) == binding.OK
+    assert binding.mkv_decode_step_layer(mk.ctx, 2, q, kv, kv, q) == binding.OK
+    mk.sync()
+    assert mk.view(0)["next_pos"] == w.prompt_len + 1 and mk.view(2)["count"] == mk.view(0)["count"]
+    assert binding.mkv_decode_step(mk.ctx, qa, kva, kva, qa) == binding.OK
+    mk.sync()
+    mk.close()
+
+
+@pytest.mark.parametrize("per_layer", [0, 1])
+def test_layer_aware_variant_first_layers_keep_every_token(per_layer):
+    # MorphKV off for the first two of four layers: their units equal full attention (an oracle unit whose capacity
+    # is never reached), the others evict as usual
+    w = SMALL.replace(layers=4, batch=2, C=250, R=16, prompt_len=320, steps=48, fusion="sum")
+    rep = run_parity(w, steps=w.steps, units=[(0, 0, 0), (1, 1, 1), (2, 0, 1), (3, 1, 0)], per_layer=per_layer,
+                     full_layers=2, max_tokens=400)
+    _report(rep)
+    assert rep.evictions == 2 * 48            # only the two units of the MorphKV layers evict
+
+
 def test_tc_matches_cuda_core_kernel_on_device():
     # the two kernels share only the per-unit epilogue; their outputs must agree closely
     w = SMALL.replace(layers=1, batch=2, C=700, R=32, prompt_len=900, steps=12, fusion="max")
