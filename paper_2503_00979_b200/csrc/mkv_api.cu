@@ -321,6 +321,7 @@ mkv_status core_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *
         ? run_prefill_static(a, f32, ctx->s.D, k, v, q_window, prompt_len, stream, &ctx->launches, ctx->device, n_states)
         : run_prefill(a, f32, ctx->s.D, k, v, q_window, prompt_len, stream, &ctx->launches, &ctx->prefill_scratch, n_states);
     if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(ctx, MKV_OOM, "%s: no memory for scratch", where); }
+    if (e == cudaErrorLaunchTimeout) { cudaGetLastError(); return fail(ctx, MKV_DEVICE_TIMEOUT, "%s: a device-side wait of the prompt phase ran out", where); }
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase: %s", cudaGetErrorString(e));
     ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
     ctx->t = prompt_len;

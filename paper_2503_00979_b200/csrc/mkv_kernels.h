@@ -38,6 +38,14 @@ struct PrefillScratch {
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
                         int P, cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states);
 
+// Tensor-core scoring of the prompt phase (mkv_prefill_tc.cu): two passes over the prompt keys, window-row
+// normalisers into ring_c and fused scores of the older tokens into Fp [nb][P].
+bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P);
+int prefill_tc_splits(int units_in_batch, int P);
+size_t prefill_tc_floats_per_unit(int P, int Rw, int G, int splits);
+cudaError_t run_prefill_scores_tc(const DecodeArgs &a, const void *k, const void *qwin, int P, int ub0, int nb, int splits,
+                                  float *Fp, float *part, int *err, unsigned long long *launches, cudaStream_t stream);
+
 // The same prompt phase with its scratch in a fixed device array of prefill_static_max_floats()
 // floats instead of a temporary allocation; cudaErrorInvalidConfiguration if one unit's
 // (R*G + 1) * P floats do not fit.

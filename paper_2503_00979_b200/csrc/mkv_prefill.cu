@@ -272,12 +272,18 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     const bool select = P - Rw > C;
     const int n = select ? C + Rw : P;
     if (n > a.cap) return cudaErrorInvalidValue;
-    const size_t per_unit = (size_t)rows * P + P;            // floats
-    if (per_unit > scratch_floats) return cudaErrorInvalidConfiguration;
-    size_t ub = scratch_floats / per_unit;
+    // bf16 / head_dim 128 shapes score on the tensor cores (two passes over the keys, no rows x P table); the
+    // others materialise the window-row logits S [rows][P] per unit and reduce them with CUDA-core kernels
+    const bool tc = prefill_tc_supported(sizeof(T) == 4, D, G, R, k, P);
+    const int tc_splits = tc ? prefill_tc_splits(U, P) : 0;
+    const size_t per_unit = tc ? prefill_tc_floats_per_unit(P, Rw, G, tc_splits) : (size_t)rows * P + P;   // floats
+    if (per_unit + 1 > scratch_floats) return cudaErrorInvalidConfiguration;
+    size_t ub = (scratch_floats - 1) / per_unit;
     if (ub > (size_t)U) ub = U;
     if (ub > 65535) ub = 65535;
-    float *Fp = S + ub * (size_t)rows * P;
+    float *Fp = tc ? S : S + ub * (size_t)rows * P;
+    float *part = S + ub * (size_t)P;                          // tensor-core path: pass-1 partials behind the scores
+    int *err_word = reinterpret_cast<int *>(S + scratch_floats - 1);
 
     const size_t logits_smem = (size_t)(kPK * (D + 4) + kPR * (D + 4) + kPK * (kPR + 1)) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(prefill_logits_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)logits_smem);
@@ -285,17 +291,29 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     const size_t init_n = max((size_t)U * a.cap, (size_t)U * R * G);
     init_arena_kernel<<<(unsigned)((init_n + 255) / 256), 256, 0, stream>>>(a);
     ++*launches;
+    if (tc) {
+        e = cudaMemsetAsync(err_word, 0, sizeof(int), stream);
+        if (e != cudaSuccess) return e;
+    }
     for (int ub0 = 0; ub0 < U; ub0 += (int)ub) {
         const int nb = min((int)ub, U - ub0);
-        prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw, G,
-                                                                                             a.scale2);
-        prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, G, R);
-        *launches += 2;
-        if (select) {
-            prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
-                S, a.ring_c, Fp, ub0, P, Rw, G, R, a.fusion);
-            prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
+        if (tc) {
+            e = run_prefill_scores_tc(a, k, qwin, P, ub0, nb, tc_splits, Fp, part, err_word, launches, stream);
+            if (e != cudaSuccess) return e;
+        } else {
+            prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw, G,
+                                                                                                 a.scale2);
+            prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, G, R);
             *launches += 2;
+        }
+        if (select) {
+            if (!tc) {
+                prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
+                    S, a.ring_c, Fp, ub0, P, Rw, G, R, a.fusion);
+                ++*launches;
+            }
+            prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
+            ++*launches;
         }
     }
     if (!select) {
@@ -309,7 +327,14 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     *launches += 3;
     e = cudaGetLastError();
     const cudaError_t e2 = cudaStreamSynchronize(stream);
-    return e != cudaSuccess ? e : e2;
+    if (e != cudaSuccess || e2 != cudaSuccess) return e != cudaSuccess ? e : e2;
+    if (tc) {       // a bounded wait of the scoring kernels that ran out
+        int werr = 0;
+        e = cudaMemcpy(&werr, err_word, sizeof(int), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return e;
+        if (werr != 0) return cudaErrorLaunchTimeout;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t dispatch_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
@@ -362,21 +387,24 @@ cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, con
                         cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states)
 {
     const int Rw = P < a.R ? P : a.R;
-    const size_t per_unit = ((size_t)Rw * a.G * P + P) * sizeof(float);
+    const bool tc = prefill_tc_supported(f32, D, a.G, a.R, k, P);
+    const size_t per_unit = (tc ? prefill_tc_floats_per_unit(P, Rw, a.G, prefill_tc_splits(a.U, P))
+                                : (size_t)Rw * a.G * P + P) * sizeof(float);
     size_t ub = ((size_t)1 << 30) / per_unit;
     if (ub < 1) ub = 1;
     if (ub > (size_t)a.U) ub = a.U;
     if (ub > 65535) ub = 65535;
+    const size_t need = ub * per_unit + sizeof(float);          // + the error word of the scoring kernels
     // The scratch belongs to the context and is kept until the context is destroyed: it only grows.
     // (Allocating and freeing it around every prompt put a cudaFree of up to 1 GiB right in front
     // of the first decode launches.)
-    if (scratch->bytes < ub * per_unit) {
+    if (scratch->bytes < need) {
         if (scratch->ptr) cudaFree(scratch->ptr);
         scratch->ptr = nullptr;
         scratch->bytes = 0;
-        const cudaError_t e = cudaMalloc(&scratch->ptr, ub * per_unit);
+        const cudaError_t e = cudaMalloc(&scratch->ptr, need);
         if (e != cudaSuccess) { scratch->ptr = nullptr; return e; }
-        scratch->bytes = ub * per_unit;
+        scratch->bytes = need;
     }
     return dispatch_prefill(a, f32, D, k, v, q_window, P, stream, launches, static_cast<float *>(scratch->ptr),
                             scratch->bytes / sizeof(float), n_states);
