@@ -142,6 +142,31 @@ class ClockSampler:
                 break
             time.sleep(self.period_s)
 
+    def background(self):
+        """Context manager that samples on a thread of its own (NVML calls release the interpreter lock) while the
+        body runs calls that block the main thread."""
+        sampler = self
+
+        class _Bg:
+            def __enter__(self):
+                self.stop = threading.Event()
+
+                def loop():
+                    while True:
+                        sampler.sample()
+                        if self.stop.wait(sampler.period_s):
+                            break
+
+                self.th = threading.Thread(target=loop, daemon=True)
+                self.th.start()
+                return self
+
+            def __exit__(self, *exc):
+                self.stop.set()
+                self.th.join(timeout=2)
+
+        return _Bg()
+
     def summary(self):
         if not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -297,6 +322,67 @@ def secondary_record(w: synth.Workload, W: int, K: int, dev, per_layer: bool = F
     del qs, kn, vn, outs
     torch.cuda.empty_cache()
     return rec
+
+
+def run_prefill_arm(args, w):
+    """Timed prompt phase: a step is one mkv_prefill call on a P-token prompt (window-row soft-max statistics, fused
+    scores of the older tokens, top-C selection, gather of the kept rows, ring set-up) for every unit; the context
+    is reset between calls.  Inputs are resident in HBM; the call synchronises the stream itself."""
+    from paper_2503_00979_b200 import binding
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1 and int(os.environ.get("RANK", "0")) != 0:
+        return
+    dev = torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', '0'))}")
+    torch.cuda.set_device(dev)
+    tdt = synth.torch_dtype(w.dtype)
+    K, W = args.steps, args.warmup
+    P, Rw = w.prompt_len, min(w.R, w.prompt_len)
+    st = synth.Stream(w, dev)
+    mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
+                         kernel=args.kernel, device=str(dev))
+    k = torch.empty((w.layers, w.batch, w.n_kv_heads, P, w.head_dim), dtype=tdt, device=dev)
+    v = torch.empty_like(k)
+    qw = torch.empty((w.layers, w.batch, w.n_q_heads, Rw, w.head_dim), dtype=tdt, device=dev)
+    chunk = 16384
+    for l in range(w.layers):
+        for p0 in range(0, P, chunk):
+            kk, vv = st.kv(np.arange(p0, min(P, p0 + chunk)), [l])
+            k[l, :, :, p0:p0 + chunk], v[l, :, :, p0:p0 + chunk] = kk[0].to(tdt), vv[0].to(tdt)
+        qw[l] = st.q(np.arange(P - Rw, P), [l])[0].to(tdt)
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    clocks = ClockSampler(dev)
+    for _ in range(W):
+        mk.reset(); mk.prefill(k, v, qw)
+    launches0 = mk.launch_count
+    torch.cuda.synchronize()
+    with clocks.background():
+        e0.record(stream)
+        for _ in range(K):
+            mk.reset(); mk.prefill(k, v, qw)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    n = mk.view(0)["count"]
+    e = 2 if w.dtype == "bf16" else 4
+    # the prompt keys twice (normalisers, then scores) and the K and V rows that are kept
+    bytes_step = w.units * (2 * P * w.head_dim * e + 2 * n * w.head_dim * e)
+    peak, peak_src = measured_peak_gbs()
+    achieved = bytes_step / (ms / K * 1e-3) / 1e9
+    line = {
+        "metric": "prefill_tokens_per_s", "value": w.batch * P * K / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
+                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "C": w.C, "R": w.R, "fusion": w.fusion,
+                   "prompt_len": P, "kept_tokens_per_unit": n, "units_per_gpu": w.units, "kernel": mk.kernel_name,
+                   "l2": f"inputs larger than L2: the prompt's keys are {w.units * P * w.head_dim * e / 1e6:.0f} MB"},
+        "clocks": clocks.summary(), "e2e": None, "gpu_launches": int(mk.launch_count - launches0),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": peak_src, "kernel": "prefill (two scoring passes + select + gather)",
+                     "algorithmic_bytes_per_launch": bytes_step},
+    }
+    print(json.dumps(line), flush=True)
+    mk.close()
 
 
 def run_ours(args, w):
@@ -474,6 +560,8 @@ def main():
         w = w.replace(prompt_len=args.prompt_len)
     if args.impl == "reference":
         run_reference(args, w)
+    elif w.name.startswith("prefill_"):
+        run_prefill_arm(args, w)
     else:
         run_ours(args, w)
 

@@ -137,6 +137,11 @@ void mkv_destroy(mkv_ctx *ctx);
 mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
                        int prompt_len, void *stream);
 
+/* Forgets the sequence a context holds, so that mkv_prefill can load the next one into the same context (and the
+ * same workspace and scratch).  Work already enqueued for the old sequence must have completed.  The paper has no
+ * counterpart: this is context life-cycle. */
+mkv_status mkv_reset(mkv_ctx *ctx);
+
 /* mkv_prefill for callers that must not allocate (the paper has no counterpart: this is an
  * integration aid, not part of the method).  Some hosts of this library cannot let it call
  * cudaMalloc: a serving engine that has already handed all of HBM to its own pool, where a

@@ -24,7 +24,7 @@ DTYPE = {"bf16": 0, "f32": 1}
 KERNEL = {"auto": 0, "simt": 1, "tc": 2}
 
 EXPORTS = [
-    "mkv_default_params", "mkv_workspace_bytes", "mkv_create", "mkv_create_ex", "mkv_destroy", "mkv_prefill",
+    "mkv_default_params", "mkv_workspace_bytes", "mkv_create", "mkv_create_ex", "mkv_destroy", "mkv_reset", "mkv_prefill",
     "mkv_prefill_static",
     "mkv_decode_step", "mkv_decode_step_layer", "mkv_decode_steps", "mkv_decode_step_host", "mkv_cache_view", "mkv_sync", "mkv_last_error",
     "mkv_launch_count", "mkv_kernel_name",
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
         L.mkv_create_ex.argtypes = [C.POINTER(vp), C.POINTER(mkv_params)]
         L.mkv_destroy.argtypes = [vp]
         L.mkv_destroy.restype = None
+        L.mkv_reset.argtypes = [vp]
         L.mkv_prefill.argtypes = [vp, vp, vp, vp, ip, vp]
         L.mkv_prefill_static.argtypes = [vp, vp, vp, vp, ip, vp]
         L.mkv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -132,6 +133,10 @@ def mkv_create_ex(p: mkv_params) -> tuple[int, int]:
 
 def mkv_destroy(ctx) -> None:
     lib().mkv_destroy(ctx)
+
+
+def mkv_reset(ctx) -> int:
+    return lib().mkv_reset(ctx)
 
 
 def mkv_prefill(ctx, k, v, q_window, prompt_len, stream=None) -> int:
@@ -244,6 +249,9 @@ class MorphKV:
     def _check(self, st, where):
         if st != OK:
             raise MkvError(st, where, mkv_last_error(self.ctx))
+
+    def reset(self):
+        self._check(mkv_reset(self.ctx), "mkv_reset")
 
     def prefill(self, k, v, q_window, stream=None):
         self._check(mkv_prefill(self.ctx, k, v, q_window, k.shape[-2], stream), "mkv_prefill")

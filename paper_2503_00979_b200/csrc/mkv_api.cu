@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <initializer_list>
 #include <new>
 
 #include "../../include/mkv.h"
@@ -492,6 +493,17 @@ static mkv_status prefill_any(mkv_ctx *ctx, const void *k, const void *v, const 
         off_q = q_bytes_per_layer(ctx) * Rw * ctx->p.full_layers;
     }
     return core_prefill(ctx, off(k, off_kv), off(v, off_kv), off(q_window, off_q), prompt_len, (cudaStream_t)stream, use_static, who);
+}
+
+mkv_status mkv_reset(mkv_ctx *ctx)
+{
+    if (!ctx) return MKV_INVALID_ARG;
+    for (mkv_ctx *c : {ctx, ctx->full}) {
+        if (!c) continue;
+        c->prefilled = false;
+        c->t = 0; c->n = 0; c->steps = 0; c->next_layer = 0; c->state_ahead = 0; c->cursor = 0;
+    }
+    return MKV_OK;
 }
 
 mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, void *stream)

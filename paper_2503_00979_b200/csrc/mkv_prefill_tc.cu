@@ -24,7 +24,7 @@ namespace mkv {
 
 namespace {
 
-constexpr int kPfStages = 3;
+constexpr int kPfMaxStages = 3;
 constexpr int kPfThreads = 192;
 enum PfWait { kPfKEmpty = 21, kPfKFull, kPfTEmpty, kPfTFull, kPfDrain };
 
@@ -41,21 +41,23 @@ struct PfArgs {
     int rpad;                    // rows padded to a multiple of 32 (pass 2: MMA N)
     int splits;                  // CTAs per unit along the keys
     int tmem_cols;
+    int stages;                  // K stages: 2 with up to 128 window rows (two CTAs share an SM), else 3
     float scale2;
     long long wait_cycles;
 };
 
-__host__ __device__ inline int pf_smem_bytes(int qrows) { return qrows * 256 + kPfStages * kStageBytes + 2048 + 1024; }
+__host__ __device__ inline int pf_stages(int qrows) { return qrows <= 128 ? 2 : kPfMaxStages; }
+__host__ __device__ inline int pf_smem_bytes(int qrows) { return qrows * 256 + pf_stages(qrows) * kStageBytes + 2048 + 1024; }
 
 template <int PASS, int G, int FUSION>
-__global__ void __launch_bounds__(kPfThreads, 1)
+__global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUtensorMap tmK)
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sp = blockIdx.x, ul = blockIdx.y, u = a.ub0 + ul;
-    const int QR = a.qrows, RB = QR / 128;
+    const int QR = a.qrows, RB = QR / 128, kPfStages = a.stages;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t q_addr = sbase, kst_addr = sbase + QR * 256;
     float *negc = reinterpret_cast<float *>(smem + QR * 256 + kPfStages * kStageBytes);     // [256]
@@ -323,7 +325,7 @@ bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P)
 int prefill_tc_splits(int units_in_batch, int P)
 {
     const int nt = (P + kTile - 1) / kTile;
-    int s = (2 * 148 + units_in_batch - 1) / units_in_batch;       // about two CTAs per SM
+    int s = (8 * 148 + units_in_batch - 1) / units_in_batch;       // about four waves of two CTAs per SM
     if (s > nt) s = nt;
     return s < 1 ? 1 : s;
 }
@@ -350,6 +352,7 @@ cudaError_t run_prefill_scores_tc(const DecodeArgs &a, const void *k, const void
     pa.rpad = (pa.rows + 31) & ~31;
     pa.splits = splits;
     pa.tmem_cols = 0;
+    pa.stages = pf_stages(pa.qrows);
     pa.scale2 = a.scale2;
     pa.wait_cycles = kWaitCycles;
     cudaError_t e = launch_pass_any<1>(pa, tm, nb, a.fusion, stream);

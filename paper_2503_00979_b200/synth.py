@@ -117,6 +117,12 @@ for _C in (512, 1024, 2048, 4096, 8192):
             f"c4_C{_C}_{_f}", 1, 128, 32, 8, 128, "bf16", _C + 32, 1024, _C, 32, _f, _SEED0 + 4)
 
 
+# long prompts compressed into a 2K cache by one application of the policy (window 32, sum fusion): the setting of
+# the paper's long-context runs, on the Llama-3.1-8B-shaped stack; `steps` decode steps follow in the parity tests
+for _P in (6144, 32768, 131072):
+    WORKLOADS[f"prefill_P{_P}"] = Workload(f"prefill_P{_P}", 32, 1, 32, 8, 128, "bf16", _P, 8, 2016, 32, "sum", _SEED0 + 5)
+
+
 class Stream:
     """Counter-based generator of a workload's q/k/v at arbitrary positions.
 

@@ -387,6 +387,41 @@ def test_config1_all_units_prompt_phase_and_first_steps_against_the_oracle():
     assert rep.prefill_resyncs <= 2
 
 
+# ---- long prompts into a 2K cache (the long-context setting): the prompt phase on the tensor cores
+@pytest.mark.parametrize("P,layers,n_units", [(6144, 4, 8), (32768, 1, 3)])
+def test_long_prompt_selection_against_the_oracle(P, layers, n_units):
+    # retained set of every checked unit against the oracle's one-shot Algorithm 1 (near-tie rule), kept K/V rows
+    # bit for bit, then a few decode steps whose outputs depend on the window rows' normalisers
+    w = synth.WORKLOADS[f"prefill_P{P}"].replace(layers=layers)
+    rep = run_parity(w, steps=8, n_units=n_units, chunk=8, check_F_every=8)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions == rep.units * 8 and rep.prefill_resyncs <= 1
+
+
+def test_reset_lets_a_context_take_the_next_prompt():
+    w = SMALL.replace(layers=1, batch=1)
+    dev = torch.device("cuda:0")
+    mk = binding.MorphKV(1, 1, 8, 2, 128, w.C, w.R, w.fusion, "bf16")
+    got = []
+    for seed in (1, 2, 1):
+        st = synth.Stream(w.replace(seed=seed), dev)
+        k, v = st.kv(np.arange(w.prompt_len))
+        qw = st.q(np.arange(w.prompt_len - w.R, w.prompt_len))
+        if got:
+            assert binding.mkv_prefill(mk.ctx, k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous(),
+                                       w.prompt_len) == binding.BAD_STATE
+            mk.reset()
+        mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+        kk, vv = st.kv([w.prompt_len])
+        o = mk.decode_step(st.q([w.prompt_len])[:, :, :, 0].bfloat16().contiguous(), kk[:, :, :, 0].bfloat16().contiguous(),
+                           vv[:, :, :, 0].bfloat16().contiguous())
+        mk.sync()
+        got.append((o.clone(), torch.sort(mk.view(0)["pos"], dim=-1).values.clone()))
+    assert torch.equal(got[0][0], got[2][0]) and torch.equal(got[0][1], got[2][1])
+    assert not torch.equal(got[0][0], got[1][0])
+    mk.close()
+
+
 # ---- per-layer entry (a model that runs its layers one after the other) and the layer-aware variant
 @pytest.mark.parametrize("kernel,dtype,d", [("tc", "bf16", 128), ("simt", "f32", 64)])
 @pytest.mark.parametrize("mode", [1, 2])
