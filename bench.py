@@ -54,13 +54,13 @@ def measured_traffic(workload: str):
     return ent["bytes"] if kernel_sources_digest() == ent["sources_sha256"] else None
 
 
-def kernel_sources_digest():
+def kernel_sources_digest(files=("mkv_tc.cu", "mkv_common.cuh", "mkv_sm100.cuh")):
     """SHA-256 of the decode kernel's sources with `//` comments and white space removed: the figure above stays
     attached to the code it was measured on, whatever happens to the comments."""
     h = hashlib.sha256()
     csrc = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2503_00979_b200", "csrc")
     try:
-        for f in ("mkv_tc.cu", "mkv_common.cuh"):
+        for f in files:
             with open(os.path.join(csrc, f), "r") as fh:
                 for line in fh:
                     code = "".join(line.split("//", 1)[0].split())
@@ -511,7 +511,7 @@ def run_ours(args, w):
                          "peak_source": peak_src, "kernel": f"decode_{mk.kernel_name}",
                          "algorithmic_bytes_per_launch": bytes_step},
         }
-        if world == 1 and args.also and w.name == "c1" and args.prompt_len == 0 and T == 1:
+        if world == 1 and args.also and w.name == "c1" and args.prompt_len == 0 and T == 1 and not (args.layers or args.batch):
             # second target configuration (started with a full cache so that every timed step evicts) and the
             # per-layer calling pattern, measured in the same run
             mk.close()
@@ -548,6 +548,8 @@ def main():
                     help="override the workload's prompt length (e.g. C + R to start config 3 with a full cache)")
     ap.add_argument("--evict-interval", type=int, default=1,
                     help="run the policy every T-th step only (coarse-grained eviction appendix)")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small cases for profiler captures)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (small cases for profiler captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", dest="also", action="store_false",
                     help="skip the secondary records (config 3 with a full cache; per-layer calls on config 1)")
@@ -558,6 +560,9 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.prompt_len > 0:
         w = w.replace(prompt_len=args.prompt_len)
+    if args.layers > 0 or args.batch > 0:
+        w = w.replace(layers=args.layers or w.layers, batch=args.batch or w.batch,
+                      name=f"{w.name} (layers={args.layers or w.layers}, batch={args.batch or w.batch})")
     if args.impl == "reference":
         run_reference(args, w)
     elif w.name.startswith("prefill_"):

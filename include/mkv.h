@@ -93,15 +93,17 @@ typedef struct mkv_view {
     float *F;               /* [batch][n_kv_heads][capacity] fused score of each slot at the
                                last selection (-1 for slots inside the recent window)      */
     int32_t *evicted_pos;   /* [batch][n_kv_heads] position evicted by the last step, -1 = none */
-    void *ring_q;           /* [batch][n_kv_heads][R][G][head_dim] recent queries; the query of
-                               position p sits in ring row p % R                            */
-    float *ring_c;          /* [batch][n_kv_heads][R][G] log2-domain soft-max normaliser of a
+    void *ring_q;           /* [batch][n_kv_heads][R][group_stride][head_dim] recent queries; the
+                               query of position p sits in ring row p % R                  */
+    float *ring_c;          /* [batch][n_kv_heads][R][group_stride] log2-domain soft-max normaliser of a
                                ring row: weight(k) = exp2(q.k * log2(e)/sqrt(d) - ring_c);
                                +inf marks an empty row                                     */
     int32_t count;          /* tokens cached per unit of this layer (the same for every unit of it) */
     int32_t capacity;       /* slots per unit: C + R, plus evict_interval if that is > 1; max_tokens
                                for a layer that keeps every token                          */
     int64_t next_pos;       /* absolute position of the next token to decode               */
+    int32_t group_stride;   /* heads per ring slot as laid out in ring_q / ring_c: G, or G rounded up
+                               to a power of two (padding heads: zero query, ring_c = +inf) */
 } mkv_view;
 
 /* Fills *p with defaults: bf16, every-step eviction, automatic kernel and split choice,

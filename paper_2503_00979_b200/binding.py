@@ -45,7 +45,7 @@ class mkv_view(C.Structure):
     _fields_ = [
         ("K", C.c_void_p), ("V", C.c_void_p), ("pos", C.c_void_p), ("F", C.c_void_p), ("evicted_pos", C.c_void_p),
         ("ring_q", C.c_void_p), ("ring_c", C.c_void_p), ("count", C.c_int32), ("capacity", C.c_int32),
-        ("next_pos", C.c_int64),
+        ("next_pos", C.c_int64), ("group_stride", C.c_int32),
     ]
 
 
@@ -291,7 +291,7 @@ class MorphKV:
         st, v = mkv_cache_view(self.ctx, layer)
         self._check(st, "mkv_cache_view")
         s = self.shape
-        B, H, cap, d, R, G = s["B"], s["Hkv"], v.capacity, s["d"], s["R"], s["G"]
+        B, H, cap, d, R, G = s["B"], s["Hkv"], v.capacity, s["d"], s["R"], v.group_stride
         dev = self.device
         return dict(
             K=_from_ptr(v.K, (B, H, cap, d), self.torch_dtype, dev),

@@ -25,6 +25,7 @@ struct Shape {
     int layers;             // layers served by this context's own arena
     int upl;                // units per layer = batch * n_kv_heads
     int U, G, D, R, C, cap, splits, T, tc_grid_size, tc_grid_layer;
+    int Gq;                 // the model's GQA ratio; G is it rounded up to a power of two on the tensor-core path
     size_t es;
 };
 
@@ -46,10 +47,10 @@ Layout make_layout(const Shape &s)
     L.ticket = take(U * 4);
     L.evicted = take(U * 4);
     L.state = take(sizeof(DevState) * (1 + (size_t)s.layers));     // whole-stack state, then one per layer
-    L.stage_q = take(U * G * D * s.es);
+    L.stage_q = take(U * (size_t)s.Gq * D * s.es);
     L.stage_k = take(U * D * s.es);
     L.stage_v = take(U * D * s.es);
-    L.stage_o = take(U * G * D * s.es);
+    L.stage_o = take(U * (size_t)s.Gq * D * s.es);
     L.total = o;
     return L;
 }
@@ -81,7 +82,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     s->layers = p->layers - p->full_layers;
     s->upl = p->batch * p->n_kv_heads;
     s->U = s->layers * s->upl;
-    s->G = p->n_q_heads / p->n_kv_heads;
+    s->G = s->Gq = p->n_q_heads / p->n_kv_heads;
     s->D = p->head_dim;
     s->R = p->R;
     s->C = p->C;
@@ -95,6 +96,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
     if (tc_ok && p->kernel != MKV_KERNEL_SIMT) {
         *kind = kKindTc;
+        s->G = tc_padded_group(s->Gq);
         // the persistent grid (148 SMs on B200; correctness does not depend on the count)
         s->tc_grid_size = tc_grid(s->U, s->cap, p->splits, 148);
         // a per-layer call sees only a layer's units: ranges of about an eighth of a unit's tiles, so that a layer
@@ -159,7 +161,7 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.ticket = (int *)(b + c->L.ticket); a.evicted_pos = (int *)(b + c->L.evicted);
     a.st = (DevState *)(b + c->L.state);
     a.u0 = 0;
-    a.U = c->s.U; a.G = c->s.G; a.R = c->s.R; a.C = c->s.C; a.cap = c->s.cap; a.splits = c->s.splits;
+    a.U = c->s.U; a.G = c->s.G; a.Gq = c->s.Gq; a.R = c->s.R; a.C = c->s.C; a.cap = c->s.cap; a.splits = c->s.splits;
     a.fusion = c->p.fusion == MKV_FUSION_SUM ? kFusionSum : kFusionMax;
     a.T = c->s.T;
     a.scale2 = (float)(1.4426950408889634 / sqrt((double)c->s.D));
@@ -377,6 +379,7 @@ void core_view(mkv_ctx *ctx, int layer, mkv_view *view)
     const bool ev = step_scores(ctx->t, ctx->n, ctx->steps, s.R, s.C, s.T);
     view->count = !ahead ? ctx->n : (!ev ? ctx->n + 1 : (s.T > 1 ? s.C + s.R : ctx->n));
     view->capacity = s.cap;
+    view->group_stride = s.G;
     view->next_pos = ctx->t + (ahead ? 1 : 0);
 }
 
@@ -578,7 +581,7 @@ mkv_status mkv_decode_step_host(mkv_ctx *ctx, const void *q_host, const void *k_
     if (!ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_decode_step_host: call mkv_prefill first%s");
     if (ctx->full) return fail(ctx, MKV_UNSUPPORTED, "mkv_decode_step_host: not available with full_layers; copy the inputs and call mkv_decode_step%s");
     cudaStream_t s = (cudaStream_t)stream;
-    const size_t qb = (size_t)ctx->s.U * ctx->s.G * ctx->s.D * ctx->s.es, kb = (size_t)ctx->s.U * ctx->s.D * ctx->s.es;
+    const size_t qb = (size_t)ctx->s.U * ctx->s.Gq * ctx->s.D * ctx->s.es, kb = (size_t)ctx->s.U * ctx->s.D * ctx->s.es;
     char *b = ctx->base;
     // Pinned host buffers are reachable from the device: the tensor-core kernel then reads q, k_new, v_new and
     // writes `out` in place over the interconnect (a few hundred KB per step, read once or twice), which saves

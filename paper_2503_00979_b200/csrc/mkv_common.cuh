@@ -47,6 +47,9 @@ struct DecodeArgs {
     int u0;                    // index of this launch's first unit in the context's arena (per-layer launches): the
                                // pointers above are already offset by it, tensor-map coordinates are not
     int U, G, R, C, cap, splits, fusion, T;
+    int Gq;                    // query heads per unit in q and out (the model's GQA ratio).  G, the group the arena
+                               // and the kernels work with, is Gq rounded up to a power of two on the tensor-core path:
+                               // heads Gq .. G-1 have a zero query and normaliser +inf (weight 0) and produce no output
     float scale2;              // log2(e) / sqrt(D)
 };
 
@@ -138,7 +141,8 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     unsigned long long *red_key = reinterpret_cast<unsigned long long *>(sm + 4 * kMaxGroup);  // [32]
     int *red_slot = reinterpret_cast<int *>(sm + 4 * kMaxGroup + 64);                          // [32]
 
-    const T *q = static_cast<const T *>(a.q) + (size_t)u * G * D;
+    const int Gq = a.Gq;
+    const T *q = static_cast<const T *>(a.q) + (size_t)u * Gq * D;
     const T *kn = static_cast<const T *>(a.k_new) + (size_t)u * D;
     const T *vn = static_cast<const T *>(a.v_new) + (size_t)u * D;
     const float *pml = a.part_ml + (size_t)u * a.splits * G * 2;
@@ -147,7 +151,8 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     // the new token attends to itself (self-inclusive Eq. 1): one more logit per head
     for (int g = warp; g < G; g += nwarp) {
         float acc = 0.f;
-        for (int i = lane; i < D; i += 32) acc += ldf(q + g * D + i) * ldf(kn + i);
+        if (g < Gq)
+            for (int i = lane; i < D; i += 32) acc += ldf(q + g * D + i) * ldf(kn + i);
         acc = warp_sum(acc);
         if (lane == 0) s_self[g] = acc * a.scale2;
     }
@@ -176,11 +181,11 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
         }
         mfin[tid] = m;
         lfin[tid] = l;
-        cnew[tid] = m + log2f(l);
+        cnew[tid] = tid < Gq ? m + log2f(l) : INFINITY;
     }
     group_sync(bar_id, nthr);
-    T *out = static_cast<T *>(a.out) + (size_t)u * G * D;
-    for (int idx = tid; idx < G * D; idx += nthr) {
+    T *out = static_cast<T *>(a.out) + (size_t)u * Gq * D;
+    for (int idx = tid; idx < Gq * D; idx += nthr) {
         const int g = idx / D, dd = idx % D;
         const float m = mfin[g];
         float o = exp2f(s_self[g] - m) * ldf(vn + dd);
@@ -287,7 +292,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     for (int i = tid; i < D; i += nthr) { Kd[i] = kn[i]; Vd[i] = vn[i]; }
     const int rs = (int)(t % a.R);
     T *rq = static_cast<T *>(a.ring_q) + ((size_t)u * a.R + rs) * G * D;
-    for (int i = tid; i < G * D; i += nthr) rq[i] = q[i];
+    for (int i = tid; i < G * D; i += nthr) stf(rq + i, i < Gq * D ? ldf(q + i) : 0.f);
     if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
     if (tid == 0) {
         pos[e_slot] = (int)t;

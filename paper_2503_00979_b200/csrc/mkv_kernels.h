@@ -18,6 +18,7 @@ cudaError_t launch_compact(const DecodeArgs &a, bool f32, int D, cudaStream_t st
 // context's arena and the launch geometry; `a.splits` must be tc_partials_per_unit()
 // of the grid (every CTA that holds tiles of a unit leaves one partial).
 bool tc_shape_supported(bool f32, int D, int G, int R);
+int tc_padded_group(int G);
 int tc_grid(int U, int cap, int splits_hint, int n_sm);
 int tc_partials_per_unit(int U, int cap, int grid);
 struct TcPlan;

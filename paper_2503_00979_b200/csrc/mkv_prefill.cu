@@ -251,12 +251,13 @@ __global__ void prefill_gather_kernel(const T *__restrict__ k, const T *__restri
 template <typename T, int D>
 __global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, int P, int Rw)
 {
-    const int u = blockIdx.x, G = a.G;
+    const int u = blockIdx.x, G = a.G, Gq = a.Gq;       // heads Gq .. G-1 of a ring slot are padding (zero query)
     T *rq = static_cast<T *>(a.ring_q) + (size_t)u * a.R * G * D;
     for (int idx = threadIdx.x; idx < Rw * G * D; idx += blockDim.x) {
         const int dd = idx % D, g = (idx / D) % G, i = idx / (D * G);
         const int rslot = (P - Rw + i) % a.R;
-        rq[((size_t)rslot * G + g) * D + dd] = qwin[(((size_t)u * G + g) * Rw + i) * D + dd];
+        if (g < Gq) rq[((size_t)rslot * G + g) * D + dd] = qwin[(((size_t)u * Gq + g) * Rw + i) * D + dd];
+        else stf(rq + ((size_t)rslot * G + g) * D + dd, 0.f);
     }
 }
 
@@ -274,7 +275,8 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     if (n > a.cap) return cudaErrorInvalidValue;
     // bf16 / head_dim 128 shapes score on the tensor cores (two passes over the keys, no rows x P table); the
     // others materialise the window-row logits S [rows][P] per unit and reduce them with CUDA-core kernels
-    const bool tc = prefill_tc_supported(sizeof(T) == 4, D, G, R, k, P);
+    const bool tc = prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P);
+    if (!tc && a.Gq != G) return cudaErrorInvalidValue;     // a padded group exists on the tensor-core path only
     const int tc_splits = tc ? prefill_tc_splits(U, P) : 0;
     const size_t per_unit = tc ? prefill_tc_floats_per_unit(P, Rw, G, tc_splits) : (size_t)rows * P + P;   // floats
     if (per_unit + 1 > scratch_floats) return cudaErrorInvalidConfiguration;
@@ -387,7 +389,7 @@ cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, con
                         cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states)
 {
     const int Rw = P < a.R ? P : a.R;
-    const bool tc = prefill_tc_supported(f32, D, a.G, a.R, k, P);
+    const bool tc = prefill_tc_supported(f32, D, a.Gq, a.R, k, P);
     const size_t per_unit = (tc ? prefill_tc_floats_per_unit(P, Rw, a.G, prefill_tc_splits(a.U, P))
                                 : (size_t)Rw * a.G * P + P) * sizeof(float);
     size_t ub = ((size_t)1 << 30) / per_unit;

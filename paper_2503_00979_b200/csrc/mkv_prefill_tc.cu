@@ -36,6 +36,7 @@ struct PfArgs {
     int *err;                    // error word (0 = none)
     int ub0;                     // first unit of this batch
     int P, Rw, G, R;
+    int Gq;                      // real heads per unit in qwin; heads Gq .. G-1 are padding
     int rows;                    // Rw * G window rows; row = window slot * G + head
     int qrows;                   // rows padded to a multiple of 128 (pass 1: MMA M blocks)
     int rpad;                    // rows padded to a multiple of 32 (pass 2: MMA N)
@@ -89,9 +90,9 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
     for (int c = tid; c < QR * 16; c += kPfThreads) {
         const int row = c >> 4, ch = c & 15;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (row < a.rows) {
+        if (row < a.rows && row % G < a.Gq) {
             const int i = row / G, g = row % G;
-            v = reinterpret_cast<const uint4 *>(a.qwin + (((size_t)u * G + g) * a.Rw + i) * kD)[ch];
+            v = reinterpret_cast<const uint4 *>(a.qwin + (((size_t)u * a.Gq + g) * a.Rw + i) * kD)[ch];
         }
         const uint32_t off = (uint32_t)((ch >> 3) * (QR * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4));
         *reinterpret_cast<uint4 *>(smem + off) = v;
@@ -109,7 +110,8 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
                     const float ms = pm[((size_t)s * QR + row) * 2];
                     if (ms > -INFINITY) l += pm[((size_t)s * QR + row) * 2 + 1] * exp2f(ms - m);
                 }
-                const float c = m + log2f(l);
+                // a padding head (zero query) takes no part: normaliser +inf, weight 0
+                const float c = row % G < a.Gq ? m + log2f(l) : INFINITY;
                 nc = -c;
                 if (sp == 0) {
                     const int i = row / G, g = row % G;
@@ -346,7 +348,7 @@ cudaError_t run_prefill_scores_tc(const DecodeArgs &a, const void *k, const void
     PfArgs pa;
     pa.qwin = static_cast<const __nv_bfloat16 *>(qwin);
     pa.part_ml = part; pa.ring_c = a.ring_c; pa.Fp = Fp; pa.err = err;
-    pa.ub0 = ub0; pa.P = P; pa.Rw = P < a.R ? P : a.R; pa.G = a.G; pa.R = a.R;
+    pa.ub0 = ub0; pa.P = P; pa.Rw = P < a.R ? P : a.R; pa.G = a.G; pa.R = a.R; pa.Gq = a.Gq;
     pa.rows = pa.Rw * a.G;
     pa.qrows = ((pa.rows + 127) / 128) * 128;
     pa.rpad = (pa.rows + 31) & ~31;

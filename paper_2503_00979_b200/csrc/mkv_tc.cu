@@ -181,7 +181,8 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     unsigned long long *red_key = reinterpret_cast<unsigned long long *>(pml_s + 256);   // [32]
     int *red_slot = reinterpret_cast<int *>(pml_s + 256 + 64);                           // [32]
 
-    const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(a.q) + (size_t)u * G * kD;
+    const int Gq = a.Gq;      // heads Gq .. G-1 are padding: zero query, normaliser +inf, no output
+    const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(a.q) + (size_t)u * Gq * kD;
     const __nv_bfloat16 *kn = static_cast<const __nv_bfloat16 *>(a.k_new) + (size_t)u * kD;
     const __nv_bfloat16 *vn = static_cast<const __nv_bfloat16 *>(a.v_new) + (size_t)u * kD;
     const float *pml = a.part_ml + (size_t)u * a.splits * G * 2;
@@ -194,7 +195,7 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     for (int i = 0; i < QCH; ++i) {
         const int c = tid + i * NT_;
         if (c < G * 16) {
-            qv[i] = reinterpret_cast<const uint4 *>(q)[c];
+            qv[i] = c < Gq * 16 ? reinterpret_cast<const uint4 *>(q)[c] : make_uint4(0, 0, 0, 0);
             kv[i] = reinterpret_cast<const uint4 *>(kn)[c & 15];
         }
     }
@@ -243,10 +244,10 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
         for (int sp = 0; sp < nseg; ++sp) l += pml_s[(sp * G + tid) * 2 + 1] * exp2f(pml_s[(sp * G + tid) * 2] - m);
         mfin[tid] = m;
         lfin[tid] = l;
-        cnew[tid] = m + log2f(l);
+        cnew[tid] = tid < Gq ? m + log2f(l) : INFINITY;
     }
     group_sync(bar_id, NT_);
-    __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(a.out) + (size_t)u * G * kD;
+    __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(a.out) + (size_t)u * Gq * kD;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         const float m = mfin[g];
@@ -254,7 +255,7 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
 #pragma unroll
         for (int sp = 0; sp < 8; ++sp)
             if (sp < nseg) o += pov[g][sp] * exp2f(pml_s[(sp * G + g) * 2] - m);
-        out[g * kD + tid] = __float2bfloat16_rn(o / lfin[g]);
+        if (g < Gq) out[g * kD + tid] = __float2bfloat16_rn(o / lfin[g]);
     }
 
     // ---- phase C: final fused scores and the eviction (Algorithm 1 / Eq. 7)
@@ -505,10 +506,10 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 if (w.nitems > 0 && lane == 0) umma_commit(bar_qempty);   // MMAs of the previous unit done with the ring
                 // the new query replaces ring row t % R (the row of the token leaving the window)
                 uint4 qv[kMaxGroup / 2];
-                const uint4 *qsrc = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(a.q) + (size_t)x.unit * G * kD);
+                const uint4 *qsrc = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(a.q) + (size_t)x.unit * a.Gq * kD);
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i)
-                    if (lane + 32 * i < G * 16) qv[i] = qsrc[lane + 32 * i];
+                    if (lane + 32 * i < G * 16) qv[i] = lane + 32 * i < a.Gq * 16 ? qsrc[lane + 32 * i] : make_uint4(0, 0, 0, 0);
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull, (uint32_t)(w.nitems & 1), abort_flag, kWaitQFull, WL));
                 if (!ok) break;
 #pragma unroll
@@ -907,10 +908,18 @@ int pad32(int x) { return (x + 31) & ~31; }
 
 }  // namespace
 
+int tc_padded_group(int G)
+{
+    int g = 1;
+    while (g < G) g *= 2;
+    return g;
+}
+
+// G: the model's GQA ratio; the kernel works with the group padded to a power of two
 bool tc_shape_supported(bool f32, int D, int G, int R)
 {
-    if (f32 || D != kD || group_index(G) < 0) return false;
-    return pad32(R * G) <= 256;
+    if (f32 || D != kD || G < 1 || G > kMaxGroup) return false;
+    return pad32(R * tc_padded_group(G)) <= 256;
 }
 
 // Grid of the persistent kernel.  `splits_hint` > 0 asks for about that many CTAs per unit

@@ -178,20 +178,21 @@ def test_auto_picks_the_tensor_core_kernel_for_bf16_d128():
     mk = binding.MorphKV(1, 1, 8, 2, 64, 64, 16, "sum", "bf16")
     assert mk.kernel_name == "simt"
     mk.close()
-    mk = binding.MorphKV(1, 1, 14, 2, 128, 64, 16, "sum", "bf16")      # G = 7: CUDA-core kernel
-    assert mk.kernel_name == "simt"
+    mk = binding.MorphKV(1, 1, 14, 2, 128, 64, 16, "sum", "bf16")      # G = 7: group padded to 8 on the tensor cores
+    assert mk.kernel_name == "tc" and mk.view(0)["ring_c"].shape[-1] == 8
     mk.close()
     p = binding.mkv_default_params()
-    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 14, 2, 128, 64, 16
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 14, 2, 128, 64, 40     # 40 * 8 rows > 256
     p.kernel = binding.KERNEL["tc"]
     st, h = binding.mkv_create_ex(p)
     assert st == binding.UNSUPPORTED and h is None
 
 
 @pytest.mark.parametrize("fusion", ["sum", "max"])
-@pytest.mark.parametrize("G,R", [(1, 32), (2, 24), (4, 32), (4, 30), (8, 16), (16, 9), (4, 64)])
+@pytest.mark.parametrize("G,R", [(1, 32), (2, 24), (4, 32), (4, 30), (8, 16), (16, 9), (4, 64), (7, 30), (3, 20), (6, 12)])
 def test_tc_groups_windows_and_fusions(fusion, G, R):
-    # R*G = 120 and 144 are padded to a multiple of 32; R*G = 256 fills both accumulator buffers
+    # R*G = 120 and 144 are padded to a multiple of 32; R*G = 256 fills both accumulator buffers; G = 7 (the 28/4 head
+    # ratio of the LongWriter table's Qwen row), 3 and 6 run with the group padded to the next power of two
     w = SMALL.replace(layers=1, batch=2, n_q_heads=2 * G, n_kv_heads=2, R=R, C=301, prompt_len=411, steps=40,
                       fusion=fusion)
     rep = run_parity(w, steps=w.steps, n_units=4, kernel="tc")
