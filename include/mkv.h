@@ -51,6 +51,10 @@ typedef enum mkv_status {
 typedef enum mkv_fusion { MKV_FUSION_SUM = 0, MKV_FUSION_MAX = 1 } mkv_fusion;   /* Eq. 5, Eq. 6 */
 typedef enum mkv_dtype { MKV_DTYPE_BF16 = 0, MKV_DTYPE_F32 = 1 } mkv_dtype;
 /* which decode kernel to use: AUTO picks the tensor-core kernel when the shape allows it */
+/* How a window row's attention weights enter the fused score (Eq. 4).  FROZEN: as the row assigned them when its
+ * token was generated ("the attention weight that w_r assigned").  CURRENT: renormalised over the tokens that are
+ * still cached when the scores are taken (a row never saw tokens newer than itself); not with evict_interval > 1. */
+typedef enum mkv_norm { MKV_NORM_FROZEN = 0, MKV_NORM_CURRENT = 1 } mkv_norm;
 typedef enum mkv_kernel { MKV_KERNEL_AUTO = 0, MKV_KERNEL_SIMT = 1, MKV_KERNEL_TC = 2 } mkv_kernel;
 
 typedef struct mkv_ctx mkv_ctx;
@@ -71,6 +75,7 @@ typedef struct mkv_params {
     void *workspace;        /* device memory owned by the caller, 256-byte aligned, or NULL
                                to let the library allocate it with cudaMalloc              */
     size_t workspace_bytes;
+    mkv_norm norm_mode;     /* MKV_NORM_FROZEN (default) or MKV_NORM_CURRENT                                 */
     int full_layers;        /* layer-aware variant (the appendix on selective layer retention): MorphKV is
                                switched off for the first full_layers layers, which keep every token; the
                                other layers run MorphKV as usual.  0 = none.                           */

@@ -66,6 +66,7 @@ bool params_valid(const mkv_params *p)
     if (p->dtype != MKV_DTYPE_BF16 && p->dtype != MKV_DTYPE_F32) return false;
     if (p->evict_interval < 0 || p->splits < 0) return false;
     if (p->kernel != MKV_KERNEL_AUTO && p->kernel != MKV_KERNEL_SIMT && p->kernel != MKV_KERNEL_TC) return false;
+    if (p->norm_mode != MKV_NORM_FROZEN && p->norm_mode != MKV_NORM_CURRENT) return false;
     if (p->full_layers < 0 || p->full_layers >= p->layers) return false;
     if (p->full_layers > 0 && p->max_tokens <= p->R) return false;
     const long long units = (long long)p->layers * p->batch * p->n_kv_heads;
@@ -91,6 +92,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     s->cap = p->C + p->R + (s->T > 1 ? s->T : 0);
     s->es = p->dtype == MKV_DTYPE_F32 ? 4 : 2;
     if (s->T > 64) return false;
+    if (p->norm_mode == MKV_NORM_CURRENT && s->T > 1) return false;     // the compaction drops several tokens at once
     const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R) &&
                        (long long)s->U * ((s->cap + 127) / 128) <= (1ll << 30);     // tile indices stay 32-bit
     if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
@@ -164,6 +166,7 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.U = c->s.U; a.G = c->s.G; a.Gq = c->s.Gq; a.R = c->s.R; a.C = c->s.C; a.cap = c->s.cap; a.splits = c->s.splits;
     a.fusion = c->p.fusion == MKV_FUSION_SUM ? kFusionSum : kFusionMax;
     a.T = c->s.T;
+    a.norm_current = c->p.norm_mode == MKV_NORM_CURRENT ? 1 : 0;
     a.scale2 = (float)(1.4426950408889634 / sqrt((double)c->s.D));
     return a;
 }

@@ -47,6 +47,7 @@ struct DecodeArgs {
     int u0;                    // index of this launch's first unit in the context's arena (per-layer launches): the
                                // pointers above are already offset by it, tensor-map coordinates are not
     int U, G, R, C, cap, splits, fusion, T;
+    int norm_current;          // 1: CURRENT normalisation - window rows are renormalised over the tokens still cached
     int Gq;                    // query heads per unit in q and out (the model's GQA ratio).  G, the group the arena
                                // and the kernels work with, is Gq rounded up to a power of two on the tensor-core path:
                                // heads Gq .. G-1 have a zero query and normaliser +inf (weight 0) and produce no output
@@ -112,7 +113,8 @@ __host__ __device__ inline bool step_scores(long long t, int n, int steps, int R
     return step_evicts(t, n, R, C);
 }
 
-constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32;
+constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32 + 128;
+
 
 // barrier over the `nthr` threads that run an epilogue together (id 0 with the whole CTA is
 // __syncthreads; warp-specialised kernels give each compute group its own id)
@@ -122,6 +124,49 @@ __device__ __forceinline__ void group_sync(int bar_id, int nthr)
     // point on different paths, e.g. straight after an `if (tid < k)` block, and each counts for itself
     asm volatile("barrier.sync %0, %1;" ::"r"(bar_id), "r"(nthr) : "memory");
 }
+
+// CURRENT normalisation (the reading of Eq. 4 in which a window row's weights are taken over the tokens that are
+// still cached): the token in `e_slot` is about to be evicted, so every window row loses the weight w it had on it
+// and its log2-domain normaliser becomes c + log2(1 - w); the surviving weights of the row grow by 1 / (1 - w).
+// Rows of the ring: the row `rs_new` is being replaced by the new query, whose normaliser is cnew[g] (shared memory,
+// updated in place) and whose logits on the evicted key are in s_new; the other rows' logits are recomputed from
+// the stored queries.  `krow` is scratch for D floats.  Called by the whole group before the evicted slot's K row
+// is overwritten.
+template <typename T, int D>
+__device__ void renormalise_after_eviction(const DecodeArgs &a, int u, int e_slot, int rs_new, float *cnew, float *krow,
+                                           int tid, int nthr, int bar_id)
+{
+    const int G = a.G;
+    const T *Ke = static_cast<const T *>(a.K) + ((size_t)u * a.cap + e_slot) * D;
+    for (int i = tid; i < D; i += nthr) krow[i] = ldf(Ke + i);
+    group_sync(bar_id, nthr);
+    const T *ring_q = static_cast<const T *>(a.ring_q) + (size_t)u * a.R * G * D;
+    float *ring_c = a.ring_c + (size_t)u * a.R * G;
+    for (int row = tid; row < a.R * G; row += nthr) {
+        const int rslot = row / G, g = row % G;
+        float c, s;
+        if (rslot == rs_new) {
+            c = cnew[g];
+            s = __ldcg(a.s_new + ((size_t)u * G + g) * a.cap + e_slot);
+        } else {
+            c = ring_c[row];
+            s = 0.f;
+            if (c < INFINITY) {
+                const T *qr = ring_q + (size_t)row * D;
+                float acc = 0.f;
+                for (int i = 0; i < D; ++i) acc += ldf(qr + i) * krow[i];
+                s = acc * a.scale2;
+            }
+        }
+        if (c < INFINITY) {
+            const float w = exp2f(s - c);
+            c += log2f(fmaxf(1.f - w, 1e-30f));
+            if (rslot == rs_new) cnew[g] = c; else ring_c[row] = c;
+        }
+    }
+    group_sync(bar_id, nthr);
+}
+
 
 // Per-unit epilogue, run by the group of threads that finished a unit last (`tid` in
 // [0, nthr), nthr a multiple of 32, all of them synchronising on barrier `bar_id`).  Data
@@ -278,6 +323,8 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
             e_slot = n;
             e_pos = -1;
             if (tid == 0 && n < a.cap) F[n] = -1.f;
+        } else if (a.norm_current) {
+            renormalise_after_eviction<T, D>(a, u, e_slot, (int)(t % a.R), cnew, sm + 4 * kMaxGroup + 3 * 32, tid, nthr, bar_id);
         }
     }
 

@@ -264,6 +264,63 @@ __global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, in
 // The prompt phase on a scratch area of `scratch_floats` floats (the window-row logits S and the fused scores of
 // as many units as fit go through it, batch after batch).  Every element a kernel reads was written earlier in the
 // same batch, so what the area held before never matters.
+// CURRENT normalisation after the prompt-phase selection: each window row's normaliser is taken again over the
+// tokens that were kept and that the row may see, c = log2 sum exp2(s), from the arena as it stands (kept K rows,
+// their positions, the ring's queries).  One CTA per (window row, unit).
+template <typename T, int D>
+__global__ void __launch_bounds__(kPT) prefill_renorm_kernel(DecodeArgs a, int P, int Rw, int n)
+{
+    __shared__ float qs[D];
+    __shared__ float red[kPT / 32];
+    __shared__ float bc;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int u = blockIdx.y, G = a.G, row = blockIdx.x, i = row / G, g = row % G;
+    const int rpos = P - Rw + i, rslot = rpos % a.R;
+    float *c_out = a.ring_c + ((size_t)u * a.R + rslot) * G + g;
+    if (*c_out == INFINITY) return;                                   // padding head
+    const T *q = static_cast<const T *>(a.ring_q) + (((size_t)u * a.R + rslot) * G + g) * D;
+    for (int d = tid; d < D; d += kPT) qs[d] = ldf(q + d);
+    __syncthreads();
+    const T *K = static_cast<const T *>(a.K) + (size_t)u * a.cap * D;
+    const int *pos = a.pos + (size_t)u * a.cap;
+    float s[8];       // up to 8 slots per thread per round
+    float m = -INFINITY, l = 0.f;
+    for (int k0 = 0; k0 < n; k0 += 8 * kPT) {
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const int k = k0 + b * kPT + tid;
+            s[b] = -INFINITY;
+            if (k < n && pos[k] <= rpos) {
+                float acc = 0.f;
+                for (int d = 0; d < D; ++d) acc += qs[d] * ldf(K + (size_t)k * D + d);
+                s[b] = acc * a.scale2;
+            }
+        }
+        float cm = m;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) cm = fmaxf(cm, s[b]);
+        if (cm > m) { l *= exp2f(m - cm); m = cm; }
+        if (m > -INFINITY)
+#pragma unroll
+            for (int b = 0; b < 8; ++b) l += exp2f(s[b] - m);
+    }
+    float bm = warp_max(m);
+    if (lane == 0) red[warp] = bm;
+    __syncthreads();
+    if (tid == 0) { float x = red[0]; for (int w = 1; w < kPT / 32; ++w) x = fmaxf(x, red[w]); bc = x; }
+    __syncthreads();
+    bm = bc;
+    float bl = warp_sum(m > -INFINITY ? l * exp2f(m - bm) : 0.f);
+    __syncthreads();
+    if (lane == 0) red[warp] = bl;
+    __syncthreads();
+    if (tid == 0) {
+        float x = 0.f;
+        for (int w = 0; w < kPT / 32; ++w) x += red[w];
+        *c_out = bm + log2f(x);
+    }
+}
+
 template <typename T, int D>
 cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
                           unsigned long long *launches, float *S, size_t scratch_floats, int n_states)
@@ -275,7 +332,8 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     if (n > a.cap) return cudaErrorInvalidValue;
     // bf16 / head_dim 128 shapes score on the tensor cores (two passes over the keys, no rows x P table); the
     // others materialise the window-row logits S [rows][P] per unit and reduce them with CUDA-core kernels
-    const bool tc = prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P);
+    // (the arena's group must be the padded one: a context that runs the CUDA-core decode kernel keeps G as it is)
+    const bool tc = prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P) && tc_padded_group(a.Gq) == G;
     if (!tc && a.Gq != G) return cudaErrorInvalidValue;     // a padded group exists on the tensor-core path only
     const int tc_splits = tc ? prefill_tc_splits(U, P) : 0;
     const size_t per_unit = tc ? prefill_tc_floats_per_unit(P, Rw, G, tc_splits) : (size_t)rows * P + P;   // floats
@@ -325,6 +383,10 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     constexpr int CH = D * sizeof(T) / 16;
     prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
     prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
+    if (a.norm_current && select) {
+        prefill_renorm_kernel<T, D><<<dim3(rows, U), kPT, 0, stream>>>(a, P, Rw, n);
+        ++*launches;
+    }
     set_state_kernel<<<1, 32, 0, stream>>>(a.st, n_states, (long long)P, n);
     *launches += 3;
     e = cudaGetLastError();
@@ -389,7 +451,7 @@ cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, con
                         cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states)
 {
     const int Rw = P < a.R ? P : a.R;
-    const bool tc = prefill_tc_supported(f32, D, a.Gq, a.R, k, P);
+    const bool tc = prefill_tc_supported(f32, D, a.Gq, a.R, k, P) && tc_padded_group(a.Gq) == a.G;
     const size_t per_unit = (tc ? prefill_tc_floats_per_unit(P, Rw, a.G, prefill_tc_splits(a.U, P))
                                 : (size_t)Rw * a.G * P + P) * sizeof(float);
     size_t ub = ((size_t)1 << 30) / per_unit;

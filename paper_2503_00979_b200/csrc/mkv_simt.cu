@@ -59,7 +59,7 @@ __host__ __device__ inline SimtSmem simt_smem_layout(int chunk_rows, int G)
     L.s_off = o; o += (size_t)kTK * (kSB + 1) * sizeof(float); o = (o + 15) & ~(size_t)15;
     L.f_off = o; o += (size_t)kTK * sizeof(float);
     L.p_off = o; o += (size_t)G * kThreads * sizeof(float);
-    L.misc_off = o; o += 256 * sizeof(float);
+    L.misc_off = o; o += 384 * sizeof(float);
     L.total = o;
     return L;
 }

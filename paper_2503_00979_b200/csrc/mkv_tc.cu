@@ -323,6 +323,9 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
             e_slot = n;
             e_pos = -1;
             if (tid == 0 && n < a.cap) F[n] = -1.f;
+        } else if (a.norm_current) {
+            // vsm (the new value row as floats) was last read for the attention output: free to hold the evicted key
+            renormalise_after_eviction<__nv_bfloat16, kD>(a, u, e_slot, (int)(t % a.R), cnew, vsm, tid, NT_, bar_id);
         }
     }
 

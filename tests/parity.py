@@ -111,7 +111,7 @@ def oracle_unit_following(make_unit, k, v, qw, device_positions, where: str):
 def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chunk: int = 32, kernel: str = "auto",
                splits: int = 0, check_F_every: int = 16, device: str = "cuda:0", use_steps_call: bool = False,
                host_call_every: int = 0, host_pinned: bool = True, synth_device=None, per_layer: int = 0,
-               full_layers: int = 0, max_tokens: int = 0, **ctx_kwargs) -> ParityReport:
+               full_layers: int = 0, max_tokens: int = 0, norm: str = "frozen", **ctx_kwargs) -> ParityReport:
     """Prefill + `steps` decode steps of workload `w` on the device, followed by the oracle on `units`.
 
     The steps of a chunk are enqueued without a synchronisation in between (the evicted positions of the
@@ -121,6 +121,7 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     synth_device     where the inputs are drawn ("cpu" keeps the drawing's many small kernels off the GPU).
     per_layer        1: every step is made of mkv_decode_step_layer calls, layer by layer; 2: steps alternate between
                      one whole-stack call and per-layer calls.
+    norm             "frozen" (default) or "current": how window rows' weights are normalised, on both sides.
     full_layers, max_tokens   layer-aware variant: the first full_layers layers keep every token (the oracle units of
                      those layers get C = max_tokens - R, so they never evict within max_tokens).
     """
@@ -131,7 +132,8 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
     units = units or pick_units(w, n_units)
     rep = ParityReport()
     mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, d, C_, R, w.fusion, w.dtype, kernel=kernel,
-                         splits=splits, device=device, full_layers=full_layers, max_tokens=max_tokens, **ctx_kwargs)
+                         splits=splits, device=device, full_layers=full_layers, max_tokens=max_tokens, norm=norm,
+                         **ctx_kwargs)
     rep.kernel = mk.kernel_name
     C_of = {l: (max_tokens - R if l < full_layers else C_) for l in range(w.layers)}     # distant tokens kept per layer
     tol = TOL_OUT[w.dtype]
@@ -162,7 +164,7 @@ def run_parity(w: synth.Workload, steps: int, units=None, n_units: int = 8, chun
 
     def prefill_unit(key):
         kp, vp, qp = prompt[key]
-        u, resync = oracle_unit_following(lambda: ora.Unit(G, d, C_of[key[0]], R, w.fusion), kp, vp, qp, dev_pos[key], f"unit {key}")
+        u, resync = oracle_unit_following(lambda: ora.Unit(G, d, C_of[key[0]], R, w.fusion, norm=norm), kp, vp, qp, dev_pos[key], f"unit {key}")
         assert count0[key[0]] == u.count, (count0[key[0]], u.count)
         return key, u, resync
 

@@ -423,6 +423,44 @@ def test_reset_lets_a_context_take_the_next_prompt():
     mk.close()
 
 
+# ---- the other reading of Eq. 4: window rows renormalised over the tokens still cached
+@pytest.mark.parametrize("kernel,dtype,d", [("tc", "bf16", 128), ("simt", "f32", 64), ("simt", "bf16", 64)])
+@pytest.mark.parametrize("fusion", ["sum", "max"])
+def test_current_normalisation_against_the_oracle(kernel, dtype, d, fusion):
+    w = SMALL.replace(layers=1, batch=2, head_dim=d, dtype=dtype, C=300, R=16, prompt_len=420, steps=64, fusion=fusion)
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel=kernel, norm="current")
+    _report(rep)
+    assert rep.kernel == kernel and rep.evictions == 4 * 64 and rep.F_compared > 0
+
+
+def test_current_normalisation_differs_from_frozen_and_rejects_coarse_eviction():
+    w = SMALL.replace(layers=1, batch=1, C=200, R=16, prompt_len=300, steps=48, fusion="sum")
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    k, v = st.kv(np.arange(w.prompt_len))
+    qw = st.q(np.arange(w.prompt_len - w.R, w.prompt_len))
+    pos = np.arange(w.prompt_len, w.prompt_len + w.steps)
+    kk, vv = st.kv(pos)
+    qn = st.q(pos).permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    kn = kk.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    vn = vv.permute(3, 0, 1, 2, 4).bfloat16().contiguous()
+    cs = []
+    for norm in ("frozen", "current"):
+        mk = binding.MorphKV(1, 1, 8, 2, 128, w.C, w.R, w.fusion, "bf16", norm=norm)
+        mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
+        mk.decode_steps(qn, kn, vn)
+        mk.sync()
+        cs.append(mk.view(0)["ring_c"].clone())
+        mk.close()
+    # evicted mass leaves the rows' normalisers (and the two policies soon keep different tokens)
+    assert not torch.allclose(cs[0], cs[1], rtol=0, atol=1e-3) and cs[1].mean() < cs[0].mean()
+    p = binding.mkv_default_params()
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 8, 2, 128, 64, 16
+    p.norm_mode, p.evict_interval = binding.NORM["current"], 4
+    st_, h = binding.mkv_create_ex(p)
+    assert st_ == binding.UNSUPPORTED and h is None
+
+
 # ---- per-layer entry (a model that runs its layers one after the other) and the layer-aware variant
 @pytest.mark.parametrize("kernel,dtype,d", [("tc", "bf16", 128), ("simt", "f32", 64)])
 @pytest.mark.parametrize("mode", [1, 2])
