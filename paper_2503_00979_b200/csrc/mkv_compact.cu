@@ -4,8 +4,8 @@
 // it drops the E = n - (C + R) lowest-ranked candidates (lower fused score first, on equal scores
 // the later position first, so that the lower position is the one kept) and moves the survivors
 // that sit beyond slot C + R into the freed slots, which restores a dense prefix of C + R slots.
-// One CTA per unit; launched after every decode step of such a context and a no-op unless the
-// device state says a compaction is pending.
+// One CTA of 1024 threads per unit, each thread holding a few slots' rank keys; launched after the
+// decode steps that ran the policy, and a no-op unless the device state says a compaction is pending.
 #include "mkv_common.cuh"
 #include "mkv_kernels.h"
 
@@ -13,10 +13,10 @@ namespace mkv {
 
 namespace {
 
-constexpr int kCT = 256;          // threads per CTA
-constexpr int kMaxPerThread = 64; // slots a thread holds: capacity up to 16384
+constexpr int kCT = 1024;         // threads per CTA
 
-template <typename T, int D>
+// KPT slots per thread, held in registers (indices are compile-time constants after unrolling)
+template <typename T, int D, int KPT>
 __global__ void __launch_bounds__(kCT) compact_kernel(DecodeArgs a)
 {
     __shared__ unsigned long long red_key[kCT / 32];
@@ -34,9 +34,9 @@ __global__ void __launch_bounds__(kCT) compact_kernel(DecodeArgs a)
         int *pos = a.pos + (size_t)u * a.cap;
         float *F = a.F + (size_t)u * a.cap;
         // every thread's candidates as rank keys (window slots carry F = -1 and never compete)
-        unsigned long long key[kMaxPerThread];
-#pragma unroll 1
-        for (int i = 0; i < kMaxPerThread; ++i) {
+        unsigned long long key[KPT];
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) {
             const int k = tid + i * kCT;
             unsigned long long v = ~0ull;
             if (k < n) {
@@ -46,10 +46,11 @@ __global__ void __launch_bounds__(kCT) compact_kernel(DecodeArgs a)
             key[i] = v;
         }
         for (int e = 0; e < E; ++e) {
+            // lowest rank key of the block: thread, warp, then the first warp over the warps' minima
             unsigned long long best = ~0ull;
             int bslot = -1;
-#pragma unroll 1
-            for (int i = 0; i < kMaxPerThread; ++i)
+#pragma unroll
+            for (int i = 0; i < KPT; ++i)
                 if (key[i] < best) { best = key[i]; bslot = tid + i * kCT; }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -59,12 +60,23 @@ __global__ void __launch_bounds__(kCT) compact_kernel(DecodeArgs a)
             }
             if (lane == 0) { red_key[warp] = best; red_slot[warp] = bslot; }
             __syncthreads();
-            best = red_key[0]; bslot = red_slot[0];
-            for (int w = 1; w < kCT / 32; ++w)
-                if (red_key[w] < best) { best = red_key[w]; bslot = red_slot[w]; }
-            if (tid == 0) ev_slot[e] = bslot;
-            if (bslot >= 0 && (bslot % kCT) == tid) key[bslot / kCT] = ~0ull;     // its owner retires it
+            if (warp == 0) {
+                best = red_key[lane]; bslot = red_slot[lane];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+                    const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+                    if (ok < best) { best = ok; bslot = os; }
+                }
+                if (lane == 0) ev_slot[e] = bslot;
+            }
             __syncthreads();
+            bslot = ev_slot[e];
+            if (bslot >= 0 && (bslot % kCT) == tid) {       // its owner retires it
+#pragma unroll
+                for (int i = 0; i < KPT; ++i)
+                    if (i == bslot / kCT) key[i] = ~0ull;
+            }
         }
         // holes: evicted slots inside the kept prefix; movers: surviving slots beyond it (both ascending)
         if (tid == 0) {
@@ -115,15 +127,23 @@ __global__ void __launch_bounds__(kCT) compact_kernel(DecodeArgs a)
 
 }  // namespace
 
+template <typename T, int D>
+static void launch_compact_t(const DecodeArgs &a, cudaStream_t stream)
+{
+    const int per = (a.cap + kCT - 1) / kCT;
+    if (per <= 2) compact_kernel<T, D, 2><<<a.U, kCT, 0, stream>>>(a);
+    else if (per <= 4) compact_kernel<T, D, 4><<<a.U, kCT, 0, stream>>>(a);
+    else if (per <= 8) compact_kernel<T, D, 8><<<a.U, kCT, 0, stream>>>(a);
+    else compact_kernel<T, D, 16><<<a.U, kCT, 0, stream>>>(a);
+}
+
 cudaError_t launch_compact(const DecodeArgs &a, bool f32, int D, cudaStream_t stream)
 {
-    if (a.T > 64 || (a.cap + kCT - 1) / kCT > kMaxPerThread) return cudaErrorInvalidConfiguration;
+    if (a.T > 64 || (a.cap + kCT - 1) / kCT > 16) return cudaErrorInvalidConfiguration;
     if (f32) {
-        if (D == 64) compact_kernel<float, 64><<<a.U, kCT, 0, stream>>>(a);
-        else compact_kernel<float, 128><<<a.U, kCT, 0, stream>>>(a);
+        if (D == 64) launch_compact_t<float, 64>(a, stream); else launch_compact_t<float, 128>(a, stream);
     } else {
-        if (D == 64) compact_kernel<__nv_bfloat16, 64><<<a.U, kCT, 0, stream>>>(a);
-        else compact_kernel<__nv_bfloat16, 128><<<a.U, kCT, 0, stream>>>(a);
+        if (D == 64) launch_compact_t<__nv_bfloat16, 64>(a, stream); else launch_compact_t<__nv_bfloat16, 128>(a, stream);
     }
     return cudaGetLastError();
 }
