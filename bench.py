@@ -43,7 +43,7 @@ def algorithmic_bytes_per_step(w: synth.Workload, n: int) -> int:
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
 # capture of a launch of that workload), valid only for the kernel sources it was taken with.
-_TRAFFIC = {"c1": {"bytes": 298.7e6, "sources_sha256": "3f17f99260dec2377fa0ea7a0fc5533205bff26d18b2923e2635f13074752b58"}}
+_TRAFFIC = {"c1": {"bytes": 284.7e6, "sources_sha256": "40e48f1c589ba996fbf3cdc5e61fa3521e2d08ad4f58332db401e35dee990d98"}}
 
 
 def measured_traffic(workload: str):
