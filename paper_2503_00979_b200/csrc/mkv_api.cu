@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <initializer_list>
 #include <new>
 
@@ -15,7 +16,7 @@ using namespace mkv;
 namespace {
 
 struct Layout {
-    size_t K, V, pos, ring_q, ring_c, s_new, F, part_ml, part_o, ticket, evicted, state, stage_q, stage_k, stage_v,
+    size_t K, V, pos, ring_q, ring_c, s_new, F, Fc, part_ml, part_o, ticket, evicted, state, stage_q, stage_k, stage_v,
         stage_o, total;
 };
 
@@ -26,6 +27,7 @@ struct Shape {
     int upl;                // units per layer = batch * n_kv_heads
     int U, G, D, R, C, cap, splits, T, tc_grid_size, tc_grid_layer;
     int Gq;                 // the model's GQA ratio; G is it rounded up to a power of two on the tensor-core path
+    int nc;                 // ring chunks of the tensor-core kernel (1 unless the window has more than 256 rows)
     size_t es;
 };
 
@@ -42,6 +44,7 @@ Layout make_layout(const Shape &s)
     L.ring_c = take(U * R * G * 4);
     L.s_new = take(U * G * cap * 4);
     L.F = take(U * cap * 4);
+    L.Fc = take(s.nc > 1 ? U * (size_t)s.nc * cap * 4 : 0);
     L.part_ml = take(U * sp * G * 2 * 4);
     L.part_o = take(U * sp * G * D * 4);
     L.ticket = take(U * 4);
@@ -91,21 +94,27 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     // with T > 1 the step that runs the policy appends first and evicts afterwards: one more slot
     s->cap = p->C + p->R + (s->T > 1 ? s->T : 0);
     s->es = p->dtype == MKV_DTYPE_F32 ? 4 : 2;
+    s->nc = 1;
     if (s->T > 64) return false;
     if (p->norm_mode == MKV_NORM_CURRENT && s->T > 1) return false;     // the compaction drops several tokens at once
+    const int nc = tc_ring_chunks(s->G, s->R);
     const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R) &&
-                       (long long)s->U * ((s->cap + 127) / 128) <= (1ll << 30);     // tile indices stay 32-bit
+                       (long long)s->U * nc * ((s->cap + 127) / 128) <= (1ll << 30);     // tile indices stay 32-bit
     if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
     if (tc_ok && p->kernel != MKV_KERNEL_SIMT) {
         *kind = kKindTc;
         s->G = tc_padded_group(s->Gq);
+        s->nc = nc;       // a unit appears in the schedule once per ring chunk
         // the persistent grid (148 SMs on B200; correctness does not depend on the count)
-        s->tc_grid_size = tc_grid(s->U, s->cap, p->splits, 148);
+        s->tc_grid_size = tc_grid(s->U * nc, s->cap, p->splits, 148);
         // a per-layer call sees only a layer's units: ranges of about an eighth of a unit's tiles, so that a layer
         // of few units still spreads over the SMs while a unit stays within eight CTAs
-        s->tc_grid_layer = tc_grid(s->upl, s->cap, p->splits > 0 ? p->splits : 8, 148);
-        const int sp_all = tc_partials_per_unit(s->U, s->cap, s->tc_grid_size);
-        const int sp_layer = tc_partials_per_unit(s->upl, s->cap, s->tc_grid_layer);
+        s->tc_grid_layer = tc_grid(s->upl * nc, s->cap, p->splits > 0 ? p->splits : 8, 148);
+        // on a step without a policy decision only the main chunks are walked: take the worse of both schedules
+        const int sp_all = std::max(tc_partials_per_unit(s->U * nc, s->cap, s->tc_grid_size),
+                                    tc_partials_per_unit(s->U, s->cap, s->tc_grid_size));
+        const int sp_layer = std::max(tc_partials_per_unit(s->upl * nc, s->cap, s->tc_grid_layer),
+                                      tc_partials_per_unit(s->upl, s->cap, s->tc_grid_layer));
         s->splits = sp_all > sp_layer ? sp_all : sp_layer;
         return true;
     }
@@ -159,6 +168,7 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.ring_q = b + c->L.ring_q; a.ring_c = (float *)(b + c->L.ring_c);
     a.q = q; a.k_new = k; a.v_new = v; a.out = out;
     a.s_new = (float *)(b + c->L.s_new); a.F = (float *)(b + c->L.F);
+    a.Fc = c->s.nc > 1 ? (float *)(b + c->L.Fc) : nullptr; a.nc = c->s.nc;
     a.part_ml = (float *)(b + c->L.part_ml); a.part_o = (float *)(b + c->L.part_o);
     a.ticket = (int *)(b + c->L.ticket); a.evicted_pos = (int *)(b + c->L.evicted);
     a.st = (DevState *)(b + c->L.state);
@@ -192,6 +202,7 @@ DecodeArgs make_args_layer(const mkv_ctx *c, int layer, const void *q, const voi
     a.pos += u0 * s.cap;
     a.ring_q = (char *)a.ring_q + u0 * s.R * s.G * s.D * s.es; a.ring_c += u0 * s.R * s.G;
     a.s_new += u0 * s.G * s.cap; a.F += u0 * s.cap;
+    if (a.Fc) a.Fc += u0 * s.nc * s.cap;
     a.part_ml += u0 * s.splits * s.G * 2; a.part_o += u0 * s.splits * s.G * s.D;
     a.ticket += u0; a.evicted_pos += u0;
     a.st = a.st + 1 + layer;

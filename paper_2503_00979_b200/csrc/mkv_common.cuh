@@ -52,6 +52,8 @@ struct DecodeArgs {
                                // and the kernels work with, is Gq rounded up to a power of two on the tensor-core path:
                                // heads Gq .. G-1 have a zero query and normaliser +inf (weight 0) and produce no output
     float scale2;              // log2(e) / sqrt(D)
+    float *Fc;                 // [U][nc][cap]  tensor-core kernel with a window of nc > 1 ring chunks: the fused score of
+    int nc;                    // each chunk's rows, combined by the unit's epilogue; unused (nullptr, 1) otherwise
 };
 
 __device__ __forceinline__ float ldf(const float *p) { return *p; }

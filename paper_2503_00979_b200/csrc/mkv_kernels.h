@@ -13,12 +13,15 @@ int simt_default_splits(int U, int cap);
 // restores the dense prefix of C + R slots; a no-op after the other steps.  Launched after every decode step.
 cudaError_t launch_compact(const DecodeArgs &a, bool f32, int D, cudaStream_t stream);
 
-// Tensor-core (tcgen05) decode step: bf16, head_dim 128, GQA group in {1,2,4,8,16} and
-// R*G padded to a multiple of 32 at most 256.  The plan holds the TMA tensor maps of a
-// context's arena and the launch geometry; `a.splits` must be tc_partials_per_unit()
-// of the grid (every CTA that holds tiles of a unit leaves one partial).
+// Tensor-core (tcgen05) decode step: bf16, head_dim 128, GQA group padded to {1,2,4,8,16}.  A window of up to
+// 256 ring rows (R * padded group) is one MMA operand; a larger one is cut into tc_ring_chunks() chunks of equal
+// width, and a unit then appears in the kernel's schedule once per chunk (U * chunks "virtual units": pass that
+// count to tc_grid() and tc_partials_per_unit()).  The plan holds the TMA tensor maps of a context's arena and
+// the launch geometry; `a.splits` must be tc_partials_per_unit() of the grid (every CTA that holds tiles of a
+// unit leaves one partial).
 bool tc_shape_supported(bool f32, int D, int G, int R);
 int tc_padded_group(int G);
+int tc_ring_chunks(int G, int R);
 int tc_grid(int U, int cap, int splits_hint, int n_sm);
 int tc_partials_per_unit(int U, int cap, int grid);
 struct TcPlan;

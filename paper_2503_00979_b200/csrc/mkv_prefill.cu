@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(kPT) prefill_logits_kernel(const T *__restrict
 
 // c = max + log2(sum exp2(s - max)) of one window row; stored in the ring row p % R.
 __global__ void __launch_bounds__(kPT) prefill_rowstats_kernel(const float *__restrict__ S, float *__restrict__ ring_c,
-                                                               int ub0, int P, int Rw, int G, int R)
+                                                               int ub0, int P, int Rw, int G, int Gs, int R)
 {
     __shared__ float red[kPT / 32];
     __shared__ float bc;
@@ -141,20 +141,20 @@ __global__ void __launch_bounds__(kPT) prefill_rowstats_kernel(const float *__re
         for (int w = 0; w < kPT / 32; ++w) x += red[w];
         const int i = row / G, g = row % G;
         const int rslot = (P - Rw + i) % R;
-        ring_c[((size_t)u * R + rslot) * G + g] = m + log2f(x);
+        ring_c[((size_t)u * R + rslot) * Gs + g] = m + log2f(x);     // Gs: heads per ring slot (G padded)
     }
 }
 
 // Eq. 4-6 with Algorithm 1's group sum: F[j] for every older prompt token j < P - Rw.
 __global__ void __launch_bounds__(kPT) prefill_fuse_kernel(const float *__restrict__ S, const float *__restrict__ ring_c,
-                                                           float *__restrict__ Fp, int ub0, int P, int Rw, int G, int R,
-                                                           int fusion)
+                                                           float *__restrict__ Fp, int ub0, int P, int Rw, int G, int Gs,
+                                                           int R, int fusion)
 {
     extern __shared__ float cs[];   // [Rw * G]
     const int u = ub0 + blockIdx.y, rows = Rw * G;
     for (int row = threadIdx.x; row < rows; row += kPT) {
         const int rslot = (P - Rw + row / G) % R;
-        cs[row] = ring_c[((size_t)u * R + rslot) * G + row % G];
+        cs[row] = ring_c[((size_t)u * R + rslot) * Gs + row % G];
     }
     __syncthreads();
     const int j = blockIdx.x * kPT + threadIdx.x;
@@ -326,7 +326,9 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
                           unsigned long long *launches, float *S, size_t scratch_floats, int n_states)
 {
     const int U = a.U, G = a.G, R = a.R, C = a.C;
-    const int Rw = P < R ? P : R, rows = Rw * G;
+    // the CUDA-core scoring kernels work on the model's Gq heads per window position (rows of S); the ring keeps G
+    // heads per slot, the padding heads with normaliser +inf from init_arena_kernel
+    const int Rw = P < R ? P : R, rows = Rw * a.Gq;
     const bool select = P - Rw > C;
     const int n = select ? C + Rw : P;
     if (n > a.cap) return cudaErrorInvalidValue;
@@ -334,7 +336,6 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     // others materialise the window-row logits S [rows][P] per unit and reduce them with CUDA-core kernels
     // (the arena's group must be the padded one: a context that runs the CUDA-core decode kernel keeps G as it is)
     const bool tc = prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P) && tc_padded_group(a.Gq) == G;
-    if (!tc && a.Gq != G) return cudaErrorInvalidValue;     // a padded group exists on the tensor-core path only
     const int tc_splits = tc ? prefill_tc_splits(U, P) : 0;
     const size_t per_unit = tc ? prefill_tc_floats_per_unit(P, Rw, G, tc_splits) : (size_t)rows * P + P;   // floats
     if (per_unit + 1 > scratch_floats) return cudaErrorInvalidConfiguration;
@@ -361,15 +362,15 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
             e = run_prefill_scores_tc(a, k, qwin, P, ub0, nb, tc_splits, Fp, part, err_word, launches, stream);
             if (e != cudaSuccess) return e;
         } else {
-            prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw, G,
-                                                                                                 a.scale2);
-            prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, G, R);
+            prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw,
+                                                                                                 a.Gq, a.scale2);
+            prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, a.Gq, G, R);
             *launches += 2;
         }
         if (select) {
             if (!tc) {
                 prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
-                    S, a.ring_c, Fp, ub0, P, Rw, G, R, a.fusion);
+                    S, a.ring_c, Fp, ub0, P, Rw, a.Gq, G, R, a.fusion);
                 ++*launches;
             }
             prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
@@ -384,7 +385,7 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
     prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
     if (a.norm_current && select) {
-        prefill_renorm_kernel<T, D><<<dim3(rows, U), kPT, 0, stream>>>(a, P, Rw, n);
+        prefill_renorm_kernel<T, D><<<dim3(Rw * G, U), kPT, 0, stream>>>(a, P, Rw, n);
         ++*launches;
     }
     set_state_kernel<<<1, 32, 0, stream>>>(a.st, n_states, (long long)P, n);

@@ -321,7 +321,7 @@ cudaError_t launch_pass_any(const PfArgs &a, const CUtensorMap &tm, int nb, int 
 
 bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P)
 {
-    return tc_shape_supported(f32, D, G, R) && ((uintptr_t)k & 15) == 0 && P >= 1;
+    return tc_shape_supported(f32, D, G, R) && tc_ring_chunks(G, R) == 1 && ((uintptr_t)k & 15) == 0 && P >= 1;
 }
 
 int prefill_tc_splits(int units_in_batch, int P)

@@ -1,5 +1,7 @@
-// Tensor-core decode kernel for sm_100a: bf16, head_dim 128, GQA group in {1,2,4,8,16},
-// R*G (padded to a multiple of 32) at most 256.
+// Tensor-core decode kernel for sm_100a: bf16, head_dim 128, GQA group in {1,2,4,8,16}.  Up to 256
+// ring rows (R*G, padded to a multiple of 32) are one MMA operand; a larger window is cut into
+// chunks of equal width and a unit is then scheduled once per chunk (template parameter MC, see the
+// kernel's prologue).
 //
 // The 128-key tiles of all units' caches form one sequence that is cut into equal contiguous
 // ranges, one per persistent, warp-specialised CTA; a work item is the run of a unit's tiles
@@ -52,7 +54,8 @@ constexpr int kFinFloats = 4 * kMaxGroup + 128 + 256 + 64 + 32 + 8;   // epilogu
 constexpr int kEpiFloats = kFinFloats + 8 + 2 * kMaxGroup + kMaxComputeWarps * kMaxGroup;
 
 struct TcGeom {
-    int rgpad;          // ring rows padded to a multiple of 32 (MMA N)
+    int rgpad;          // ring rows of one chunk, padded to a multiple of 32 (MMA N)
+    int nc;             // ring chunks (1 unless the window has more than 256 rows)
     int sk, sv;         // K stages, V stages
     int ng;             // compute groups; tile T belongs to group T % ng
     int nb;             // TMEM accumulator buffers (a multiple of ng)
@@ -355,7 +358,7 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     }
 }
 
-template <int G, int FUSION, int NG>
+template <int G, int FUSION, int NG, bool MC>
 __global__ void __launch_bounds__(tc_threads(NG), 1)
 decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
@@ -415,6 +418,14 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 
     const bool evict = step_scores(t, n, steps_done, a.R, a.C, a.T);
     const int rs_new = (int)(t % a.R);
+    // MC (a window of more than 256 ring rows): the ring is cut into geo.nc chunks of RGP rows = RGP / G ring
+    // slots, and the schedule walks U * nc "virtual units": virtual unit v is chunk v % nc of unit v / nc.  The
+    // chunk that holds the slot of the new query (the main chunk) does everything a unit does otherwise; the
+    // other chunks only score their rows against the unit's keys, into their own slab of a.Fc.  On a step that
+    // does not run the policy only the main chunks are walked.
+    const int NCe = MC ? (evict ? geo.nc : 1) : 1;               // chunks walked per unit on this step
+    const int c_main = MC ? rs_new / (RGP / G) : 0;
+    const int rs_loc = MC ? rs_new - c_main * (RGP / G) : rs_new;  // the new query's slot inside its chunk
     // Every thread of this CTA holds its copy of the step state (the barrier above orders their reads
     // before this point), so the CTA can be counted now: the last CTA of the launch to get here advances
     // the state for the next launch while the tiles stream, instead of at the tail of the kernel.
@@ -432,7 +443,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     if (warp == 0) {
         // ------------------------------------------------ TMA producer: query ring and K tiles (one lane)
         if (lane == 0) {
-            Walk w(a.U, n);
+            Walk w(a.U * NCe, n);
             Item x;
             int issued = 0, rings = 0;
             bool ok = true;
@@ -441,9 +452,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             while (ok && w.next(x)) {
                 ok = mbar_wait(bar_qempty, (uint32_t)((w.nitems & 1) ^ 1), abort_flag, kWaitQEmpty, WL);
                 if (!ok) break;
+                const int u = MC ? x.unit / NCe : x.unit;
+                const int qrow = MC ? (NCe == 1 ? c_main : x.unit - u * NCe) * RGP : 0;   // rows past R*G read as zero
                 mbar_expect_tx(bar_qfull, (uint32_t)(RGP * 256));
-                tma_load_3d(q_addr, &tmQ, 0, 0, a.u0 + x.unit, bar_qfull, pol_keep);
-                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, 0, a.u0 + x.unit, bar_qfull, pol_keep);
+                tma_load_3d(q_addr, &tmQ, 0, qrow, a.u0 + u, bar_qfull, pol_keep);
+                tma_load_3d(q_addr + RGP * 128, &tmQ, 64, qrow, a.u0 + u, bar_qfull, pol_keep);
                 ++rings;
                 for (int j = 0; j < x.nk && ok; ++j, rk.step(1, SK)) {
                     const int T = w.T0 + j, s = rk.idx;
@@ -451,8 +464,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_kfull + 8 * s, kStageBytes);
-                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, a.u0 + x.unit, bar_kfull + 8 * s, pol_stream);
-                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, a.u0 + x.unit, bar_kfull + 8 * s, pol_stream);
+                    tma_load_3d(kst_addr + s * kStageBytes, &tmK, 0, row, a.u0 + u, bar_kfull + 8 * s, pol_stream);
+                    tma_load_3d(kst_addr + s * kStageBytes + kStageBytes / 2, &tmK, 64, row, a.u0 + u, bar_kfull + 8 * s, pol_stream);
                     issued = T + 1;
                 }
                 w.advance(x);
@@ -470,22 +483,24 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     } else if (warp == 2) {
         // ------------------------------------------------ TMA producer: V tiles (one lane)
         if (lane == 0) {
-            Walk w(a.U, n);
+            Walk w(a.U * NCe, n);
             Item x;
-            int issued = 0;
+            int issued = 0;                                 // V tiles loaded so far (only main chunks read V)
             bool ok = true;
             RingPos rv(0, SV);
             const uint64_t pol_stream = l2_policy_evict_first();
             while (ok && w.next(x)) {
-                for (int j = 0; j < x.nk && ok; ++j, rv.step(1, SV)) {
-                    const int T = w.T0 + j, s = rv.idx;
+                const int u = MC ? x.unit / NCe : x.unit;
+                const bool main_item = MC ? (NCe == 1 || x.unit - u * NCe == c_main) : true;
+                for (int j = 0; main_item && j < x.nk && ok; ++j, rv.step(1, SV)) {
+                    const int s = rv.idx;
                     ok = mbar_wait(bar_vempty + 8 * s, (uint32_t)(rv.lap ^ 1), abort_flag, kWaitVEmpty, WL);
                     if (!ok) break;
                     const int row = (x.tile0 + j) * kTile;
                     mbar_expect_tx(bar_vfull + 8 * s, kStageBytes);
-                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, a.u0 + x.unit, bar_vfull + 8 * s, pol_stream);
-                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, a.u0 + x.unit, bar_vfull + 8 * s, pol_stream);
-                    issued = T + 1;
+                    tma_load_3d(vst_addr + s * kStageBytes, &tmV, 0, row, a.u0 + u, bar_vfull + 8 * s, pol_stream);
+                    tma_load_3d(vst_addr + s * kStageBytes + kStageBytes / 2, &tmV, 64, row, a.u0 + u, bar_vfull + 8 * s, pol_stream);
+                    ++issued;
                 }
                 w.advance(x);
             }
@@ -498,7 +513,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         __syncwarp();       // see the K producer
     } else if (warp == 1) {
         // ------------------------------------------------ new-query substitution + MMA issue
-        Walk w(a.U, n);
+        Walk w(a.U * NCe, n);
         Item x;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RGP >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
         bool ok = true;
@@ -508,8 +523,10 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             {
                 if (w.nitems > 0 && lane == 0) umma_commit(bar_qempty);   // MMAs of the previous unit done with the ring
                 // the new query replaces ring row t % R (the row of the token leaving the window)
+                const int u = MC ? x.unit / NCe : x.unit;
+                const bool main_item = MC ? (NCe == 1 || x.unit - u * NCe == c_main) : true;   // the chunk with the new query's slot
                 uint4 qv[kMaxGroup / 2];
-                const uint4 *qsrc = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(a.q) + (size_t)x.unit * a.Gq * kD);
+                const uint4 *qsrc = reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(a.q) + (size_t)u * a.Gq * kD);
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i)
                     if (lane + 32 * i < G * 16) qv[i] = lane + 32 * i < a.Gq * 16 ? qsrc[lane + 32 * i] : make_uint4(0, 0, 0, 0);
@@ -518,8 +535,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 #pragma unroll
                 for (int i = 0; i < (G * 16 + 31) / 32; ++i) {
                     const int c = lane + 32 * i;
-                    if (c < G * 16) {
-                        const int row = rs_new * G + c / 16, ch = c % 16;
+                    if (c < G * 16 && main_item) {
+                        const int row = rs_loc * G + c / 16, ch = c % 16;
                         const uint32_t off = (uint32_t)((ch >> 3) * (RGP * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4));
                         *reinterpret_cast<uint4 *>(smem + L.q + off) = qv[i];
                     }
@@ -588,18 +605,22 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         int seg_tiles = 0;
         int npub = 0;                                  // partials this warp has handed to the epilogue group
 
-        Walk w(a.U, n);
+        Walk w(a.U * NCe, n);
         Item x;
         bool ok = true;
         int Tn = grp;                                  // next tile of this group
+        int skipped = 0;                               // MC: tiles of the items that read no V
         RingPos rb(grp, NB), rv(grp, SV);
         while (w.next(x)) {
-            const int u = x.unit;
+            const int u = MC ? x.unit / NCe : x.unit;
+            const int cc = MC ? (NCe == 1 ? c_main : x.unit - u * NCe) : 0;      // ring chunk of this item
+            const bool main_item = MC ? cc == c_main : true;
             {
                 // frozen normalisers of the ring rows, negated; the new row and padding give weight 0
                 for (int c = lane; c < RGP; c += 32) {
                     float v = -INFINITY;
-                    if (c < RG && c / G != rs_new) v = -a.ring_c[(size_t)u * RG + c];
+                    const int row = MC ? cc * RGP + c : c;
+                    if (row < RG && row / G != rs_new) v = -a.ring_c[(size_t)u * RG + row];
                     negc[c] = v;
                 }
 #pragma unroll
@@ -614,8 +635,35 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 __syncwarp();
             }
             float *s_new = a.s_new + (size_t)u * G * a.cap;
+            float *Fdst = MC ? a.Fc + ((size_t)u * geo.nc + cc) * a.cap : a.F + (size_t)u * a.cap;
+            if constexpr (MC) {
+                if (main_item) {
+                    rv = RingPos(Tn - skipped, SV);      // V tiles are numbered over the main items only
+                } else {
+                    // a chunk without the new query: fused scores of its rows over this group's tiles, nothing else
+                    for (; Tn < w.T0 + x.nk && ok; Tn += NG, rb.step(NG, NB)) {
+                        const int buf = rb.idx;
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, (uint32_t)rb.lap, abort_flag, kWaitTFull, WL));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const int key = (x.tile0 + (Tn - w.T0)) * kTile + gtid;
+                        const uint32_t taddr = tmem_base + (uint32_t)(buf * RGP) + ((uint32_t)(wq * 32) << 16);
+                        float F = 0.f;
+                        for (int c = 0; c < RGP; c += 32) {
+                            uint32_t v[32];
+                            tmem_ld32(taddr + (uint32_t)c, v);
+                            score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
+                        }
+                        if (key < n) Fdst[key] = F;
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                    }
+                    skipped += x.nk;
+                }
+            }
             // this group's tiles are T = grp, grp + NG, ...: walk them directly
-            for (; Tn < w.T0 + x.nk && ok; Tn += NG, rb.step(NG, NB), rv.step(NG, SV)) {
+            for (; main_item && Tn < w.T0 + x.nk && ok; Tn += NG, rb.step(NG, NB), rv.step(NG, SV)) {
                 const int j = Tn - w.T0;
                 const int buf = rb.idx;
                 // ---- scores of this warp's 32 keys (Eq. 4-6) and the new row's logits
@@ -628,7 +676,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 // Each TMEM load and its wait form one asm statement: the destination registers are
                 // written asynchronously, so nothing may touch them between the two.
                 uint32_t sv[G];
-                tmem_ld_n<G>(taddr + (uint32_t)(rs_new * G), sv);
+                tmem_ld_n<G>(taddr + (uint32_t)(rs_loc * G), sv);
 
                 // ---- online soft-max of the new row over this warp's keys (Eq. 1)
                 bool changed = false;
@@ -724,7 +772,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                         tmem_ld32(taddr + (uint32_t)c, v);
                         score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
                     }
-                    if (valid) a.F[(size_t)u * a.cap + key] = F;
+                    if (valid) Fdst[key] = F;
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -739,7 +787,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 if (npub > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * cw, (uint32_t)((npub - 1) & 1), abort_flag, kWaitPFree, WL));
                 if (ok) {
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
+                    for (int nt = 0; nt < NT && main_item; ++nt) {
                         const int gr = gid + 8 * nt, gc = tig * 2 + 8 * nt;
                         float l = lsum[nt];
                         l += __shfl_xor_sync(0xffffffffu, l, 1);
@@ -779,16 +827,17 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         int *flag = reinterpret_cast<int *>(epi + kFinFloats);
         float *cml = epi + kFinFloats + 8;                            // merged (m, l) [g][2]
         float *sc = cml + 2 * kMaxGroup;                              // [warp][g] scale to the merged reference
-        Walk w(a.U, n);
+        Walk w(a.U * NCe, n);
         Item x;
         bool ok = true;
         int k = 0;                                                    // units finished so far
         while (ok && w.next(x)) {
             {
-                const int u = x.unit;
+                const int u = MC ? x.unit / NCe : x.unit;
+                const bool main_item = MC ? (NCe == 1 || x.unit - u * NCe == c_main) : true;
                 if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag, kWaitUDone, WL))) { ok = false; break; }
                 // merge the compute warps' partials: common reference = max of theirs
-                if (etid < G) {
+                if (etid < G && main_item) {
                     float m = -INFINITY;
                     for (int cwi = 0; cwi < NCW; ++cwi) m = fmaxf(m, wml[cwi * 2 * kMaxGroup + etid * 2]);
                     float l = 0.f;
@@ -813,8 +862,44 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 group_sync(kEpiBar, kGroupThreads);                       // every warp buffer has been read
                 if (etid < NCW) mbar_arrive(bar_pfree + 8 * etid);
                 int my_index;
-                const int ncta = w.ctas_of_unit(u, my_index);
-                if (ncta == 1) {
+                const int ncta = w.ctas_of_unit(x.unit, my_index);
+                if constexpr (MC) {
+                    // Every (CTA, chunk) item of a unit takes one ticket; the items of the main chunk publish their
+                    // partial of the attention output first.  The last item of the unit combines the chunks' fused
+                    // scores and finishes the unit with the general epilogue.
+                    if (main_item) {
+                        float *pml = a.part_ml + ((size_t)u * a.splits + my_index) * G * 2;
+                        float *po = a.part_o + ((size_t)u * a.splits + my_index) * G * kD;
+#pragma unroll
+                        for (int g = 0; g < G; ++g) po[g * kD + etid] = o[g];
+                        if (etid < 2 * G) pml[etid] = cml[etid];
+                    }
+                    group_sync(kEpiBar, kGroupThreads);
+                    if (etid == 0) {
+                        int items = 0, idx;
+                        for (int c = 0; c < NCe; ++c) items += w.ctas_of_unit(u * NCe + c, idx);
+                        __threadfence();
+                        const int last = atomicAdd(&a.ticket[u], 1) == items - 1;
+                        __threadfence();
+                        *flag = last;
+                    }
+                    group_sync(kEpiBar, kGroupThreads);
+                    if (*flag) {
+                        if (evict) {
+                            float *F = a.F + (size_t)u * a.cap;
+                            const float *Fc = a.Fc + (size_t)u * geo.nc * a.cap;
+                            for (int key = etid; key < n; key += kGroupThreads) {
+                                float f = __ldcg(Fc + key);
+                                for (int c = 1; c < NCe; ++c) f = fuse(FUSION, f, __ldcg(Fc + (size_t)c * a.cap + key));
+                                F[key] = f;
+                            }
+                            group_sync(kEpiBar, kGroupThreads);
+                        }
+                        int idx;
+                        const int ncta_main = w.ctas_of_unit(u * NCe + (NCe == 1 ? 0 : c_main), idx);
+                        finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, ncta_main, evict, fin_sm, etid, kGroupThreads, kEpiBar);
+                    }
+                } else if (ncta == 1) {
                     finalize_fast<G, true>(a, u, t, n, 1, evict, fin_sm, etid, kEpiBar, o, cml);
                 } else {
                     // the unit is shared: publish this CTA's partial; the last CTA to do so finishes the unit.
@@ -863,18 +948,18 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 struct TcPlan {
     CUtensorMap tmK, tmV, tmQ;
     TcGeom geo;
-    bool attr_set[5][2];
+    bool attr_set[5][2][2];
 };
 
 namespace {
 
 int group_index(int G) { return G == 1 ? 0 : G == 2 ? 1 : G == 4 ? 2 : G == 8 ? 3 : G == 16 ? 4 : -1; }
 
-template <int G, int FUSION, int NG>
+template <int G, int FUSION, int NG, bool MC>
 cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    auto kern = decode_tc_kernel<G, FUSION, NG>;
-    bool &set = plan->attr_set[group_index(G)][FUSION];
+    auto kern = decode_tc_kernel<G, FUSION, NG, MC>;
+    bool &set = plan->attr_set[group_index(G)][FUSION][MC ? 1 : 0];
     if (!set) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan->geo.smem_bytes);
         if (e != cudaSuccess) return e;
@@ -898,7 +983,8 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 template <int G, int FUSION>
 cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    return launch_gfn<G, FUSION, kComputeGroups>(plan, a, stream);
+    return plan->geo.nc > 1 ? launch_gfn<G, FUSION, kComputeGroups, true>(plan, a, stream)
+                            : launch_gfn<G, FUSION, kComputeGroups, false>(plan, a, stream);
 }
 
 template <int G>
@@ -918,11 +1004,29 @@ int tc_padded_group(int G)
     return g;
 }
 
+// Chunks the recent-query ring is cut into: one MMA takes at most 256 ring rows (N of the instruction, and with
+// two accumulator buffers the 512 TMEM columns).
+int tc_ring_chunks(int G, int R)
+{
+    const int rows = R * tc_padded_group(G);
+    return rows <= 256 ? 1 : (rows + 255) / 256;
+}
+
+namespace {
+constexpr int kMaxRingChunks = 8;
+// rows of one chunk: the chunks are made equally wide (a multiple of 32, hence of the padded group)
+int chunk_rows(int G, int R)
+{
+    const int rows = R * tc_padded_group(G), nc = tc_ring_chunks(G, R);
+    return pad32((rows + nc - 1) / nc);
+}
+}  // namespace
+
 // G: the model's GQA ratio; the kernel works with the group padded to a power of two
 bool tc_shape_supported(bool f32, int D, int G, int R)
 {
-    if (f32 || D != kD || G < 1 || G > kMaxGroup) return false;
-    return pad32(R * tc_padded_group(G)) <= 256;
+    if (f32 || D != kD || G < 1 || G > kMaxGroup || R < 1) return false;
+    return tc_ring_chunks(G, R) <= kMaxRingChunks;
 }
 
 // Grid of the persistent kernel.  `splits_hint` > 0 asks for about that many CTAs per unit
@@ -971,7 +1075,13 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned
     if (e != cudaSuccess) { delete p; return e; }
     TcGeom &g = p->geo;
     const int G = a.G;
-    g.rgpad = pad32(a.R * G);
+    g.nc = a.nc;
+    g.rgpad = g.nc > 1 ? chunk_rows(a.Gq, a.R) : pad32(a.R * G);
+    if (g.nc != tc_ring_chunks(a.Gq, a.R) || g.rgpad > 256 || g.rgpad * g.nc < a.R * G || (g.nc > 1 && !a.Fc)) {
+        snprintf(err, err_len, "tensor-core kernel: ring chunk geometry does not match the shape");
+        delete p;
+        return cudaErrorInvalidValue;
+    }
     g.ng = kComputeGroups;
     g.nb = g.rgpad <= 128 ? 4 : 2;
     g.tmem_cols = 32;
@@ -990,6 +1100,7 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned
         return cudaErrorInvalidConfiguration;
     }
     g.sk = total_stages >= 7 ? 3 : total_stages >= 5 ? 2 : 1;
+    if (g.nc > 1 && total_stages >= 4) g.sk = 2;      // most items of a chunked window read K only
     g.sv = total_stages - g.sk;
     g.smem_bytes = tc_smem_layout(g, G).total + 1024;
     if (!encode_map(&p->tmK, a.K, a.U, a.cap, kTile) || !encode_map(&p->tmV, a.V, a.U, a.cap, kTile) ||

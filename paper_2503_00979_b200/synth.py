@@ -122,6 +122,10 @@ for _C in (512, 1024, 2048, 4096, 8192):
 for _P in (6144, 32768, 131072):
     WORKLOADS[f"prefill_P{_P}"] = Workload(f"prefill_P{_P}", 32, 1, 32, 8, 128, "bf16", _P, 8, 2016, 32, "sum", _SEED0 + 5)
 
+# the long-response setting with a window of 200 recent tokens inside a 4K budget, on the Llama-3.1-8B-shaped stack:
+# 800 ring rows per unit, more than one tensor-core operand holds
+WORKLOADS["w200"] = Workload("w200", 32, 1, 32, 8, 128, "bf16", 4096, 4096, 3896, 200, "sum", _SEED0 + 6)
+
 
 class Stream:
     """Counter-based generator of a workload's q/k/v at arbitrary positions.

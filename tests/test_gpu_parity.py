@@ -182,10 +182,17 @@ def test_auto_picks_the_tensor_core_kernel_for_bf16_d128():
     assert mk.kernel_name == "tc" and mk.view(0)["ring_c"].shape[-1] == 8
     mk.close()
     p = binding.mkv_default_params()
-    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 14, 2, 128, 64, 40     # 40 * 8 rows > 256
+    mk = binding.MorphKV(1, 1, 14, 2, 128, 64, 40, "sum", "bf16")      # 40 * 8 = 320 ring rows: two chunks
+    assert mk.kernel_name == "tc"
+    mk.close()
+    p = binding.mkv_default_params()
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 14, 2, 128, 64, 300    # 2400 rows: more than 8 chunks
     p.kernel = binding.KERNEL["tc"]
     st, h = binding.mkv_create_ex(p)
     assert st == binding.UNSUPPORTED and h is None
+    mk = binding.MorphKV(1, 1, 14, 2, 128, 64, 300, "sum", "bf16")
+    assert mk.kernel_name == "simt"
+    mk.close()
 
 
 @pytest.mark.parametrize("fusion", ["sum", "max"])
@@ -288,12 +295,44 @@ def test_full_size_config1_coarse_grained_launched_back_to_back():
     mk.close()
 
 
-def test_longgenbench_shape_window_200_uses_the_cuda_core_kernel():
-    # R = 200 with a 4K budget (the LongGenBench setting): R*G = 800 rows do not fit the tensor-core kernel
-    w = synth.Workload("r200", 1, 1, 8, 2, 128, "bf16", 4200, 24, 3896, 200, "sum", 31)
-    rep = run_parity(w, steps=w.steps, n_units=2, kernel="auto", check_F_every=8)
+@pytest.mark.parametrize("kernel", ["auto", "simt"])
+def test_longgenbench_shape_window_200(kernel):
+    # R = 200 with a 4K budget (the LongGenBench setting): R*G = 800 ring rows.  The tensor-core kernel cuts the ring
+    # into four chunks of 56 slots; the prompt length makes the new query's slot cross from chunk 0 to chunk 1.
+    w = synth.Workload("r200", 1, 1, 8, 2, 128, "bf16", 4250, 24, 3896, 200, "sum", 31)
+    rep = run_parity(w, steps=w.steps, n_units=2, kernel=kernel, check_F_every=8)
     _report(rep)
-    assert rep.kernel == "simt" and rep.evictions == 2 * 24
+    assert rep.kernel == ("tc" if kernel == "auto" else "simt") and rep.evictions == 2 * 24
+
+
+@pytest.mark.parametrize("q_heads,kv_heads,R,C,P,fusion", [(14, 2, 40, 300, 420, "max"),     # group 7 -> 8, two chunks of 20 slots
+                                                           (8, 2, 65, 300, 300, "sum"),      # 260 rows: chunks of 160; starts in the fill phase
+                                                           (32, 2, 33, 200, 300, "max"),     # group 16, three chunks
+                                                           (2, 2, 300, 700, 1100, "sum")])   # MHA, window 300: two chunks
+def test_windows_of_more_than_256_ring_rows_on_the_tensor_cores(q_heads, kv_heads, R, C, P, fusion):
+    # many small units (several work items per CTA) as well as units shared by several CTAs; prompts shorter than
+    # C + R start in the fill phase, where only the chunk with the new query's slot is walked
+    w = synth.Workload("wide", 2, 2, q_heads, kv_heads, 128, "bf16", P, 2 * R + 9, C, R, fusion, 77 + R)
+    rep = run_parity(w, steps=w.steps, n_units=8, kernel="auto", check_F_every=5)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+
+
+def test_wide_window_with_per_layer_calls_and_current_normalisation():
+    w = synth.Workload("wide_layer", 3, 1, 8, 2, 128, "bf16", 500, 90, 400, 70, "sum", 5)
+    rep = run_parity(w, steps=w.steps, n_units=6, kernel="auto", per_layer=1)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+    rep = run_parity(w, steps=w.steps, n_units=6, kernel="auto", norm="current")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+
+
+def test_wide_window_with_coarse_grained_eviction():
+    w = synth.Workload("wide_coarse", 1, 2, 8, 2, 128, "bf16", 700, 40, 500, 80, "max", 4243)
+    rep = run_parity_coarse(w, 4, steps=5 * 4 + 2, n_units=4, kernel="tc")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions == 4 * 5 * 4
 
 
 # ---- coarse-grained eviction: the policy runs every T-th step and drops several tokens at once
