@@ -43,7 +43,7 @@ def algorithmic_bytes_per_step(w: synth.Workload, n: int) -> int:
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
 # capture of a launch of that workload), valid only for the kernel sources it was taken with.
-_TRAFFIC = {"c1": {"bytes": 284.7e6, "sources_sha256": "40e48f1c589ba996fbf3cdc5e61fa3521e2d08ad4f58332db401e35dee990d98"}}
+_TRAFFIC = {"c1": {"bytes": 284.1e6, "sources_sha256": "7435109163d3524ba9fb9fa3e894339858d2d30986238975b980e87251ce04da"}}
 
 
 def measured_traffic(workload: str):

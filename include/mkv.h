@@ -171,6 +171,26 @@ mkv_status mkv_reset(mkv_ctx *ctx);
 mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
                               int prompt_len, void *stream);
 
+/* Prompt phase of a batch whose rows have prompts of different lengths (the paper's runs use one length per
+ * batch; a serving batch does not).  Tensors are padded to padded_len tokens: k, v
+ * [layers][batch][n_kv_heads][padded_len][head_dim], of which row b's first prompt_len[b] tokens are read;
+ * q_window [layers][batch][n_q_heads][min(R, padded_len)][head_dim], of which row b's first
+ * min(R, prompt_len[b]) entries are the queries of its last prompt positions, oldest first.  prompt_len is a HOST
+ * array of `batch` lengths, each in [1, padded_len].  Every row ends up exactly as mkv_prefill with its own length
+ * would leave it (Algorithm 1 once over the row's prompt), and every later decode step appends one token to every
+ * row: row b's token of step s has position prompt_len[b] + s, its window, eviction decisions and cache fill are
+ * its own.  mkv_view.count is then the largest fill among the rows and mkv_view.next_pos the longest row's
+ * position; mkv_row_state reports each row.  Rows are processed one by one with the CUDA-core scoring kernels
+ * (set-up speed, not tuned).  Not available (MKV_UNSUPPORTED) together with evict_interval > 1 or with a window
+ * of more than 256 ring rows on the tensor-core kernel.  Synchronises the stream before returning. */
+mkv_status mkv_prefill_ragged(mkv_ctx *ctx, const void *k, const void *v, const void *q_window,
+                              const int32_t *prompt_len, int padded_len, void *stream);
+
+/* Cached tokens (count[b]) and position of the next token (next_pos[b]) of every batch row as `layer` holds them
+ * now; HOST arrays of `batch` entries, either may be NULL.  Reads the host mirror only (call mkv_sync first if
+ * steps were replayed from a CUDA graph).  All rows are equal unless the context was loaded by mkv_prefill_ragged. */
+mkv_status mkv_row_state(mkv_ctx *ctx, int layer, int32_t *count, int64_t *next_pos);
+
 /* One decode step for every unit (Eq. 1, Eq. 4-7, Algorithm 1): q, out
  * [layers][batch][n_q_heads][head_dim]; k_new, v_new [layers][batch][n_kv_heads][head_dim].
  * Asynchronous; launches a fixed kernel sequence with no host-side dependence on the step

@@ -26,7 +26,7 @@ NORM = {"frozen": 0, "current": 1}
 
 EXPORTS = [
     "mkv_default_params", "mkv_workspace_bytes", "mkv_create", "mkv_create_ex", "mkv_destroy", "mkv_reset", "mkv_prefill",
-    "mkv_prefill_static",
+    "mkv_prefill_static", "mkv_prefill_ragged", "mkv_row_state",
     "mkv_decode_step", "mkv_decode_step_layer", "mkv_decode_steps", "mkv_decode_step_host", "mkv_cache_view", "mkv_sync", "mkv_last_error",
     "mkv_launch_count", "mkv_kernel_name",
 ]
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         L.mkv_reset.argtypes = [vp]
         L.mkv_prefill.argtypes = [vp, vp, vp, vp, ip, vp]
         L.mkv_prefill_static.argtypes = [vp, vp, vp, vp, ip, vp]
+        L.mkv_prefill_ragged.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int32), ip, vp]
+        L.mkv_row_state.argtypes = [vp, ip, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
         L.mkv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
         L.mkv_decode_step_layer.argtypes = [vp, ip, vp, vp, vp, vp, vp]
         L.mkv_decode_steps.argtypes = [vp, vp, vp, vp, vp, ip, vp]
@@ -143,6 +145,19 @@ def mkv_reset(ctx) -> int:
 
 def mkv_prefill(ctx, k, v, q_window, prompt_len, stream=None) -> int:
     return lib().mkv_prefill(ctx, _ptr(k), _ptr(v), _ptr(q_window), prompt_len, _stream(stream))
+
+
+def mkv_prefill_ragged(ctx, k, v, q_window, prompt_lens, padded_len, stream=None) -> int:
+    """Prompt phase of a batch whose rows have different prompt lengths (tensors padded to padded_len)."""
+    lens = (C.c_int32 * len(prompt_lens))(*[int(x) for x in prompt_lens])
+    return lib().mkv_prefill_ragged(ctx, _ptr(k), _ptr(v), _ptr(q_window), lens, padded_len, _stream(stream))
+
+
+def mkv_row_state(ctx, layer, batch):
+    """(status, counts, next positions) of the batch rows as `layer` holds them."""
+    cnt, nxt = (C.c_int32 * batch)(), (C.c_int64 * batch)()
+    st = lib().mkv_row_state(ctx, layer, cnt, nxt)
+    return st, list(cnt), list(nxt)
 
 
 def mkv_prefill_static(ctx, k, v, q_window, prompt_len, stream=None) -> int:
@@ -258,6 +273,18 @@ class MorphKV:
 
     def prefill(self, k, v, q_window, stream=None):
         self._check(mkv_prefill(self.ctx, k, v, q_window, k.shape[-2], stream), "mkv_prefill")
+
+    def prefill_ragged(self, k, v, q_window, prompt_lens, stream=None):
+        """Prompt phase with one prompt length per batch row; k, v are padded to k.shape[-2] tokens."""
+        if len(prompt_lens) != self.shape["B"]:
+            raise ValueError("one prompt length per batch row")
+        self._check(mkv_prefill_ragged(self.ctx, k, v, q_window, prompt_lens, k.shape[-2], stream), "mkv_prefill_ragged")
+
+    def row_state(self, layer: int):
+        """(cached tokens, next position) of every batch row in `layer`."""
+        st, cnt, nxt = mkv_row_state(self.ctx, layer, self.shape["B"])
+        self._check(st, "mkv_row_state")
+        return cnt, nxt
 
     def prefill_static(self, k, v, q_window, stream=None):
         """Prompt phase for hosts that cannot allocate device memory; see mkv_prefill_static in mkv.h."""

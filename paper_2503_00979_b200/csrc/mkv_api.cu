@@ -16,7 +16,7 @@ using namespace mkv;
 namespace {
 
 struct Layout {
-    size_t K, V, pos, ring_q, ring_c, s_new, F, Fc, part_ml, part_o, ticket, evicted, state, stage_q, stage_k, stage_v,
+    size_t K, V, pos, ring_q, ring_c, s_new, F, Fc, part_ml, part_o, ticket, evicted, state, rows, row_shift, stage_q, stage_k, stage_v,
         stage_o, total;
 };
 
@@ -25,6 +25,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct Shape {
     int layers;             // layers served by this context's own arena
     int upl;                // units per layer = batch * n_kv_heads
+    int B, Hkv;             // batch rows and KV heads (upl = B * Hkv)
     int U, G, D, R, C, cap, splits, T, tc_grid_size, tc_grid_layer;
     int Gq;                 // the model's GQA ratio; G is it rounded up to a power of two on the tensor-core path
     int nc;                 // ring chunks of the tensor-core kernel (1 unless the window has more than 256 rows)
@@ -50,6 +51,8 @@ Layout make_layout(const Shape &s)
     L.ticket = take(U * 4);
     L.evicted = take(U * 4);
     L.state = take(sizeof(DevState) * (1 + (size_t)s.layers));     // whole-stack state, then one per layer
+    L.rows = take((1 + (size_t)s.layers) * 2 * s.B * 4);           // per state: the batch rows' fills, by step parity
+    L.row_shift = take((size_t)s.B * 4);
     L.stage_q = take(U * (size_t)s.Gq * D * s.es);
     L.stage_k = take(U * D * s.es);
     L.stage_v = take(U * D * s.es);
@@ -85,6 +88,8 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
 {
     s->layers = p->layers - p->full_layers;
     s->upl = p->batch * p->n_kv_heads;
+    s->B = p->batch;
+    s->Hkv = p->n_kv_heads;
     s->U = s->layers * s->upl;
     s->G = s->Gq = p->n_q_heads / p->n_kv_heads;
     s->D = p->head_dim;
@@ -141,6 +146,9 @@ struct mkv_ctx {
     int device;       // the CUDA device the context was created on
     bool owns_workspace;
     bool prefilled;
+    bool ragged;      // the batch rows' prompts had different lengths: per-row fills and position offsets are in use
+    int *row_n;       // [B] host mirror of the rows' fills (ragged only)
+    int *row_shift;   // [B] positions a row is behind the longest one
     long long t;      // host mirror of the device step state
     int n;
     int steps;
@@ -153,6 +161,8 @@ struct mkv_ctx {
 };
 
 namespace {
+
+const char *off(const void *p, size_t bytes) { return (const char *)p + bytes; }
 
 mkv_status fail(mkv_ctx *ctx, mkv_status st, const char *fmt, const char *detail = "")
 {
@@ -178,6 +188,9 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.T = c->s.T;
     a.norm_current = c->p.norm_mode == MKV_NORM_CURRENT ? 1 : 0;
     a.scale2 = (float)(1.4426950408889634 / sqrt((double)c->s.D));
+    a.row_n = c->ragged ? (int *)(b + c->L.rows) : nullptr;
+    a.row_shift = c->ragged ? (const int *)(b + c->L.row_shift) : nullptr;
+    a.B = c->s.B; a.Hkv = c->s.Hkv;
     return a;
 }
 
@@ -193,11 +206,12 @@ bool clear_arena(mkv_ctx *c, cudaStream_t stream)
 
 // Arguments of a launch that covers one layer of the context's own: every arena pointer is moved to the layer's
 // first unit, the inputs and `out` are that layer's tensors, and the layer's own step state is used.
-DecodeArgs make_args_layer(const mkv_ctx *c, int layer, const void *q, const void *k, const void *v, void *out)
+// `row` >= 0 narrows the launch further, to that batch row's units of the layer (prompt phase of a ragged batch).
+DecodeArgs make_args_layer(const mkv_ctx *c, int layer, const void *q, const void *k, const void *v, void *out, int row = -1)
 {
     DecodeArgs a = make_args(c, q, k, v, out);
     const Shape &s = c->s;
-    const size_t u0 = (size_t)layer * s.upl;
+    const size_t u0 = (size_t)layer * s.upl + (row >= 0 ? (size_t)row * s.Hkv : 0);
     a.K = (char *)a.K + u0 * s.cap * s.D * s.es; a.V = (char *)a.V + u0 * s.cap * s.D * s.es;
     a.pos += u0 * s.cap;
     a.ring_q = (char *)a.ring_q + u0 * s.R * s.G * s.D * s.es; a.ring_c += u0 * s.R * s.G;
@@ -206,8 +220,9 @@ DecodeArgs make_args_layer(const mkv_ctx *c, int layer, const void *q, const voi
     a.part_ml += u0 * s.splits * s.G * 2; a.part_o += u0 * s.splits * s.G * s.D;
     a.ticket += u0; a.evicted_pos += u0;
     a.st = a.st + 1 + layer;
+    if (a.row_n) a.row_n += (size_t)(1 + layer) * 2 * s.B;
     a.u0 = (int)u0;
-    a.U = s.upl;
+    a.U = row >= 0 ? s.Hkv : s.upl;
     return a;
 }
 
@@ -217,8 +232,11 @@ mkv_status level_states(mkv_ctx *ctx, int want, cudaStream_t stream)
 {
     if (ctx->state_ahead == 0 || ctx->state_ahead == want) return MKV_OK;
     DevState *st = (DevState *)(ctx->base + ctx->L.state);
-    const cudaError_t e = ctx->state_ahead == 1 ? launch_copy_state(st + 1, ctx->s.layers, st, stream)
-                                                : launch_copy_state(st, 1, st + 1, stream);
+    int *rows = ctx->ragged ? (int *)(ctx->base + ctx->L.rows) : nullptr;
+    const int ri = 2 * ctx->s.B;
+    const cudaError_t e = ctx->state_ahead == 1
+        ? launch_copy_state(st + 1, ctx->s.layers, st, stream, rows ? rows + ri : nullptr, rows, ri)
+        : launch_copy_state(st, 1, st + 1, stream, rows, rows ? rows + ri : nullptr, ri);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "state copy launch failed: %s", cudaGetErrorString(e));
     ctx->launches += 1;
     ctx->state_ahead = 0;
@@ -250,10 +268,20 @@ mkv_status launch_step(mkv_ctx *ctx, int layer, const void *q, const void *k, co
     } else {
         ctx->state_ahead = 1;
     }
+    if (ctx->ragged) {       // every row by its own fill; the uniform fill is the largest
+        int nmax = 0;
+        for (int b = 0; b < ctx->s.B; ++b) {
+            if (!step_scores(ctx->t - ctx->row_shift[b], ctx->row_n[b], ctx->steps, ctx->s.R, ctx->s.C, ctx->s.T)) ctx->row_n[b] += 1;
+            nmax = std::max(nmax, ctx->row_n[b]);
+        }
+        ctx->n = nmax;
+    } else if (!ev) {
+        ctx->n += 1;
+    } else if (ctx->s.T > 1) {
+        ctx->n = ctx->s.C + ctx->s.R;
+    }
     ctx->t += 1;
     ctx->steps += 1;
-    if (!ev) ctx->n += 1;
-    else if (ctx->s.T > 1) ctx->n = ctx->s.C + ctx->s.R;
     return MKV_OK;
 }
 
@@ -270,13 +298,17 @@ mkv_status core_create(mkv_ctx **out, const mkv_params *p, void *workspace, size
     if (!c) return MKV_OOM;
     memset(c, 0, sizeof(*c));
     c->p = *p; c->s = s; c->L = L; c->kind = kind;
-    if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); delete c; return MKV_CUDA; }
+    c->row_n = new (std::nothrow) int[2 * (size_t)s.B];
+    if (!c->row_n) { delete c; return MKV_OOM; }
+    c->row_shift = c->row_n + s.B;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { cudaGetLastError(); delete[] c->row_n; delete c; return MKV_CUDA; }
     if (workspace) {
         c->base = (char *)workspace;
     } else {
         void *mem = nullptr;
         if (cudaMalloc(&mem, L.total) != cudaSuccess) {
             cudaGetLastError();
+            delete[] c->row_n;
             delete c;
             return MKV_OOM;
         }
@@ -292,6 +324,7 @@ mkv_status core_create(mkv_ctx **out, const mkv_params *p, void *workspace, size
             cudaGetLastError();
             if (c->plan) tc_plan_destroy(c->plan);
             if (c->owns_workspace) cudaFree(c->base);
+            delete[] c->row_n;
             delete c;
             return e == cudaErrorMemoryAllocation ? MKV_OOM : MKV_CUDA;
         }
@@ -307,6 +340,7 @@ void core_destroy(mkv_ctx *ctx)
     if (ctx->plan_layer) tc_plan_destroy(ctx->plan_layer);
     if (ctx->prefill_scratch.ptr) cudaFree(ctx->prefill_scratch.ptr);
     if (ctx->owns_workspace && ctx->base) cudaFree(ctx->base);
+    delete[] ctx->row_n;
     delete ctx;
 }
 
@@ -330,6 +364,7 @@ mkv_status core_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *
         if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device)
             return fail(ctx, MKV_INVALID_ARG, "%s: the current CUDA device is not the one the context was created on", where);
     }
+    ctx->ragged = false;
     const DecodeArgs a = make_args(ctx, nullptr, nullptr, nullptr, nullptr);
     if (!clear_arena(ctx, stream)) return fail(ctx, MKV_CUDA, "%s: clearing the arena failed", where);
     const bool f32 = ctx->p.dtype == MKV_DTYPE_F32;
@@ -342,6 +377,61 @@ mkv_status core_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase: %s", cudaGetErrorString(e));
     ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
     ctx->t = prompt_len;
+    ctx->steps = 0;
+    ctx->next_layer = 0;
+    ctx->state_ahead = 0;
+    ctx->prefilled = true;
+    return MKV_OK;
+}
+
+// Prompt phase of a batch whose rows have prompts of different lengths (tensors padded to `padded_len` tokens): every
+// row goes through the prompt phase by itself, layer by layer, then the common step state is set.
+mkv_status core_prefill_ragged(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, const int32_t *prompt_len,
+                               int padded_len, cudaStream_t stream)
+{
+    const Shape &s = ctx->s;
+    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill_ragged: context already holds a sequence%s");
+    if (s.T > 1) return fail(ctx, MKV_UNSUPPORTED, "mkv_prefill_ragged: not available with coarse-grained eviction%s");
+    if (s.nc > 1) return fail(ctx, MKV_UNSUPPORTED, "mkv_prefill_ragged: not available with a window of more than 256 ring rows on the tensor-core kernel; create the context with the CUDA-core kernel%s");
+    int longest = 0;
+    for (int b = 0; b < s.B; ++b) longest = std::max(longest, (int)prompt_len[b]);
+    ctx->ragged = true;          // make_args hands the row arrays to the kernels from here on
+    if (!clear_arena(ctx, stream)) return fail(ctx, MKV_CUDA, "mkv_prefill_ragged: clearing the arena failed%s");
+    const bool f32 = ctx->p.dtype == MKV_DTYPE_F32;
+    const int qw_stride = padded_len < s.R ? padded_len : s.R;
+    int nmax = 0;
+    for (int b = 0; b < s.B; ++b) {
+        const int P = prompt_len[b], Rw = P < s.R ? P : s.R;
+        ctx->row_n[b] = (P - Rw > s.C) ? s.C + Rw : P;
+        ctx->row_shift[b] = longest - P;
+        nmax = std::max(nmax, ctx->row_n[b]);
+    }
+    for (int layer = 0; layer < s.layers; ++layer) {
+        for (int b = 0; b < s.B; ++b) {
+            const DecodeArgs a = make_args_layer(ctx, layer, nullptr, nullptr, nullptr, nullptr, b);
+            const size_t unit = ((size_t)layer * s.B + b) * s.Hkv;
+            const PrefillRow row = {padded_len, qw_stride, ctx->row_shift[b]};
+            const cudaError_t e = run_prefill(a, f32, s.D, off(k, unit * padded_len * s.D * s.es), off(v, unit * padded_len * s.D * s.es),
+                                              off(q_window, unit * s.Gq * qw_stride * s.D * s.es), prompt_len[b], stream,
+                                              &ctx->launches, &ctx->prefill_scratch, 0, &row);
+            if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(ctx, MKV_OOM, "mkv_prefill_ragged: no memory for scratch%s"); }
+            if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase: %s", cudaGetErrorString(e));
+        }
+    }
+    // the rows' fills for every state and both step parities, their offsets, then the common state
+    const int ns = 1 + s.layers;
+    int *rows_h = new (std::nothrow) int[(size_t)ns * 2 * s.B];
+    if (!rows_h) return fail(ctx, MKV_OOM, "mkv_prefill_ragged: out of host memory%s");
+    for (int i = 0; i < ns * 2; ++i) memcpy(rows_h + (size_t)i * s.B, ctx->row_n, sizeof(int) * s.B);
+    cudaError_t e = cudaMemcpyAsync(ctx->base + ctx->L.rows, rows_h, sizeof(int) * ns * 2 * s.B, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->base + ctx->L.row_shift, ctx->row_shift, sizeof(int) * s.B, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = launch_set_state((DevState *)(ctx->base + ctx->L.state), ns, (long long)longest, nmax, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    delete[] rows_h;
+    if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase: %s", cudaGetErrorString(e));
+    ctx->launches += 1;
+    ctx->n = nmax;
+    ctx->t = longest;
     ctx->steps = 0;
     ctx->next_layer = 0;
     ctx->state_ahead = 0;
@@ -372,8 +462,27 @@ mkv_status core_sync(mkv_ctx *ctx, cudaStream_t stream)
     }
     // the device-resident state is authoritative (steps replayed from a CUDA graph advance
     // it without passing through this library); the host mirror follows it at a step boundary
-    if (ctx->prefilled && ctx->next_layer == 0) { ctx->t = cur.t; ctx->n = cur.n; ctx->steps = cur.steps; }
+    if (ctx->prefilled && ctx->next_layer == 0) {
+        ctx->t = cur.t; ctx->n = cur.n; ctx->steps = cur.steps;
+        if (ctx->ragged) {       // the rows' fills of that state, in the buffer of the current step parity
+            const size_t at = ((size_t)(ctx->state_ahead == 2 ? 1 : 0) * 2 + (cur.steps & 1)) * ctx->s.B;
+            e = cudaMemcpy(ctx->row_n, (const int *)(ctx->base + ctx->L.rows) + at, sizeof(int) * ctx->s.B, cudaMemcpyDeviceToHost);
+            if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "mkv_sync: %s", cudaGetErrorString(e));
+        }
+    }
     return MKV_OK;
+}
+
+// fill and next position of batch row `row` as layer `layer` of this context sees them now
+void core_row_state(const mkv_ctx *ctx, int layer, int row, int32_t *count, int64_t *next_pos)
+{
+    const Shape &s = ctx->s;
+    const bool ahead = layer < ctx->next_layer;     // the layer has taken the step that is under way
+    const int sh = ctx->ragged ? ctx->row_shift[row] : 0;
+    const int n = ctx->ragged ? ctx->row_n[row] : ctx->n;
+    const bool ev = step_scores(ctx->t - sh, n, ctx->steps, s.R, s.C, s.T);
+    if (count) *count = !ahead ? n : (!ev ? n + 1 : (s.T > 1 ? s.C + s.R : n));
+    if (next_pos) *next_pos = ctx->t - sh + (ahead ? 1 : 0);
 }
 
 void core_view(mkv_ctx *ctx, int layer, mkv_view *view)
@@ -392,6 +501,11 @@ void core_view(mkv_ctx *ctx, int layer, mkv_view *view)
     const bool ahead = layer < ctx->next_layer;
     const bool ev = step_scores(ctx->t, ctx->n, ctx->steps, s.R, s.C, s.T);
     view->count = !ahead ? ctx->n : (!ev ? ctx->n + 1 : (s.T > 1 ? s.C + s.R : ctx->n));
+    if (ctx->ragged) {      // the largest fill among the rows; mkv_row_state gives each row's own
+        int32_t cnt[1];
+        view->count = 0;
+        for (int r = 0; r < s.B; ++r) { core_row_state(ctx, layer, r, cnt, nullptr); view->count = std::max(view->count, cnt[0]); }
+    }
     view->capacity = s.cap;
     view->group_stride = s.G;
     view->next_pos = ctx->t + (ahead ? 1 : 0);
@@ -400,7 +514,6 @@ void core_view(mkv_ctx *ctx, int layer, mkv_view *view)
 // byte offsets of the first own layer inside whole-model tensors
 size_t q_bytes_per_layer(const mkv_ctx *c) { return (size_t)c->p.batch * c->p.n_q_heads * c->s.D * c->s.es; }
 size_t kv_bytes_per_layer(const mkv_ctx *c) { return (size_t)c->p.batch * c->p.n_kv_heads * c->s.D * c->s.es; }
-const char *off(const void *p, size_t bytes) { return (const char *)p + bytes; }
 
 }  // namespace
 
@@ -518,6 +631,7 @@ mkv_status mkv_reset(mkv_ctx *ctx)
     for (mkv_ctx *c : {ctx, ctx->full}) {
         if (!c) continue;
         c->prefilled = false;
+        c->ragged = false;
         c->t = 0; c->n = 0; c->steps = 0; c->next_layer = 0; c->state_ahead = 0; c->cursor = 0;
     }
     return MKV_OK;
@@ -531,6 +645,39 @@ mkv_status mkv_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *q
 mkv_status mkv_prefill_static(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, int prompt_len, void *stream)
 {
     return prefill_any(ctx, k, v, q_window, prompt_len, stream, true, "mkv_prefill_static");
+}
+
+mkv_status mkv_prefill_ragged(mkv_ctx *ctx, const void *k, const void *v, const void *q_window, const int32_t *prompt_len,
+                              int padded_len, void *stream)
+{
+    if (!ctx) return MKV_INVALID_ARG;
+    if (!k || !v || !q_window || !prompt_len) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_ragged: NULL argument%s");
+    if (padded_len < 1 || padded_len > (1 << 24)) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_ragged: padded_len out of range%s");
+    for (int b = 0; b < ctx->p.batch; ++b)
+        if (prompt_len[b] < 1 || prompt_len[b] > padded_len)
+            return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_ragged: every prompt_len must lie in [1, padded_len]%s");
+    if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill_ragged: context already holds a sequence%s");
+    const int qw = padded_len < ctx->s.R ? padded_len : ctx->s.R;
+    size_t off_kv = 0, off_q = 0;
+    if (ctx->full) {
+        for (int b = 0; b < ctx->p.batch; ++b)
+            if (prompt_len[b] > ctx->p.max_tokens) return fail(ctx, MKV_INVALID_ARG, "mkv_prefill_ragged: a prompt is longer than max_tokens%s");
+        const mkv_status st = core_prefill_ragged(ctx->full, k, v, q_window, prompt_len, padded_len, (cudaStream_t)stream);
+        if (st != MKV_OK) { snprintf(ctx->err, sizeof(ctx->err), "%s", ctx->full->err); return st; }
+        off_kv = kv_bytes_per_layer(ctx) * padded_len * ctx->p.full_layers;
+        off_q = q_bytes_per_layer(ctx) * qw * ctx->p.full_layers;
+    }
+    return core_prefill_ragged(ctx, off(k, off_kv), off(v, off_kv), off(q_window, off_q), prompt_len, padded_len, (cudaStream_t)stream);
+}
+
+mkv_status mkv_row_state(mkv_ctx *ctx, int layer, int32_t *count, int64_t *next_pos)
+{
+    if (!ctx || (!count && !next_pos)) return MKV_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->p.layers) return fail(ctx, MKV_INVALID_ARG, "mkv_row_state: layer out of range%s");
+    const mkv_ctx *c = layer < ctx->p.full_layers ? ctx->full : ctx;
+    const int l = layer < ctx->p.full_layers ? layer : layer - ctx->p.full_layers;
+    for (int b = 0; b < ctx->p.batch; ++b) core_row_state(c, l, b, count ? count + b : nullptr, next_pos ? next_pos + b : nullptr);
+    return MKV_OK;
 }
 
 mkv_status mkv_decode_step(mkv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *out, void *stream)

@@ -54,6 +54,20 @@ struct DecodeArgs {
     float scale2;              // log2(e) / sqrt(D)
     float *Fc;                 // [U][nc][cap]  tensor-core kernel with a window of nc > 1 ring chunks: the fused score of
     int nc;                    // each chunk's rows, combined by the unit's epilogue; unused (nullptr, 1) otherwise
+    // Batch rows with prompts of different lengths (nullptr / unused otherwise).  The step state then counts time
+    // from the longest prompt: st->t is that row's position and st->n the largest fill; row b is row_shift[b]
+    // positions behind (its token has position st->t - row_shift[b]) and holds row_n[(st->steps & 1) * B + b]
+    // tokens.  The fills are double-buffered by step parity because the CTA that advances the state does so while
+    // other CTAs of the launch still read the current fills.  Ring slots are assigned by st->t in every row.
+    int *row_n;                // [2][B]
+    const int *row_shift;      // [B]
+    int B, Hkv;                // unit u (of this launch) belongs to batch row (u / Hkv) % B
+};
+
+// Fill, position offset and policy decision of one unit on this step.
+struct UnitStep {
+    int n, shift;
+    bool evict;
 };
 
 __device__ __forceinline__ float ldf(const float *p) { return *p; }
@@ -117,6 +131,42 @@ __host__ __device__ inline bool step_scores(long long t, int n, int steps, int R
 
 constexpr int kFinalizeSmemFloats = 4 * kMaxGroup + 3 * 32 + 128;
 
+// `evict` is the decision for the uniform state (t, n); rows of different lengths take their own.
+__device__ __forceinline__ UnitStep unit_step(const DecodeArgs &a, int u, long long t, int n, int steps, bool evict)
+{
+    UnitStep s;
+    s.n = n; s.shift = 0; s.evict = evict;
+    if (a.row_n != nullptr) {
+        const int b = (u / a.Hkv) % a.B;
+        s.n = a.row_n[(steps & 1) * a.B + b];
+        s.shift = a.row_shift[b];
+        s.evict = step_scores(t - s.shift, s.n, steps, a.R, a.C, a.T);
+    }
+    return s;
+}
+
+// The step state after this launch (called by one thread, once per launch, after every CTA has read the state).
+__device__ __forceinline__ void advance_state(const DecodeArgs &a, long long t, int n, int steps, bool evict)
+{
+    int n_next = (evict && a.T == 1) ? n : n + 1;
+    if (a.row_n != nullptr) {      // every row appends or evicts by its own fill; the uniform fill is the largest
+        n_next = 0;
+        const int *cur = a.row_n + (steps & 1) * a.B;
+        int *nxt = a.row_n + ((steps + 1) & 1) * a.B;
+        for (int b = 0; b < a.B; ++b) {
+            const int nb = cur[b];
+            const int v = step_scores(t - a.row_shift[b], nb, steps, a.R, a.C, a.T) ? nb : nb + 1;
+            nxt[b] = v;
+            n_next = v > n_next ? v : n_next;
+        }
+    }
+    a.st->t = t + 1;
+    a.st->n = n_next;
+    a.st->compact = (evict && a.T > 1) ? 1 : 0;
+    a.st->steps = steps + 1;
+    a.st->done = 0;
+}
+
 
 // barrier over the `nthr` threads that run an epilogue together (id 0 with the whole CTA is
 // __syncthreads; warp-specialised kernels give each compute group its own id)
@@ -179,7 +229,7 @@ __device__ void renormalise_after_eviction(const DecodeArgs &a, int u, int e_slo
 // round trips.
 template <typename T, int D, int GT>
 __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, int active, bool evict, float *sm,
-                              int tid, int nthr, int bar_id)
+                              int tid, int nthr, int bar_id, int shift = 0)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const int G = GT > 0 ? GT : a.G;
@@ -256,7 +306,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     int e_slot = n, e_pos = -1;
     if (evict) {
         const float *sn = a.s_new + (size_t)u * G * a.cap;
-        const long long thr = t - a.R;
+        const long long thr = t - shift - a.R;        // positions are the row's own; ring slots follow t
         unsigned long long best = ~0ull;
         int bslot = -1;
         // four slots per thread and round, all their loads in flight together
@@ -344,7 +394,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     for (int i = tid; i < G * D; i += nthr) stf(rq + i, i < Gq * D ? ldf(q + i) : 0.f);
     if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
     if (tid == 0) {
-        pos[e_slot] = (int)t;
+        pos[e_slot] = (int)(t - shift);
         a.evicted_pos[u] = e_pos;
         a.ticket[u] = 0;
     }
@@ -360,11 +410,7 @@ __device__ __forceinline__ void finish_cta(const DecodeArgs &a, long long t, int
         __threadfence();
         const unsigned int total = gridDim.x * gridDim.y * gridDim.z;
         if (atomicAdd(&a.st->done, 1u) == total - 1) {
-            a.st->t = t + 1;
-            a.st->n = (evict && a.T == 1) ? n : n + 1;
-            a.st->compact = (evict && a.T > 1) ? 1 : 0;
-            a.st->steps += 1;
-            a.st->done = 0;
+            advance_state(a, t, n, a.st->steps, evict);
             __threadfence();
         }
     }

@@ -39,8 +39,17 @@ struct PrefillScratch {
     void *ptr;
     size_t bytes;
 };
+// One batch row of a batch whose prompts have different lengths: `a` covers the row's units of one layer, k / v /
+// q_window point at the row's first unit inside tensors padded to the longest prompt (kv_stride tokens per unit,
+// qw_stride window entries per head), and the row is `shift` positions behind the longest on the context's common
+// time axis, which assigns the ring slots.  Such a call leaves the step state alone and does not synchronise.
+struct PrefillRow {
+    int kv_stride, qw_stride, shift;
+};
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
-                        int P, cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states);
+                        int P, cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states,
+                        const PrefillRow *row = nullptr);
+cudaError_t launch_set_state(DevState *st, int n_states, long long t, int n, cudaStream_t stream);
 
 // Tensor-core scoring of the prompt phase (mkv_prefill_tc.cu): two passes over the prompt keys, window-row
 // normalisers into ring_c and fused scores of the older tokens into Fp [nb][P].
@@ -59,6 +68,7 @@ cudaError_t run_prefill_static(const DecodeArgs &a, bool f32, int D, const void 
 
 // Copies one step state over n_dst others (the whole-stack state and the per-layer states are brought level when
 // a context switches between whole-stack and per-layer calls).
-cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream);
+cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream, int *rows_dst = nullptr,
+                              const int *rows_src = nullptr, int row_ints = 0);
 
 }  // namespace mkv

@@ -53,15 +53,17 @@ __global__ void set_state_kernel(DevState *st, int n_states, long long t, int n)
 template <typename T, int D>
 __global__ void __launch_bounds__(kPT) prefill_logits_kernel(const T *__restrict__ k, const T *__restrict__ qwin,
                                                              float *__restrict__ S, int ub0, int P, int Rw, int G,
-                                                             float scale2)
+                                                             float scale2, int Ps, int Rws)
 {
+    // Ps, Rws: tokens per unit in k and entries per head in qwin as laid out by the caller (P and Rw unless the
+    // batch rows' prompts have different lengths and the tensors are padded to the longest)
     extern __shared__ __align__(16) float psm[];
     float *Ks = psm, *Qs = psm + kPK * (D + 4), *Ssm = Qs + kPR * (D + 4);
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     const int u = ub0 + blockIdx.y, kt = blockIdx.x * kPK;
     const int rows = Rw * G;
     constexpr int KS = D + 4, C4 = D / 4;
-    const T *Ku = k + (size_t)u * P * D;
+    const T *Ku = k + (size_t)u * Ps * D;
     for (int idx = tid; idx < kPK * C4; idx += kPT) {
         const int key = idx / C4, c4 = idx % C4;
         float v[4] = {0.f, 0.f, 0.f, 0.f};
@@ -75,7 +77,7 @@ __global__ void __launch_bounds__(kPT) prefill_logits_kernel(const T *__restrict
             const int rl = idx / C4, c4 = idx % C4;
             const int row = r0 + rl, i = row / G, g = row % G;
             float v[4];
-            ld4(qwin + (((size_t)u * G + g) * Rw + i) * D + c4 * 4, v);
+            ld4(qwin + (((size_t)u * G + g) * Rws + i) * D + c4 * 4, v);
             *reinterpret_cast<float4 *>(Qs + rl * KS + c4 * 4) = make_float4(v[0], v[1], v[2], v[3]);
         }
         __syncthreads();
@@ -115,7 +117,7 @@ __global__ void __launch_bounds__(kPT) prefill_logits_kernel(const T *__restrict
 
 // c = max + log2(sum exp2(s - max)) of one window row; stored in the ring row p % R.
 __global__ void __launch_bounds__(kPT) prefill_rowstats_kernel(const float *__restrict__ S, float *__restrict__ ring_c,
-                                                               int ub0, int P, int Rw, int G, int Gs, int R)
+                                                               int ub0, int P, int Rw, int G, int Gs, int R, int shift)
 {
     __shared__ float red[kPT / 32];
     __shared__ float bc;
@@ -140,7 +142,7 @@ __global__ void __launch_bounds__(kPT) prefill_rowstats_kernel(const float *__re
         float x = 0.f;
         for (int w = 0; w < kPT / 32; ++w) x += red[w];
         const int i = row / G, g = row % G;
-        const int rslot = (P - Rw + i) % R;
+        const int rslot = (P - Rw + i + shift) % R;     // ring slots are assigned on the context's common time axis
         ring_c[((size_t)u * R + rslot) * Gs + g] = m + log2f(x);     // Gs: heads per ring slot (G padded)
     }
 }
@@ -148,12 +150,12 @@ __global__ void __launch_bounds__(kPT) prefill_rowstats_kernel(const float *__re
 // Eq. 4-6 with Algorithm 1's group sum: F[j] for every older prompt token j < P - Rw.
 __global__ void __launch_bounds__(kPT) prefill_fuse_kernel(const float *__restrict__ S, const float *__restrict__ ring_c,
                                                            float *__restrict__ Fp, int ub0, int P, int Rw, int G, int Gs,
-                                                           int R, int fusion)
+                                                           int R, int fusion, int shift)
 {
     extern __shared__ float cs[];   // [Rw * G]
     const int u = ub0 + blockIdx.y, rows = Rw * G;
     for (int row = threadIdx.x; row < rows; row += kPT) {
-        const int rslot = (P - Rw + row / G) % R;
+        const int rslot = (P - Rw + row / G + shift) % R;
         cs[row] = ring_c[((size_t)u * R + rslot) * Gs + row % G];
     }
     __syncthreads();
@@ -233,7 +235,7 @@ __global__ void prefill_identity_pos_kernel(int *pos, int U, int n, int cap)
 
 // K/V rows of the kept prompt positions into the arena, 16 bytes per thread.
 template <typename T, int D>
-__global__ void prefill_gather_kernel(const T *__restrict__ k, const T *__restrict__ v, DecodeArgs a, int P, int n)
+__global__ void prefill_gather_kernel(const T *__restrict__ k, const T *__restrict__ v, DecodeArgs a, int Ps, int n)
 {
     constexpr int CH = D * sizeof(T) / 16;
     const int u = blockIdx.x;
@@ -241,22 +243,22 @@ __global__ void prefill_gather_kernel(const T *__restrict__ k, const T *__restri
     if (idx >= n * CH) return;
     const int slot = idx / CH, c = idx % CH;
     const int p = a.pos[(size_t)u * a.cap + slot];
-    const uint4 *ks = reinterpret_cast<const uint4 *>(k + ((size_t)u * P + p) * D) + c;
-    const uint4 *vs = reinterpret_cast<const uint4 *>(v + ((size_t)u * P + p) * D) + c;
+    const uint4 *ks = reinterpret_cast<const uint4 *>(k + ((size_t)u * Ps + p) * D) + c;
+    const uint4 *vs = reinterpret_cast<const uint4 *>(v + ((size_t)u * Ps + p) * D) + c;
     reinterpret_cast<uint4 *>(static_cast<T *>(a.K) + ((size_t)u * a.cap + slot) * D)[c] = *ks;
     reinterpret_cast<uint4 *>(static_cast<T *>(a.V) + ((size_t)u * a.cap + slot) * D)[c] = *vs;
 }
 
 // window queries into their ring rows (row p % R)
 template <typename T, int D>
-__global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, int P, int Rw)
+__global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, int P, int Rw, int Rws, int shift)
 {
     const int u = blockIdx.x, G = a.G, Gq = a.Gq;       // heads Gq .. G-1 of a ring slot are padding (zero query)
     T *rq = static_cast<T *>(a.ring_q) + (size_t)u * a.R * G * D;
     for (int idx = threadIdx.x; idx < Rw * G * D; idx += blockDim.x) {
         const int dd = idx % D, g = (idx / D) % G, i = idx / (D * G);
-        const int rslot = (P - Rw + i) % a.R;
-        if (g < Gq) rq[((size_t)rslot * G + g) * D + dd] = qwin[(((size_t)u * Gq + g) * Rw + i) * D + dd];
+        const int rslot = (P - Rw + i + shift) % a.R;
+        if (g < Gq) rq[((size_t)rslot * G + g) * D + dd] = qwin[(((size_t)u * Gq + g) * Rws + i) * D + dd];
         else stf(rq + ((size_t)rslot * G + g) * D + dd, 0.f);
     }
 }
@@ -268,14 +270,14 @@ __global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, in
 // tokens that were kept and that the row may see, c = log2 sum exp2(s), from the arena as it stands (kept K rows,
 // their positions, the ring's queries).  One CTA per (window row, unit).
 template <typename T, int D>
-__global__ void __launch_bounds__(kPT) prefill_renorm_kernel(DecodeArgs a, int P, int Rw, int n)
+__global__ void __launch_bounds__(kPT) prefill_renorm_kernel(DecodeArgs a, int P, int Rw, int n, int shift)
 {
     __shared__ float qs[D];
     __shared__ float red[kPT / 32];
     __shared__ float bc;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int u = blockIdx.y, G = a.G, row = blockIdx.x, i = row / G, g = row % G;
-    const int rpos = P - Rw + i, rslot = rpos % a.R;
+    const int rpos = P - Rw + i, rslot = (rpos + shift) % a.R;
     float *c_out = a.ring_c + ((size_t)u * a.R + rslot) * G + g;
     if (*c_out == INFINITY) return;                                   // padding head
     const T *q = static_cast<const T *>(a.ring_q) + (((size_t)u * a.R + rslot) * G + g) * D;
@@ -323,8 +325,11 @@ __global__ void __launch_bounds__(kPT) prefill_renorm_kernel(DecodeArgs a, int P
 
 template <typename T, int D>
 cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *qwin, int P, cudaStream_t stream,
-                          unsigned long long *launches, float *S, size_t scratch_floats, int n_states)
+                          unsigned long long *launches, float *S, size_t scratch_floats, int n_states, const PrefillRow *row)
 {
+    // `row`: the units of `a` are one batch row of a ragged batch - the tensors are padded to the longest prompt, the
+    // ring slots follow the common time axis, the caller sets the step state and synchronises after the last row
+    const int Ps = row ? row->kv_stride : P, shift = row ? row->shift : 0;
     const int U = a.U, G = a.G, R = a.R, C = a.C;
     // the CUDA-core scoring kernels work on the model's Gq heads per window position (rows of S); the ring keeps G
     // heads per slot, the padding heads with normaliser +inf from init_arena_kernel
@@ -335,7 +340,8 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     // bf16 / head_dim 128 shapes score on the tensor cores (two passes over the keys, no rows x P table); the
     // others materialise the window-row logits S [rows][P] per unit and reduce them with CUDA-core kernels
     // (the arena's group must be the padded one: a context that runs the CUDA-core decode kernel keeps G as it is)
-    const bool tc = prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P) && tc_padded_group(a.Gq) == G;
+    const bool tc = !row && prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P) && tc_padded_group(a.Gq) == G;
+    const int Rws = row ? row->qw_stride : Rw;
     const int tc_splits = tc ? prefill_tc_splits(U, P) : 0;
     const size_t per_unit = tc ? prefill_tc_floats_per_unit(P, Rw, G, tc_splits) : (size_t)rows * P + P;   // floats
     if (per_unit + 1 > scratch_floats) return cudaErrorInvalidConfiguration;
@@ -363,14 +369,14 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
             if (e != cudaSuccess) return e;
         } else {
             prefill_logits_kernel<T, D><<<dim3((P + kPK - 1) / kPK, nb), kPT, logits_smem, stream>>>(k, qwin, S, ub0, P, Rw,
-                                                                                                 a.Gq, a.scale2);
-            prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, a.Gq, G, R);
+                                                                                                 a.Gq, a.scale2, Ps, Rws);
+            prefill_rowstats_kernel<<<dim3(rows, nb), kPT, 0, stream>>>(S, a.ring_c, ub0, P, Rw, a.Gq, G, R, shift);
             *launches += 2;
         }
         if (select) {
             if (!tc) {
                 prefill_fuse_kernel<<<dim3((P - Rw + kPT - 1) / kPT, nb), kPT, rows * sizeof(float), stream>>>(
-                    S, a.ring_c, Fp, ub0, P, Rw, a.Gq, G, R, a.fusion);
+                    S, a.ring_c, Fp, ub0, P, Rw, a.Gq, G, R, a.fusion, shift);
                 ++*launches;
             }
             prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
@@ -382,14 +388,16 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
         ++*launches;
     }
     constexpr int CH = D * sizeof(T) / 16;
-    prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, P, n);
-    prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw);
+    prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, Ps, n);
+    prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw, Rws, shift);
     if (a.norm_current && select) {
-        prefill_renorm_kernel<T, D><<<dim3(Rw * G, U), kPT, 0, stream>>>(a, P, Rw, n);
+        prefill_renorm_kernel<T, D><<<dim3(Rw * G, U), kPT, 0, stream>>>(a, P, Rw, n, shift);
         ++*launches;
     }
+    *launches += 2;
+    if (row) return cudaGetLastError();
     set_state_kernel<<<1, 32, 0, stream>>>(a.st, n_states, (long long)P, n);
-    *launches += 3;
+    *launches += 1;
     e = cudaGetLastError();
     const cudaError_t e2 = cudaStreamSynchronize(stream);
     if (e != cudaSuccess || e2 != cudaSuccess) return e != cudaSuccess ? e : e2;
@@ -403,17 +411,18 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
 }
 
 cudaError_t dispatch_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
-                             cudaStream_t stream, unsigned long long *launches, float *S, size_t scratch_floats, int n_states)
+                             cudaStream_t stream, unsigned long long *launches, float *S, size_t scratch_floats, int n_states,
+                             const PrefillRow *row = nullptr)
 {
     if (f32) {
         auto kk = static_cast<const float *>(k), vv = static_cast<const float *>(v), qq = static_cast<const float *>(q_window);
-        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states)
-                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states);
+        return D == 64 ? run_prefill_t<float, 64>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states, row)
+                       : run_prefill_t<float, 128>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states, row);
     }
     auto kk = static_cast<const __nv_bfloat16 *>(k), vv = static_cast<const __nv_bfloat16 *>(v),
          qq = static_cast<const __nv_bfloat16 *>(q_window);
-    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states)
-                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states);
+    return D == 64 ? run_prefill_t<__nv_bfloat16, 64>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states, row)
+                   : run_prefill_t<__nv_bfloat16, 128>(a, kk, vv, qq, P, stream, launches, S, scratch_floats, n_states, row);
 }
 
 // ---- scratch of mkv_prefill_static -------------------------------------------------------------------------
@@ -449,10 +458,11 @@ cudaError_t static_scratch_address(int device, float **out)
 }  // namespace
 
 cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window, int P,
-                        cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states)
+                        cudaStream_t stream, unsigned long long *launches, PrefillScratch *scratch, int n_states,
+                        const PrefillRow *row)
 {
     const int Rw = P < a.R ? P : a.R;
-    const bool tc = prefill_tc_supported(f32, D, a.Gq, a.R, k, P) && tc_padded_group(a.Gq) == a.G;
+    const bool tc = !row && prefill_tc_supported(f32, D, a.Gq, a.R, k, P) && tc_padded_group(a.Gq) == a.G;
     const size_t per_unit = (tc ? prefill_tc_floats_per_unit(P, Rw, a.G, prefill_tc_splits(a.U, P))
                                 : (size_t)Rw * a.G * P + P) * sizeof(float);
     size_t ub = ((size_t)1 << 30) / per_unit;
@@ -472,21 +482,32 @@ cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, con
         scratch->bytes = need;
     }
     return dispatch_prefill(a, f32, D, k, v, q_window, P, stream, launches, static_cast<float *>(scratch->ptr),
-                            scratch->bytes / sizeof(float), n_states);
+                            scratch->bytes / sizeof(float), n_states, row);
+}
+
+cudaError_t launch_set_state(DevState *st, int n_states, long long t, int n, cudaStream_t stream)
+{
+    set_state_kernel<<<1, 32, 0, stream>>>(st, n_states, t, n);
+    return cudaGetLastError();
 }
 
 namespace {
-__global__ void copy_state_kernel(DevState *dst, int n_dst, const DevState *src)
+// rows_dst / rows_src: the states' per-row fills ([2][B] ints per state, see DecodeArgs::row_n), or nullptr
+__global__ void copy_state_kernel(DevState *dst, int n_dst, const DevState *src, int *rows_dst, const int *rows_src,
+                                  int row_ints)
 {
     const DevState s = *src;
     __syncthreads();            // src may be one of the destinations
     for (int i = threadIdx.x; i < n_dst; i += blockDim.x) { dst[i] = s; dst[i].done = 0; }
+    if (rows_dst != nullptr && rows_dst != rows_src)
+        for (int i = threadIdx.x; i < n_dst * row_ints; i += blockDim.x) rows_dst[i] = rows_src[i % row_ints];
 }
 }  // namespace
 
-cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream)
+cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream, int *rows_dst,
+                              const int *rows_src, int row_ints)
 {
-    copy_state_kernel<<<1, 64, 0, stream>>>(dst, n_dst, src);
+    copy_state_kernel<<<1, 64, 0, stream>>>(dst, n_dst, src, rows_dst, rows_src, row_ints);
     return cudaGetLastError();
 }
 

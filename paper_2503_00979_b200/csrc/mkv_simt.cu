@@ -73,10 +73,15 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(const __grid_cons
     const int u = blockIdx.x / a.splits, sp = blockIdx.x % a.splits;
     const long long t = a.st->t;
     const int n = a.st->n;
-    const bool evict = step_scores(t, n, a.st->steps, R, a.C, a.T);
+    const int steps_done = a.st->steps;
+    const bool evict_all = step_scores(t, n, steps_done, R, a.C, a.T);
+    // the unit's own fill and policy decision (they differ from the uniform ones only between batch rows whose
+    // prompts had different lengths); the splits are laid out over the largest fill
+    const UnitStep us = unit_step(a, u, t, n, steps_done, evict_all);
+    const bool evict = us.evict;
     int active;
     const int per = split_len(n, a.splits, kTK, &active);
-    const int k0 = sp * per, k1 = min(n, k0 + per);
+    const int k0 = sp * per, k1 = min(us.n, k0 + per);
 
     const SimtSmem L = simt_smem_layout<T, D>(chunk_rs * G, G);
     T *Qs = reinterpret_cast<T *>(smem_raw + L.q_off);
@@ -269,10 +274,10 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(const __grid_cons
         __syncthreads();
         if (is_last) {
             __threadfence();
-            finalize_unit<T, D, 0>(a, u, t, n, active, evict, misc + 64, tid, kThreads, 0);
+            finalize_unit<T, D, 0>(a, u, t, us.n, active, evict, misc + 64, tid, kThreads, 0, us.shift);
         }
     }
-    finish_cta(a, t, n, evict);
+    finish_cta(a, t, n, evict_all);
 }
 
 template <typename T, int D>

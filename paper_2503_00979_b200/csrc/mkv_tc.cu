@@ -174,7 +174,7 @@ struct RingPos {
 // l_ml [G][2] sits in shared memory.
 template <int G, bool LOCAL>
 __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, int nseg, bool evict, float *sm, int tid,
-                              int bar_id, const float (&l_o)[G], const float *l_ml)
+                              int bar_id, const float (&l_o)[G], const float *l_ml, int shift)
 {
     constexpr int NT_ = kGroupThreads;
     const int lane = tid & 31, warp = tid >> 5;
@@ -271,7 +271,7 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
         if (tid == 0 && n < a.cap) F[n] = -1.f;
     } else {
         const float *sn = a.s_new + (size_t)u * G * a.cap;
-        const long long thr = t - a.R;
+        const long long thr = t - shift - a.R;        // positions are the row's own; ring slots follow t
         float cn[G];
 #pragma unroll
         for (int g = 0; g < G; ++g) cn[g] = cnew[g];
@@ -352,13 +352,15 @@ __device__ void finalize_fast(const DecodeArgs &a, int u, long long t, int n, in
     }
     if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
     if (tid == 0) {
-        pos[e_slot] = (int)t;
+        pos[e_slot] = (int)(t - shift);
         a.evicted_pos[u] = e_pos;
         a.ticket[u] = 0;
     }
 }
 
-template <int G, int FUSION, int NG, bool MC>
+// MC: the window is cut into ring chunks.  RAGGED: the batch rows have their own fills and position offsets
+// (DecodeArgs::row_n); compiled separately so that the uniform kernel carries none of it.
+template <int G, int FUSION, int NG, bool MC, bool RAGGED>
 __global__ void __launch_bounds__(tc_threads(NG), 1)
 decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
@@ -432,11 +434,15 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     if (tid == 0) {
         __threadfence();
         if (atomicAdd(&a.st->done, 1u) == gridDim.x - 1) {
-            a.st->t = t + 1;
-            a.st->n = (evict && a.T == 1) ? n : n + 1;
-            a.st->compact = (evict && a.T > 1) ? 1 : 0;
-            a.st->steps = steps_done + 1;
-            a.st->done = 0;
+            if constexpr (RAGGED) {
+                advance_state(a, t, n, steps_done, evict);
+            } else {
+                a.st->t = t + 1;
+                a.st->n = (evict && a.T == 1) ? n : n + 1;
+                a.st->compact = (evict && a.T > 1) ? 1 : 0;
+                a.st->steps = steps_done + 1;
+                a.st->done = 0;
+            }
         }
     }
 
@@ -615,6 +621,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             const int u = MC ? x.unit / NCe : x.unit;
             const int cc = MC ? (NCe == 1 ? c_main : x.unit - u * NCe) : 0;      // ring chunk of this item
             const bool main_item = MC ? cc == c_main : true;
+            const UnitStep us = RAGGED ? unit_step(a, u, t, n, steps_done, evict) : UnitStep{n, 0, evict};   // the unit's own fill and policy decision
             {
                 // frozen normalisers of the ring rows, negated; the new row and padding give weight 0
                 for (int c = lane; c < RGP; c += 32) {
@@ -654,7 +661,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                             tmem_ld32(taddr + (uint32_t)c, v);
                             score_chunk<G, FUSION>(v, negc + c, a.scale2, F);
                         }
-                        if (key < n) Fdst[key] = F;
+                        if (key < us.n) Fdst[key] = F;
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
@@ -671,7 +678,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 if (!ok) break;
                 tc_fence_after();
                 const int key = (x.tile0 + j) * kTile + gtid;
-                const bool valid = key < n;
+                const bool valid = key < us.n;
                 const uint32_t taddr = tmem_base + (uint32_t)(buf * RGP) + ((uint32_t)(wq * 32) << 16);
                 // Each TMEM load and its wait form one asm statement: the destination registers are
                 // written asynchronously, so nothing may touch them between the two.
@@ -684,7 +691,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 for (int g = 0; g < G; ++g) {
                     const float s2 = valid ? __uint_as_float(sv[g]) * a.scale2 : -INFINITY;
                     st_w[g * 32 + lane] = s2;
-                    if (valid && evict) s_new[(size_t)g * a.cap + key] = s2;
+                    if (valid && us.evict) s_new[(size_t)g * a.cap + key] = s2;
                     const float mn = fmaxf(mrun[g], warp_max(s2));
                     // factor that brings what was accumulated under the old reference to the new one
                     const float f = mn == mrun[g] ? 1.f : ex2f(mrun[g] - mn);
@@ -765,7 +772,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 // ---- fused scores of this warp's 32 keys over the ring rows (Eq. 4-6): only on steps that run the
                 // policy.  While the cache is still filling, and between two runs of a coarse-grained policy, nothing
                 // is evicted and the accumulator buffer goes back as soon as the new row's logits have been read.
-                if (evict) {
+                if (us.evict) {
                     float F = 0.f;
                     for (int c = 0; c < RGP; c += 32) {
                         uint32_t v[32];
@@ -835,6 +842,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
             {
                 const int u = MC ? x.unit / NCe : x.unit;
                 const bool main_item = MC ? (NCe == 1 || x.unit - u * NCe == c_main) : true;
+                const UnitStep us = RAGGED ? unit_step(a, u, t, n, steps_done, evict) : UnitStep{n, 0, evict};
                 if (group_any(kEpiBar, !mbar_wait(bar_udone, (uint32_t)(k & 1), abort_flag, kWaitUDone, WL))) { ok = false; break; }
                 // merge the compute warps' partials: common reference = max of theirs
                 if (etid < G && main_item) {
@@ -885,10 +893,10 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     }
                     group_sync(kEpiBar, kGroupThreads);
                     if (*flag) {
-                        if (evict) {
+                        if (us.evict) {
                             float *F = a.F + (size_t)u * a.cap;
                             const float *Fc = a.Fc + (size_t)u * geo.nc * a.cap;
-                            for (int key = etid; key < n; key += kGroupThreads) {
+                            for (int key = etid; key < us.n; key += kGroupThreads) {
                                 float f = __ldcg(Fc + key);
                                 for (int c = 1; c < NCe; ++c) f = fuse(FUSION, f, __ldcg(Fc + (size_t)c * a.cap + key));
                                 F[key] = f;
@@ -897,10 +905,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                         }
                         int idx;
                         const int ncta_main = w.ctas_of_unit(u * NCe + (NCe == 1 ? 0 : c_main), idx);
-                        finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, ncta_main, evict, fin_sm, etid, kGroupThreads, kEpiBar);
+                        finalize_unit<__nv_bfloat16, kD, G>(a, u, t, us.n, ncta_main, us.evict, fin_sm, etid, kGroupThreads, kEpiBar,
+                                                            RAGGED ? us.shift : 0);
                     }
                 } else if (ncta == 1) {
-                    finalize_fast<G, true>(a, u, t, n, 1, evict, fin_sm, etid, kEpiBar, o, cml);
+                    finalize_fast<G, true>(a, u, t, us.n, 1, us.evict, fin_sm, etid, kEpiBar, o, cml, RAGGED ? us.shift : 0);
                 } else {
                     // the unit is shared: publish this CTA's partial; the last CTA to do so finishes the unit.
                     // The group barrier orders every thread's writes (and, through the mbarrier above, the compute
@@ -921,9 +930,10 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     group_sync(kEpiBar, kGroupThreads);
                     if (*flag) {
                         if (ncta <= 8 && ncta * G * 2 <= 256)
-                            finalize_fast<G, false>(a, u, t, n, ncta, evict, fin_sm, etid, kEpiBar, o, nullptr);
+                            finalize_fast<G, false>(a, u, t, us.n, ncta, us.evict, fin_sm, etid, kEpiBar, o, nullptr, RAGGED ? us.shift : 0);
                         else
-                            finalize_unit<__nv_bfloat16, kD, G>(a, u, t, n, ncta, evict, fin_sm, etid, kGroupThreads, kEpiBar);
+                            finalize_unit<__nv_bfloat16, kD, G>(a, u, t, us.n, ncta, us.evict, fin_sm, etid, kGroupThreads, kEpiBar,
+                                                                RAGGED ? us.shift : 0);
                     }
                 }
                 group_sync(kEpiBar, kGroupThreads);
@@ -948,18 +958,18 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
 struct TcPlan {
     CUtensorMap tmK, tmV, tmQ;
     TcGeom geo;
-    bool attr_set[5][2][2];
+    bool attr_set[5][2][3];
 };
 
 namespace {
 
 int group_index(int G) { return G == 1 ? 0 : G == 2 ? 1 : G == 4 ? 2 : G == 8 ? 3 : G == 16 ? 4 : -1; }
 
-template <int G, int FUSION, int NG, bool MC>
+template <int G, int FUSION, int NG, bool MC, bool RAGGED>
 cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    auto kern = decode_tc_kernel<G, FUSION, NG, MC>;
-    bool &set = plan->attr_set[group_index(G)][FUSION][MC ? 1 : 0];
+    auto kern = decode_tc_kernel<G, FUSION, NG, MC, RAGGED>;
+    bool &set = plan->attr_set[group_index(G)][FUSION][MC ? 1 : RAGGED ? 2 : 0];
     if (!set) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan->geo.smem_bytes);
         if (e != cudaSuccess) return e;
@@ -983,8 +993,9 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 template <int G, int FUSION>
 cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    return plan->geo.nc > 1 ? launch_gfn<G, FUSION, kComputeGroups, true>(plan, a, stream)
-                            : launch_gfn<G, FUSION, kComputeGroups, false>(plan, a, stream);
+    if (plan->geo.nc > 1) return a.row_n ? cudaErrorInvalidValue : launch_gfn<G, FUSION, kComputeGroups, true, false>(plan, a, stream);
+    return a.row_n ? launch_gfn<G, FUSION, kComputeGroups, false, true>(plan, a, stream)
+                   : launch_gfn<G, FUSION, kComputeGroups, false, false>(plan, a, stream);
 }
 
 template <int G>

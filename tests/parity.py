@@ -376,3 +376,113 @@ def run_parity_coarse(w: synth.Workload, T: int, steps: int, n_units: int = 4, k
     rep.F_compared = peak        # reused: the largest fill seen (C + R + T - 1 expected)
     mk.close()
     return rep
+
+
+def run_parity_ragged(w: synth.Workload, prompt_lens, steps: int, kernel: str = "auto", per_layer: int = 0,
+                      norm: str = "frozen", device: str = "cuda:0", full_layers: int = 0, max_tokens: int = 0,
+                      synth_device=None) -> ParityReport:
+    """Lock-step parity for a batch whose rows have prompts of different lengths (`prompt_lens[b]`; `w.prompt_len`
+    is ignored).  Every unit of the workload is checked.  Row b's stream is the workload's stream of that row: its
+    prompt is positions [0, prompt_lens[b]) and its token of decode step s has position prompt_lens[b] + s, so each
+    oracle unit is simply that row's sequence run alone.  The padding of the prompt tensors beyond a row's length
+    holds huge values: a kernel that read it would miss the output tolerance at once."""
+    dev = torch.device(device)
+    st = _DeviceStream(w, synth_device or dev, dev)
+    tdt = synth.torch_dtype(w.dtype)
+    G, d, R, C_ = w.group, w.head_dim, w.R, w.C
+    B, Hkv, L = w.batch, w.n_kv_heads, w.layers
+    assert len(prompt_lens) == B
+    Pm = max(prompt_lens)
+    rep = ParityReport()
+    mk = binding.MorphKV(L, B, w.n_q_heads, Hkv, d, C_, R, w.fusion, w.dtype, kernel=kernel, device=device, norm=norm,
+                         full_layers=full_layers, max_tokens=max_tokens)
+    rep.kernel = mk.kernel_name
+    C_of = {l: (max_tokens - R if l < full_layers else C_) for l in range(L)}
+    tol = TOL_OUT[w.dtype]
+    k32, v32 = st.kv(np.arange(Pm))                       # [L,B,Hkv,Pm,d]
+    q32 = st.q(np.arange(Pm))                             # [L,B,Hq,Pm,d]
+    qw_len = min(R, Pm)
+    k_all, v_all = k32.to(tdt).clone(), v32.to(tdt).clone()
+    qw_all = torch.full((L, B, w.n_q_heads, qw_len, d), 1.0e4, dtype=tdt, device=dev)
+    for b, P in enumerate(prompt_lens):
+        Rw = min(R, P)
+        k_all[:, b, :, P:] = 1.0e4
+        v_all[:, b, :, P:] = 1.0e4
+        qw_all[:, b, :, :Rw] = q32[:, b, :, P - Rw:P].to(tdt)
+    mk.prefill_ragged(k_all.contiguous(), v_all.contiguous(), qw_all.contiguous(), list(prompt_lens))
+    mk.sync()
+    units = [(l, b, h) for l in range(L) for b in range(B) for h in range(Hkv)]
+    orac = {}
+    for l in range(L):
+        view = mk.view(l)
+        cnt, nxt = mk.row_state(l)
+        assert nxt == list(prompt_lens), (nxt, prompt_lens)
+        for b, P in enumerate(prompt_lens):
+            Rw = min(R, P)
+            assert cnt[b] == (C_of[l] + Rw if P - Rw > C_of[l] else P), (l, b, cnt[b])
+            for h in range(Hkv):
+                gp = view["pos"][b, h, :cnt[b]].cpu().numpy()
+                u, resync = oracle_unit_following(
+                    lambda: ora.Unit(G, d, C_of[l], R, w.fusion, norm=norm), _f64(k32[l, b, h, :P]), _f64(v32[l, b, h, :P]),
+                    _f64(q32[l, b, h * G:(h + 1) * G, P - Rw:P]), gp, f"unit {(l, b, h)}")
+                rep.prefill_resyncs += int(resync)
+                idx = torch.from_numpy(gp).long().to(dev)
+                assert torch.equal(view["K"][b, h, :cnt[b]], k_all[l, b, h][idx]), f"unit {(l, b, h)}: K rows differ from the prompt's"
+                assert torch.equal(view["V"][b, h, :cnt[b]], v_all[l, b, h][idx]), f"unit {(l, b, h)}: V rows differ from the prompt's"
+                orac[(l, b, h)] = u
+    rep.units = len(orac)
+    for i in range(steps):
+        # row b's token of this step has position prompt_lens[b] + i
+        q1 = torch.empty((L, B, w.n_q_heads, d), dtype=torch.float32, device=dev)
+        k1 = torch.empty((L, B, Hkv, d), dtype=torch.float32, device=dev)
+        v1 = torch.empty_like(k1)
+        for P in sorted(set(prompt_lens)):
+            kk, vv = st.kv([P + i])
+            qq = st.q([P + i])
+            for b in [b for b in range(B) if prompt_lens[b] == P]:
+                q1[:, b], k1[:, b], v1[:, b] = qq[:, b, :, 0], kk[:, b, :, 0], vv[:, b, :, 0]
+        qs, ks, vs = q1.to(tdt).contiguous(), k1.to(tdt).contiguous(), v1.to(tdt).contiguous()
+        out = torch.empty_like(qs)
+        if per_layer == 1 or (per_layer == 2 and i % 2 == 1):
+            for l in range(L):
+                mk.decode_step_layer(l, qs[l], ks[l], vs[l], out[l])
+        else:
+            mk.decode_step(qs, ks, vs, out)
+        mk.sync()
+        out_c = out.float().cpu().numpy()
+        q_c, k_c, v_c = _f64(q1), _f64(k1), _f64(v1)
+        for l in range(L):
+            view = mk.view(l)
+            cnt, nxt = mk.row_state(l)
+            ev = view["evicted_pos"].cpu().numpy()
+            pos_l = view["pos"].cpu().numpy()
+            for b in range(B):
+                t = prompt_lens[b] + i
+                assert nxt[b] == t + 1
+                for h in range(Hkv):
+                    u = orac[(l, b, h)]
+                    e_g = int(ev[b, h])
+                    o = u.step(np.ascontiguousarray(q_c[l, b, h * G:(h + 1) * G]), k_c[l, b, h], v_c[l, b, h],
+                               forced=[e_g] if e_g >= 0 else None)
+                    err = float(np.abs(o - out_c[l, b, h * G:(h + 1) * G]).max())
+                    rep.max_out_err = max(rep.max_out_err, err)
+                    assert err <= tol, f"unit {(l, b, h)} position {t}: attention output error {err:.3e} > {tol}"
+                    cp, cF = u.last_scores()
+                    if len(cp) > C_of[l]:
+                        rep.evictions += 1
+                        assert e_g >= 0, f"unit {(l, b, h)} position {t}: device did not evict"
+                        own = int(cp[C_of[l]])
+                        if e_g != own:
+                            Fg = float(cF[np.nonzero(cp == e_g)[0][0]])
+                            assert near_tie(Fg, float(cF[C_of[l]])), \
+                                f"unit {(l, b, h)} position {t}: device evicted {e_g}, the oracle ranks {own} last, no near tie"
+                            rep.near_tie_resyncs += 1
+                    else:
+                        assert e_g == -1, f"unit {(l, b, h)} position {t}: device evicted {e_g} but the row's cache is not full"
+                    assert cnt[b] == u.count, f"unit {(l, b, h)} position {t}: fill {cnt[b]} against the oracle's {u.count}"
+                    assert set(pos_l[b, h, :cnt[b]].tolist()) == set(u.positions().tolist()), \
+                        f"unit {(l, b, h)} position {t}: retained sets differ"
+                    rep.unit_steps += 1
+        rep.steps = i + 1
+    mk.close()
+    return rep

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from paper_2503_00979_b200 import binding, synth
-from tests.parity import run_parity, run_parity_coarse
+from tests.parity import run_parity, run_parity_coarse, run_parity_ragged
 
 pytestmark = pytest.mark.gpu
 
@@ -676,3 +676,40 @@ def test_tc_runs_are_bitwise_reproducible(ipu):
         mk.close()
     for r in runs[1:]:
         assert torch.equal(r[0], runs[0][0]) and torch.equal(r[1], runs[0][1]) and torch.equal(r[2], runs[0][2])
+
+
+# ---- batch rows with prompts of different lengths
+@pytest.mark.parametrize("kernel,dtype,d", [("tc", "bf16", 128), ("simt", "bf16", 128), ("simt", "f32", 64)])
+def test_ragged_prompt_lengths_per_batch_row(kernel, dtype, d):
+    # C + R = 216: row 0 starts full and evicts from the first step, row 1 reaches capacity after 66 steps, row 2
+    # starts shorter than the window, row 3 is the longest and sets the common time axis
+    w = synth.Workload("ragged", 2, 4, 8, 2, d, dtype, 0, 90, 200, 16, "sum", 606)
+    rep = run_parity_ragged(w, [300, 150, 9, 411], steps=w.steps, kernel=kernel)
+    _report(rep)
+    assert rep.kernel == kernel and rep.units == 16
+    assert rep.evictions == 4 * (90 + 24 + 0 + 90)        # 4 units per row
+
+
+def test_ragged_rows_with_per_layer_calls_layer_aware_and_current_normalisation():
+    w = synth.Workload("ragged2", 3, 3, 14, 2, 128, "bf16", 0, 40, 120, 12, "max", 607)      # group 7 -> 8
+    rep = run_parity_ragged(w, [140, 77, 200], steps=w.steps, kernel="auto", per_layer=2)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+    rep = run_parity_ragged(w, [140, 77, 200], steps=w.steps, kernel="auto", full_layers=1, max_tokens=256)
+    _report(rep)
+    assert rep.evictions > 0
+    rep = run_parity_ragged(w, [140, 77, 200], steps=w.steps, kernel="auto", norm="current")
+    _report(rep)
+    assert rep.evictions > 0
+
+
+def test_ragged_prefill_rejects_what_it_does_not_support():
+    mk = binding.MorphKV(1, 2, 8, 2, 128, 64, 16, "sum", "bf16", evict_interval=4)
+    k = torch.zeros((1, 2, 2, 100, 128), dtype=torch.bfloat16, device="cuda:0")
+    q = torch.zeros((1, 2, 8, 16, 128), dtype=torch.bfloat16, device="cuda:0")
+    assert binding.mkv_prefill_ragged(mk.ctx, k, k, q, [100, 50], 100) == binding.UNSUPPORTED
+    mk.close()
+    mk = binding.MorphKV(1, 2, 8, 2, 128, 64, 16, "sum", "bf16")
+    assert binding.mkv_prefill_ragged(mk.ctx, k, k, q, [100, 101], 100) == binding.INVALID_ARG
+    assert binding.mkv_prefill_ragged(mk.ctx, k, k, q, [100, 0], 100) == binding.INVALID_ARG
+    mk.close()
