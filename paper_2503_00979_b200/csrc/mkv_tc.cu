@@ -38,6 +38,7 @@
 
 #include "mkv_common.cuh"
 #include "mkv_kernels.h"
+#include "mkv_schedule.h"
 #include "mkv_sm100.cuh"
 
 namespace mkv {
@@ -88,71 +89,8 @@ __host__ __device__ inline SmemLayout tc_smem_layout(const TcGeom &g, int G)
     return L;
 }
 
-// ---------------------------------------------------------------- schedule shared by all roles
-struct Item {
-    int unit, tile0, nk;      // tiles [tile0, tile0 + nk) of the unit
-};
-// The same deterministic walk over this CTA's items in every role.  With nt tiles per unit at
-// the current cache length, global tile i is tile i % nt of unit i / nt, and CTA c of the
-// E = min(grid, U * nt) working CTAs owns tiles [c * T / E, (c + 1) * T / E), T = U * nt: every
-// working CTA owns at least one tile and consecutive items belong to different units.
-struct Walk {
-    int tile, tile_begin, tile_end;   // the host keeps U * tiles per unit below 2^31
-    int nt;           // tiles per unit
-    int unit, off;    // unit and tile inside it of `tile`
-    int nitems;       // items returned so far (= units seen: ring loads, partials)
-    int T0;           // tiles of the items already advanced over
-    int eff;          // working CTAs
-    long long total;
-    __device__ Walk(int U, int n)
-    {
-        nt = (n + kTile - 1) / kTile;
-        total = (long long)U * nt;
-        eff = (int)(total < (long long)gridDim.x ? total : (long long)gridDim.x);
-        if ((int)blockIdx.x < eff) {
-            tile = (int)(total * blockIdx.x / eff);
-            tile_end = (int)(total * (blockIdx.x + 1) / eff);
-        } else {
-            tile = tile_end = 0;
-        }
-        tile_begin = tile;
-        unit = tile / nt;
-        off = tile - unit * nt;
-        nitems = 0; T0 = 0;
-    }
-    __device__ bool next(Item &x)
-    {
-        if (tile >= tile_end) return false;
-        x.unit = unit;
-        x.tile0 = off;
-        x.nk = min(nt - off, tile_end - tile);
-        tile += x.nk;
-        off += x.nk;
-        if (off == nt) { off = 0; ++unit; }
-        return true;
-    }
-    __device__ void advance(const Item &x)
-    {
-        T0 += x.nk;
-        ++nitems;
-    }
-    // the CTA that owns global tile i: the largest c with c * T / E <= i
-    __device__ int owner(long long i) const { return (int)(((i + 1) * eff - 1) / total); }
-    // How many CTAs hold tiles of unit u, and this CTA's index among them.
-    __device__ int ctas_of_unit(int u, int &my_index) const
-    {
-        const long long i0 = (long long)u * nt;
-        const int c0 = owner(i0), c1 = owner(i0 + nt - 1);
-        my_index = (int)blockIdx.x - c0;
-        return c1 - c0 + 1;
-    }
-    // true if all tiles of unit u belong to this CTA
-    __device__ bool unit_is_local(int u) const
-    {
-        const int first = u * nt;
-        return first >= tile_begin && first + nt <= tile_end;
-    }
-};
+// ---------------------------------------------------------------- schedule shared by all roles: mkv_schedule.h
+static_assert(kSchedTile == kTile, "the schedule and the kernel must agree on the tile");
 
 // position in a ring of n slots (stage or accumulator buffer) and the parity of the lap,
 // advanced without divisions
@@ -449,7 +387,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     if (warp == 0) {
         // ------------------------------------------------ TMA producer: query ring and K tiles (one lane)
         if (lane == 0) {
-            Walk w(a.U * NCe, n);
+            Walk w(a.U * NCe, n, (int)gridDim.x, (int)blockIdx.x);
             Item x;
             int issued = 0, rings = 0;
             bool ok = true;
@@ -489,7 +427,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     } else if (warp == 2) {
         // ------------------------------------------------ TMA producer: V tiles (one lane)
         if (lane == 0) {
-            Walk w(a.U * NCe, n);
+            Walk w(a.U * NCe, n, (int)gridDim.x, (int)blockIdx.x);
             Item x;
             int issued = 0;                                 // V tiles loaded so far (only main chunks read V)
             bool ok = true;
@@ -519,7 +457,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         __syncwarp();       // see the K producer
     } else if (warp == 1) {
         // ------------------------------------------------ new-query substitution + MMA issue
-        Walk w(a.U * NCe, n);
+        Walk w(a.U * NCe, n, (int)gridDim.x, (int)blockIdx.x);
         Item x;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(RGP >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
         bool ok = true;
@@ -611,7 +549,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         int seg_tiles = 0;
         int npub = 0;                                  // partials this warp has handed to the epilogue group
 
-        Walk w(a.U * NCe, n);
+        Walk w(a.U * NCe, n, (int)gridDim.x, (int)blockIdx.x);
         Item x;
         bool ok = true;
         int Tn = grp;                                  // next tile of this group
@@ -834,7 +772,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
         int *flag = reinterpret_cast<int *>(epi + kFinFloats);
         float *cml = epi + kFinFloats + 8;                            // merged (m, l) [g][2]
         float *sc = cml + 2 * kMaxGroup;                              // [warp][g] scale to the merged reference
-        Walk w(a.U * NCe, n);
+        Walk w(a.U * NCe, n, (int)gridDim.x, (int)blockIdx.x);
         Item x;
         bool ok = true;
         int k = 0;                                                    // units finished so far
@@ -1040,37 +978,9 @@ bool tc_shape_supported(bool f32, int D, int G, int R)
     return tc_ring_chunks(G, R) <= kMaxRingChunks;
 }
 
-// Grid of the persistent kernel.  `splits_hint` > 0 asks for about that many CTAs per unit
-// (ranges of cap_tiles / splits_hint tiles); otherwise one CTA per SM.
-int tc_grid(int U, int cap, int splits_hint, int n_sm)
-{
-    const long long ntiles = (cap + kTile - 1) / kTile, total = (long long)U * ntiles;
-    long long grid = n_sm;
-    if (splits_hint > 0) {
-        const long long chunk = (ntiles + splits_hint - 1) / splits_hint;
-        grid = (total + chunk - 1) / chunk;
-        if (grid > n_sm) grid = n_sm;
-    }
-    if (grid > total) grid = total;
-    return (int)(grid < 1 ? 1 : grid);
-}
+int tc_grid(int U, int cap, int splits_hint, int n_sm) { return sched_grid(U, cap, splits_hint, n_sm); }
 
-// Upper bound, over every cache length up to cap, of the CTAs that hold tiles of one unit
-// (= partial slots a unit needs).
-int tc_partials_per_unit(int U, int cap, int grid)
-{
-    const int ntiles = (cap + kTile - 1) / kTile;
-    int worst = 1;
-    for (int nt = 1; nt <= ntiles; ++nt) {
-        const long long total = (long long)U * nt;
-        const long long eff = total < grid ? total : grid;
-        const long long len = total / eff;                     // shortest range of a CTA
-        long long c = (nt + len - 1) / len + 1;
-        if (c > nt) c = nt;
-        if (c > worst) worst = (int)c;
-    }
-    return worst;
-}
+int tc_partials_per_unit(int U, int cap, int grid) { return sched_partials_per_unit(U, cap, grid); }
 
 cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned long long wait_limit_cycles, char *err,
                            size_t err_len)
