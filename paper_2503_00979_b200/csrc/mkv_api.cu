@@ -191,6 +191,7 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.row_n = c->ragged ? (int *)(b + c->L.rows) : nullptr;
     a.row_shift = c->ragged ? (const int *)(b + c->L.row_shift) : nullptr;
     a.B = c->s.B; a.Hkv = c->s.Hkv;
+    a.n_hint = c->prefilled ? c->n : 0;
     return a;
 }
 
@@ -318,8 +319,8 @@ mkv_status core_create(mkv_ctx **out, const mkv_params *p, void *workspace, size
     if (kind == kKindTc) {
         const DecodeArgs a = make_args(c, nullptr, nullptr, nullptr, nullptr);
         char msg[200] = "";
-        cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, p->wait_limit_cycles, msg, sizeof(msg));
-        if (e == cudaSuccess) e = tc_plan_create(&c->plan_layer, a, s.tc_grid_layer, p->wait_limit_cycles, msg, sizeof(msg));
+        cudaError_t e = tc_plan_create(&c->plan, a, s.tc_grid_size, p->wait_limit_cycles, true, msg, sizeof(msg));
+        if (e == cudaSuccess) e = tc_plan_create(&c->plan_layer, a, s.tc_grid_layer, p->wait_limit_cycles, false, msg, sizeof(msg));
         if (e != cudaSuccess) {
             cudaGetLastError();
             if (c->plan) tc_plan_destroy(c->plan);

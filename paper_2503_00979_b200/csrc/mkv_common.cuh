@@ -62,6 +62,8 @@ struct DecodeArgs {
     int *row_n;                // [2][B]
     const int *row_shift;      // [B]
     int B, Hkv;                // unit u (of this launch) belongs to batch row (u / Hkv) % B
+    int n_hint;                // the host's view of st->n when the launch was enqueued (0: none).  Only used to
+                               // prefetch: a stale value (steps replayed from a CUDA graph) costs time, not results
 };
 
 // Fill, position offset and policy decision of one unit on this step.

@@ -25,8 +25,9 @@ int tc_ring_chunks(int G, int R);
 int tc_grid(int U, int cap, int splits_hint, int n_sm);
 int tc_partials_per_unit(int U, int cap, int grid);
 struct TcPlan;
-cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int grid, unsigned long long wait_limit_cycles, char *err,
-                           size_t err_len);
+// `prefetch`: CTAs ask for the first tiles of their range into L2 while the previous launch drains.
+cudaError_t tc_plan_create(TcPlan **plan, const DecodeArgs &a, int grid, unsigned long long wait_limit_cycles, bool prefetch,
+                           char *err, size_t err_len);
 void tc_plan_destroy(TcPlan *plan);
 cudaError_t launch_decode_tc(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream);
 

@@ -111,6 +111,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy) : "memory");
 }
 
+// Asks for the box at (x, y, z) to be brought into L2; no data reaches the SM and no barrier is involved.  The same
+// coordinate rules as for the load: x * element size a multiple of 16 bytes, out-of-range parts are skipped.
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
 // brings a tensor map into the descriptor cache ahead of its first copy
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
 {

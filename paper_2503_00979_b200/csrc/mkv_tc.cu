@@ -64,6 +64,7 @@ struct TcGeom {
     int grid;
     int smem_bytes;
     long long wait_cycles;   // limit of every device-side wait, in clock64 ticks
+    int prefetch_tiles;      // K and V tiles a CTA asks into L2 before it waits for the previous grid (0: none)
 };
 
 struct SmemLayout {
@@ -349,6 +350,27 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     // early.  Nothing that grid wrote - step state, cache rows, query ring - is read before this wait, which
     // returns once that grid has completed and its memory operations are visible.  The next grid in the stream is
     // released at once: it parks at the same wait.
+    // While the grid before this one drains (its last CTAs are in their epilogues, a chain of latencies that leaves
+    // DRAM idle), this CTA asks for the first tiles of its range to be brought into L2.  A prefetch delivers no data
+    // to the SM, so it may run before the wait below: rows that the previous grid's epilogues still overwrite are
+    // updated in L2, which is where the loads after the wait read them.  The range is computed from the host's
+    // view of the fill; if that is stale the wrong lines are prefetched and nothing else happens.  (Not in the
+    // chunked-window and ragged instantiations, whose first items depend on state read after the wait.)
+    if constexpr (!MC && !RAGGED) {
+        if ((tid == 0 || tid == 64) && a.n_hint > 0 && geo.prefetch_tiles > 0) {
+            const CUtensorMap *pm = tid == 0 ? &tmK : &tmV;
+            Walk w(a.U, a.n_hint, (int)gridDim.x, (int)blockIdx.x);
+            Item x;
+            int left = geo.prefetch_tiles;
+            while (left > 0 && w.next(x)) {
+                for (int j = 0; j < x.nk && left > 0; ++j, --left) {
+                    tma_prefetch_l2_3d(pm, 0, (x.tile0 + j) * kTile, a.u0 + x.unit);
+                    tma_prefetch_l2_3d(pm, 64, (x.tile0 + j) * kTile, a.u0 + x.unit);
+                }
+                w.advance(x);
+            }
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long t = a.st->t;
@@ -982,8 +1004,8 @@ int tc_grid(int U, int cap, int splits_hint, int n_sm) { return sched_grid(U, ca
 
 int tc_partials_per_unit(int U, int cap, int grid) { return sched_partials_per_unit(U, cap, grid); }
 
-cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned long long wait_limit_cycles, char *err,
-                           size_t err_len)
+cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned long long wait_limit_cycles, bool prefetch,
+                           char *err, size_t err_len)
 {
     *out = nullptr;
     TcPlan *p = new (std::nothrow) TcPlan;
@@ -1009,6 +1031,12 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned
     while (g.tmem_cols < g.nb * g.rgpad) g.tmem_cols *= 2;
     g.grid = grid;
     g.wait_cycles = wait_limit_cycles > 0 ? (long long)wait_limit_cycles : kWaitCycles;
+    // Two tiles: what counts is that a CTA's first loads after the wait hit L2 (config 1: 56.1 instead of 57.1 us per
+    // step with 1 to 3 tiles).  More is worse - 8 tiles cost 3 us, 32 tiles 10 us - because the prefetches compete
+    // with the previous grid's last CTAs.  Prefetching the first item's query ring as well changed nothing.
+    // A launch over one layer's few units, whose CTAs hold two tiles or so each, is slower with it (17.9 instead of
+    // 16.9 us per call): the caller asks for it on the whole-stack plan only.
+    g.prefetch_tiles = prefetch ? 2 : 0;
     // as many 32 KB stages as fit, split between the K ring (short-lived tiles) and the V ring
     int total_stages = 0;
     for (int st = 9; st >= 2; --st) {
