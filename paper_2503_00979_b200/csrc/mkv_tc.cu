@@ -882,10 +882,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     if (etid < 2 * G) pml[etid] = cml[etid];
                     group_sync(kEpiBar, kGroupThreads);
                     if (etid == 0) {
-                        __threadfence();
-                        const int last = atomicAdd(&a.ticket[u], 1) == ncta - 1;
-                        __threadfence();
-                        *flag = last;
+                        // release: the group's writes above (ordered before this thread by the barrier) become visible
+                        // to whoever observes the ticket; acquire: the last arriver's reads below see the others'
+                        int old;
+                        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(a.ticket + u) : "memory");
+                        *flag = old == ncta - 1;
                     }
                     group_sync(kEpiBar, kGroupThreads);
                     if (*flag) {
