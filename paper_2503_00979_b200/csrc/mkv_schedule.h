@@ -21,8 +21,14 @@ struct Item {
 // the current cache length, global tile i is tile i % nt of unit i / nt, and CTA c of the
 // E = min(grid, U * nt) working CTAs owns tiles [c * T / E, (c + 1) * T / E), T = U * nt: every
 // working CTA owns at least one tile and consecutive items belong to different units.
+// Order of a CTA's items: if its range ends inside a unit, that last piece comes first, then the rest in tile order.
+// A unit cut by a range boundary is then worked on early by both CTAs that hold a piece of it (the one before the
+// boundary starts with it, the one after it takes it first or second), so its cross-CTA merge runs while tiles
+// still stream, and the item a CTA ends with is a unit all of its own, whose epilogue needs no other CTA.
 struct Walk {
     int tile, tile_begin, tile_end;   // the host keeps U * tiles per unit below 2^31
+    int nat_end;      // end of the part of the range that is handed out in tile order
+    int lead_nk;      // tiles of the piece handed out first (0: none, or already handed out)
     int nt;           // tiles per unit
     int unit, off;    // unit and tile inside it of `tile`
     int nitems;       // items returned so far (= units seen: ring loads, partials)
@@ -46,13 +52,30 @@ struct Walk {
         unit = tile / nt;         // n >= 1: a context holds at least its prompt
         off = tile - unit * nt;
         nitems = 0; T0 = 0;
+        nat_end = tile_end;
+        lead_nk = 0;
+        if (tile_end > tile_begin) {
+            const int ul = (tile_end - 1) / nt;                 // the unit the range ends in
+            const int first = ul * nt;                          // its first tile
+            if (tile_end != first + nt && first > tile_begin) { // the range ends inside it and starts before it
+                nat_end = first;
+                lead_nk = tile_end - first;
+            }
+        }
     }
     MKV_HD bool next(Item &x)
     {
-        if (tile >= tile_end) return false;
+        if (lead_nk > 0) {
+            x.unit = nat_end / nt;
+            x.tile0 = 0;
+            x.nk = lead_nk;
+            lead_nk = 0;
+            return true;
+        }
+        if (tile >= nat_end) return false;
         x.unit = unit;
         x.tile0 = off;
-        x.nk = nt - off < tile_end - tile ? nt - off : tile_end - tile;
+        x.nk = nt - off < nat_end - tile ? nt - off : nat_end - tile;
         tile += x.nk;
         off += x.nk;
         if (off == nt) { off = 0; ++unit; }

@@ -1,6 +1,7 @@
 // Replays the tensor-core decode kernel's work schedule on the host, for every number of tiles per unit up to the
 // capacity, and checks what the kernel relies on:
-//   - every tile of every unit is owned by exactly one CTA, and a CTA's tiles are one contiguous range;
+//   - every tile of every unit is owned by exactly one CTA, and a CTA's tiles are one contiguous range (handed out
+//     with the piece of a unit at the end of the range first, the rest in tile order);
 //   - a CTA's consecutive items belong to different units (one ring load and one partial per item);
 //   - ctas_of_unit() agrees with the CTAs that really hold tiles of the unit (the ticket count of the unit's
 //     epilogue), and their indices are 0 .. ncta-1 in CTA order;
@@ -34,14 +35,24 @@ int main(int argc, char **argv)
                 Walk w(U, n, grid, cta);
                 Item x;
                 int prev_unit = -1, seen = 0;
-                long long expect_tile = w.tile_begin;
+                long long got_tiles = 0, expect_tile = w.tile_begin;
+                const bool lead = w.lead_nk > 0;
                 while (w.next(x)) {
                     if (x.unit < 0 || x.unit >= U || x.nk < 1 || x.tile0 < 0 || x.tile0 + x.nk > nt) {
                         printf("bad item: n=%d cta=%d unit=%d tile0=%d nk=%d\n", n, cta, x.unit, x.tile0, x.nk);
                         return 1;
                     }
                     if (x.unit == prev_unit) { printf("n=%d cta=%d: two items of unit %d in a row\n", n, cta, x.unit); return 1; }
-                    if ((long long)x.unit * nt + x.tile0 != expect_tile) { printf("n=%d cta=%d: range not contiguous\n", n, cta); return 1; }
+                    const long long g0 = (long long)x.unit * nt + x.tile0;
+                    if (g0 < w.tile_begin || g0 + x.nk > w.tile_end) { printf("n=%d cta=%d: item outside the CTA's range\n", n, cta); return 1; }
+                    if (lead && seen == 0) {
+                        // the piece at the end of the range: a proper part of its unit, starting at the unit's first tile
+                        if (x.tile0 != 0 || x.nk >= nt || g0 + x.nk != w.tile_end) { printf("n=%d cta=%d: bad leading piece\n", n, cta); return 1; }
+                    } else {
+                        if (g0 != expect_tile) { printf("n=%d cta=%d: range not in tile order\n", n, cta); return 1; }
+                        expect_tile += x.nk;
+                    }
+                    got_tiles += x.nk;
                     if ((x.tile0 + x.nk) * kSchedTile > ntiles * kSchedTile) { printf("n=%d cta=%d: key row beyond the capacity\n", n, cta); return 1; }
                     for (int j = 0; j < x.nk; ++j) {
                         int &o = owner[(size_t)x.unit * nt + x.tile0 + j];
@@ -58,12 +69,11 @@ int main(int argc, char **argv)
                     }
                     ++next_index[x.unit];
                     ++holders[x.unit];
-                    expect_tile += x.nk;
                     prev_unit = x.unit;
                     w.advance(x);
                     ++seen;
                 }
-                if (expect_tile != w.tile_end) { printf("n=%d cta=%d: walk stopped early\n", n, cta); return 1; }
+                if (got_tiles != w.tile_end - w.tile_begin) { printf("n=%d cta=%d: walk stopped early\n", n, cta); return 1; }
                 if (w.nitems != seen || w.T0 != w.tile_end - w.tile_begin) { printf("n=%d cta=%d: counters off\n", n, cta); return 1; }
             }
             for (size_t i = 0; i < owner.size(); ++i)
