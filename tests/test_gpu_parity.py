@@ -713,3 +713,62 @@ def test_ragged_prefill_rejects_what_it_does_not_support():
     assert binding.mkv_prefill_ragged(mk.ctx, k, k, q, [100, 101], 100) == binding.INVALID_ARG
     assert binding.mkv_prefill_ragged(mk.ctx, k, k, q, [100, 0], 100) == binding.INVALID_ARG
     mk.close()
+
+
+# ---- the step index lives on the device: steps recorded in a CUDA graph and replayed
+@pytest.mark.parametrize("kernel,dtype,d", [("tc", "bf16", 128), ("simt", "f32", 64)])
+def test_steps_replayed_from_a_cuda_graph_equal_direct_calls(kernel, dtype, d):
+    # Four steps are captured once (launches only, on a side stream) and replayed three times with fresh inputs in
+    # the same buffers; a second context takes the same twelve steps by direct calls.  Outputs bit for bit, the
+    # same retained positions, and the host mirror follows the device state after mkv_sync.  The cache fills
+    # during the first replays and evicts afterwards, so the graph's launches meet both kinds of step.
+    w = synth.Workload("graph", 2, 2, 8, 2, d, dtype, 90, 12, 80, 16, "max", 808)
+    dev = torch.device("cuda:0")
+    tdt = synth.torch_dtype(dtype)
+    st = synth.Stream(w, dev)
+    P, S, reps = w.prompt_len, 4, 3
+    k, v = st.kv(np.arange(P))
+    qw = st.q(np.arange(P - w.R, P))
+    kk, vv = st.kv(np.arange(P, P + S * reps))
+    qq = st.q(np.arange(P, P + S * reps))
+    qs = qq.permute(3, 0, 1, 2, 4).to(tdt).contiguous()        # [steps, L, B, Hq, d]
+    ks = kk.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+    vs = vv.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
+
+    def fresh():
+        mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, d, w.C, w.R, w.fusion, dtype, kernel=kernel)
+        mk.prefill(k.to(tdt).contiguous(), v.to(tdt).contiguous(), qw.to(tdt).contiguous())
+        mk.sync()
+        return mk
+
+    direct = fresh()
+    want = torch.empty_like(qs)
+    for i in range(S * reps):
+        direct.decode_step(qs[i], ks[i], vs[i], want[i])
+    direct.sync()
+
+    mk = fresh()
+    q_in, k_in, v_in = torch.empty_like(qs[:S]), torch.empty_like(ks[:S]), torch.empty_like(vs[:S])
+    out = torch.empty_like(qs[:S])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for i in range(S):
+            mk.decode_step(q_in[i], k_in[i], v_in[i], out[i], stream=torch.cuda.current_stream())
+    # the capture enqueued nothing: the context's host mirror ran ahead by S steps, the device did not
+    mk.sync()
+    got = torch.empty_like(qs)
+    for r in range(reps):
+        q_in.copy_(qs[r * S:(r + 1) * S]); k_in.copy_(ks[r * S:(r + 1) * S]); v_in.copy_(vs[r * S:(r + 1) * S])
+        g.replay()
+        torch.cuda.synchronize()
+        got[r * S:(r + 1) * S] = out
+    mk.sync()
+    assert torch.equal(got, want)
+    for l in range(w.layers):
+        a, b = mk.view(l), direct.view(l)
+        assert a["count"] == b["count"] and a["next_pos"] == b["next_pos"] == P + S * reps
+        assert torch.equal(torch.sort(a["pos"][:, :, :a["count"]], dim=-1).values, torch.sort(b["pos"][:, :, :b["count"]], dim=-1).values)
+    mk.close()
+    direct.close()
