@@ -47,7 +47,7 @@ NOMINAL_HBM_GBS = 7700.0
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
 # capture of a launch of that workload), valid only for the kernel sources it was taken with.
-_TRAFFIC = {"c1": {"bytes": 284.1e6, "sources_sha256": "7435109163d3524ba9fb9fa3e894339858d2d30986238975b980e87251ce04da"}}
+_TRAFFIC = {"c1": {"bytes": 284.1e6, "sources_sha256": "17674191a2b155fdd107782d84a585c031b50a3ee0ce5982b608d4e675924e51"}}
 
 
 def measured_traffic(workload: str):
