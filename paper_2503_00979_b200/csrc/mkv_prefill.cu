@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__rest
 {
     __shared__ unsigned int hist[256];
     __shared__ unsigned long long prefix_s;
-    __shared__ int remaining_s;
+    __shared__ int remaining_s, done_s;
     __shared__ int wtot[kPT / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int u = ub0 + blockIdx.x, M = P - Rw;
@@ -202,13 +202,20 @@ __global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__rest
                 if (acc + (int)hist[b] >= remaining) break;
                 acc += (int)hist[b];
             }
+            const unsigned long long np = (prefix << 8) | (unsigned long long)b;
+            // the bucket fills the remaining places exactly: every key in it is kept, so the smallest key with
+            // this prefix is the threshold and the finer passes (mostly tie-breaking position bits) are not needed
+            const bool exact = acc + (int)hist[b] == remaining;
             remaining_s = remaining - acc;
-            prefix_s = (prefix << 8) | (unsigned long long)b;
+            prefix_s = exact ? np << shift : np;
+            done_s = exact ? 1 : 0;
         }
         __syncthreads();
         prefix = prefix_s;
         remaining = remaining_s;
+        const bool done = done_s != 0;
         __syncthreads();
+        if (done) break;
     }
     int base = 0;
     for (int c0 = 0; c0 < M; c0 += kPT) {
@@ -261,6 +268,21 @@ __global__ void prefill_ring_kernel(const T *__restrict__ qwin, DecodeArgs a, in
         if (g < Gq) rq[((size_t)rslot * G + g) * D + dd] = qwin[(((size_t)u * Gq + g) * Rws + i) * D + dd];
         else stf(rq + ((size_t)rslot * G + g) * D + dd, 0.f);
     }
+}
+
+// the same, 16 bytes per thread (q_window 16-byte aligned)
+template <typename T, int D>
+__global__ void prefill_ring_vec_kernel(const T *__restrict__ qwin, DecodeArgs a, int P, int Rw, int Rws, int shift)
+{
+    constexpr int CH = D * sizeof(T) / 16;
+    const int u = blockIdx.x, G = a.G, Gq = a.Gq;
+    const int idx = blockIdx.y * blockDim.x + threadIdx.x;
+    if (idx >= Rw * G * CH) return;
+    const int c = idx % CH, g = (idx / CH) % G, i = idx / (CH * G);
+    const int rslot = (P - Rw + i + shift) % a.R;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (g < Gq) v = reinterpret_cast<const uint4 *>(qwin + (((size_t)u * Gq + g) * Rws + i) * D)[c];
+    reinterpret_cast<uint4 *>(static_cast<T *>(a.ring_q) + (((size_t)u * a.R + rslot) * G + g) * D)[c] = v;
 }
 
 // The prompt phase on a scratch area of `scratch_floats` floats (the window-row logits S and the fused scores of
@@ -389,7 +411,10 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     }
     constexpr int CH = D * sizeof(T) / 16;
     prefill_gather_kernel<T, D><<<dim3(U, (n * CH + 255) / 256), 256, 0, stream>>>(k, v, a, Ps, n);
-    prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw, Rws, shift);
+    if (((uintptr_t)qwin & 15) == 0)
+        prefill_ring_vec_kernel<T, D><<<dim3(U, (Rw * G * CH + 255) / 256), 256, 0, stream>>>(qwin, a, P, Rw, Rws, shift);
+    else
+        prefill_ring_kernel<T, D><<<U, 256, 0, stream>>>(qwin, a, P, Rw, Rws, shift);
     if (a.norm_current && select) {
         prefill_renorm_kernel<T, D><<<dim3(Rw * G, U), kPT, 0, stream>>>(a, P, Rw, n, shift);
         ++*launches;
