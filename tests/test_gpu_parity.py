@@ -772,3 +772,43 @@ def test_steps_replayed_from_a_cuda_graph_equal_direct_calls(kernel, dtype, d):
         assert torch.equal(torch.sort(a["pos"][:, :, :a["count"]], dim=-1).values, torch.sort(b["pos"][:, :, :b["count"]], dim=-1).values)
     mk.close()
     direct.close()
+
+
+def test_reset_after_ragged_prompts_gives_a_uniform_context_again():
+    # a context that held rows of different lengths, reset and loaded with one uniform prompt, behaves like a fresh one
+    w = synth.Workload("ragged_reset", 2, 3, 8, 2, 128, "bf16", 150, 6, 100, 16, "sum", 611)
+    dev = torch.device("cuda:0")
+    st = synth.Stream(w, dev)
+    P = w.prompt_len
+    k, v = st.kv(np.arange(P))
+    qw = st.q(np.arange(P - w.R, P))
+    kb, vb, qb = k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous()
+    kk, vv = st.kv(np.arange(P, P + w.steps))
+    qq = st.q(np.arange(P, P + w.steps))
+
+    def steps(mk):
+        outs = []
+        for i in range(w.steps):
+            outs.append(mk.decode_step(qq[..., i, :].bfloat16().contiguous(), kk[..., i, :].bfloat16().contiguous(),
+                                       vv[..., i, :].bfloat16().contiguous()).clone())
+        mk.sync()
+        return torch.stack(outs), [torch.sort(mk.view(l)["pos"][:, :, :mk.view(l)["count"]], dim=-1).values.clone() for l in range(w.layers)]
+
+    fresh = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, 128, w.C, w.R, w.fusion, "bf16")
+    fresh.prefill(kb, vb, qb)
+    want = steps(fresh)
+    fresh.close()
+    mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, 128, w.C, w.R, w.fusion, "bf16")
+    mk.prefill_ragged(kb, vb, qb, [150, 60, 97])
+    mk.decode_step(qq[..., 0, :].bfloat16().contiguous(), kk[..., 0, :].bfloat16().contiguous(), vv[..., 0, :].bfloat16().contiguous())
+    mk.sync()
+    cnt, nxt = mk.row_state(0)
+    assert nxt == [151, 61, 98] and cnt == [116, 61, 98]
+    mk.reset()
+    mk.prefill(kb, vb, qb)
+    got = steps(mk)
+    cnt, nxt = mk.row_state(1)
+    assert nxt == [P + w.steps] * 3 and cnt == [w.C + w.R] * 3
+    mk.close()
+    assert torch.equal(got[0], want[0])
+    assert all(torch.equal(a, b) for a, b in zip(got[1], want[1]))
