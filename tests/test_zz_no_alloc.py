@@ -32,7 +32,7 @@ def _prefill_and_decode(w, use_static, steps=6):
     mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype)
     args = (k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
     if use_static:
-        # the call must not take device memory: the driver's free-byte count is the same before and after
+        # the call must not take device memory: the CUDA runtime's free-byte count is the same before and after
         torch.cuda.synchronize()
         free_before = torch.cuda.mem_get_info()[0]
         mk.prefill_static(*args)
