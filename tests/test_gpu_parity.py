@@ -812,3 +812,13 @@ def test_reset_after_ragged_prompts_gives_a_uniform_context_again():
     mk.close()
     assert torch.equal(got[0], want[0])
     assert all(torch.equal(a, b) for a, b in zip(got[1], want[1]))
+
+
+@pytest.mark.parametrize("lens", [[5, 9, 3], [7], [40, 40, 40]])
+def test_ragged_prompts_degenerate_cases(lens):
+    # every prompt shorter than the window (the padded tensors are then shorter than R too), a batch of one row, and
+    # rows that happen to be equally long
+    w = synth.Workload("ragged_edge", 2, len(lens), 8, 2, 128, "bf16", 0, 50, 30, 16, "sum", 612)
+    rep = run_parity_ragged(w, lens, steps=w.steps, kernel="auto")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
