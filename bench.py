@@ -411,7 +411,8 @@ def run_ours(args, w):
 
     st = synth.Stream(w, dev)
     mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.C, w.R, w.fusion, w.dtype,
-                         evict_interval=args.evict_interval, kernel=args.kernel, splits=args.splits, device=str(dev))
+                         evict_interval=args.evict_interval, kernel=args.kernel, splits=args.splits, device=str(dev),
+                         profile=args.profile)
     # prompt phase (untimed), drawn layer by layer to bound the temporary memory
     ks, vs, qws = [], [], []
     for l in range(w.layers):
@@ -505,7 +506,7 @@ def run_ours(args, w):
             "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
                        "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "C": w.C, "R": w.R, "fusion": w.fusion,
                        "prompt_len": P, "evict_interval": T, "cached_tokens_per_unit": n_steady, "units_per_gpu": w.units,
-                       "kernel": mk.kernel_name, "parallelism": f"replicas x{world}",
+                       "kernel": mk.kernel_name, "profile_mode": args.profile, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2: each step streams the whole K/V cache "
                              f"({bytes_step / 1e6:.0f} MB per step against 126 MB of L2)"},
             "clocks": clocks.summary(),
@@ -549,6 +550,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--profile", default="recompute", choices=["recompute", "stored"],
+                    help="where the window tokens' attention profiles come from (mkv_params.profile_mode); the roofline "
+                         "figure keeps the algorithmic bytes of the default mode")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--cpu-steps", type=int, default=512, help="steady-state steps per unit for the CPU baseline")
     ap.add_argument("--prompt-len", type=int, default=0,

@@ -55,6 +55,14 @@ typedef enum mkv_dtype { MKV_DTYPE_BF16 = 0, MKV_DTYPE_F32 = 1 } mkv_dtype;
  * token was generated ("the attention weight that w_r assigned").  CURRENT: renormalised over the tokens that are
  * still cached when the scores are taken (a row never saw tokens newer than itself); not with evict_interval > 1. */
 typedef enum mkv_norm { MKV_NORM_FROZEN = 0, MKV_NORM_CURRENT = 1 } mkv_norm;
+/* where the window tokens' attention profiles come from when the fused scores are taken (Eq. 4-6):
+ * RECOMPUTE (default): from the stored window queries and their frozen soft-max normalisers, inside the decode
+ *   kernel (same numbers, no table);
+ * STORED: from a table of the weights themselves, kept beside the KV cache as the paper's implementation keeps
+ *   them (Implementation paragraph): R * (C + R) more floats per unit, read once per policy step.  Trades bytes
+ *   for arithmetic; it pays for wide windows.  bf16 / head_dim 128 on the tensor-core kernel only, with per-step
+ *   eviction and MKV_NORM_FROZEN; not with mkv_prefill_ragged. */
+typedef enum mkv_profile { MKV_PROFILE_RECOMPUTE = 0, MKV_PROFILE_STORED = 1 } mkv_profile;
 typedef enum mkv_kernel { MKV_KERNEL_AUTO = 0, MKV_KERNEL_SIMT = 1, MKV_KERNEL_TC = 2 } mkv_kernel;
 
 typedef struct mkv_ctx mkv_ctx;
@@ -82,6 +90,8 @@ typedef struct mkv_params {
     int max_tokens;         /* with full_layers > 0: the cache of those layers holds this many tokens (prompt
                                plus generated; > R).  While the sequence stays within it nothing is evicted
                                there; beyond it those layers fall back to MorphKV with that capacity.    */
+    mkv_profile profile_mode;
+                            /* MKV_PROFILE_RECOMPUTE (default) or MKV_PROFILE_STORED                         */
     unsigned long long wait_limit_cycles;
                             /* how long a device-side wait (on a copy, on the tensor cores, on another
                                warp) may spin before the kernel gives up, in GPU clock ticks; 0 = the

@@ -23,6 +23,7 @@ FUSION = {"sum": 0, "max": 1}
 DTYPE = {"bf16": 0, "f32": 1}
 KERNEL = {"auto": 0, "simt": 1, "tc": 2}
 NORM = {"frozen": 0, "current": 1}
+PROFILE = {"recompute": 0, "stored": 1}
 
 EXPORTS = [
     "mkv_default_params", "mkv_workspace_bytes", "mkv_create", "mkv_create_ex", "mkv_destroy", "mkv_reset", "mkv_prefill",
@@ -38,7 +39,7 @@ class mkv_params(C.Structure):
         ("head_dim", C.c_int), ("C", C.c_int), ("R", C.c_int), ("fusion", C.c_int), ("dtype", C.c_int),
         ("evict_interval", C.c_int), ("kernel", C.c_int), ("splits", C.c_int),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("norm_mode", C.c_int), ("full_layers", C.c_int),
-        ("max_tokens", C.c_int),
+        ("max_tokens", C.c_int), ("profile_mode", C.c_int),
         ("wait_limit_cycles", C.c_ulonglong),
     ]
 
@@ -228,7 +229,7 @@ class MorphKV:
 
     def __init__(self, layers, batch, n_q_heads, n_kv_heads, head_dim, C_, R, fusion="sum", dtype="bf16",
                  evict_interval=1, kernel="auto", splits=0, device="cuda:0", wait_limit_cycles=0,
-                 full_layers=0, max_tokens=0, norm="frozen"):
+                 full_layers=0, max_tokens=0, norm="frozen", profile="recompute"):
         self.device = torch.device(device)
         p = mkv_default_params()
         p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = layers, batch, n_q_heads, n_kv_heads, head_dim
@@ -239,6 +240,7 @@ class MorphKV:
         p.wait_limit_cycles = wait_limit_cycles
         p.full_layers, p.max_tokens = full_layers, max_tokens
         p.norm_mode = NORM[norm]
+        p.profile_mode = PROFILE[profile]
         self.torch_dtype = torch.float32 if p.dtype == 1 else torch.bfloat16
         self.shape = dict(L=layers, B=batch, Hq=n_q_heads, Hkv=n_kv_heads, d=head_dim, C=C_, R=R,
                           G=n_q_heads // max(1, n_kv_heads))

@@ -16,7 +16,7 @@ using namespace mkv;
 namespace {
 
 struct Layout {
-    size_t K, V, pos, ring_q, ring_c, s_new, F, Fc, part_ml, part_o, ticket, evicted, state, rows, row_shift, stage_q, stage_k, stage_v,
+    size_t K, V, pos, ring_q, ring_c, s_new, F, Fc, prof, part_ml, part_o, ticket, evicted, state, rows, row_shift, stage_q, stage_k, stage_v,
         stage_o, total;
 };
 
@@ -29,6 +29,7 @@ struct Shape {
     int U, G, D, R, C, cap, splits, T, tc_grid_size, tc_grid_layer;
     int Gq;                 // the model's GQA ratio; G is it rounded up to a power of two on the tensor-core path
     int nc;                 // ring chunks of the tensor-core kernel (1 unless the window has more than 256 rows)
+    int stored;             // 1: the window tokens' attention profiles are kept as a table (profile_mode STORED)
     size_t es;
 };
 
@@ -45,7 +46,8 @@ Layout make_layout(const Shape &s)
     L.ring_c = take(U * R * G * 4);
     L.s_new = take(U * G * cap * 4);
     L.F = take(U * cap * 4);
-    L.Fc = take(s.nc > 1 ? U * (size_t)s.nc * cap * 4 : 0);
+    L.Fc = take(s.nc > 1 && !s.stored ? U * (size_t)s.nc * cap * 4 : 0);
+    L.prof = take(s.stored ? U * R * cap * 4 : 0);
     L.part_ml = take(U * sp * G * 2 * 4);
     L.part_o = take(U * sp * G * D * 4);
     L.ticket = take(U * 4);
@@ -73,6 +75,7 @@ bool params_valid(const mkv_params *p)
     if (p->evict_interval < 0 || p->splits < 0) return false;
     if (p->kernel != MKV_KERNEL_AUTO && p->kernel != MKV_KERNEL_SIMT && p->kernel != MKV_KERNEL_TC) return false;
     if (p->norm_mode != MKV_NORM_FROZEN && p->norm_mode != MKV_NORM_CURRENT) return false;
+    if (p->profile_mode != MKV_PROFILE_RECOMPUTE && p->profile_mode != MKV_PROFILE_STORED) return false;
     if (p->full_layers < 0 || p->full_layers >= p->layers) return false;
     if (p->full_layers > 0 && p->max_tokens <= p->R) return false;
     const long long units = (long long)p->layers * p->batch * p->n_kv_heads;
@@ -100,6 +103,8 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     s->cap = p->C + p->R + (s->T > 1 ? s->T : 0);
     s->es = p->dtype == MKV_DTYPE_F32 ? 4 : 2;
     s->nc = 1;
+    s->stored = p->profile_mode == MKV_PROFILE_STORED ? 1 : 0;
+    if (s->stored && (s->T > 1 || p->norm_mode != MKV_NORM_FROZEN || p->kernel == MKV_KERNEL_SIMT)) return false;
     if (s->T > 64) return false;
     if (p->norm_mode == MKV_NORM_CURRENT && s->T > 1) return false;     // the compaction drops several tokens at once
     const int nc = tc_ring_chunks(s->G, s->R);
@@ -123,6 +128,7 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
         s->splits = sp_all > sp_layer ? sp_all : sp_layer;
         return true;
     }
+    if (s->stored) return false;        // the profile table is kept by the tensor-core kernel's epilogue only
     *kind = kKindSimt;
     const int max_splits = (s->cap + 31) / 32;
     int sp = p->splits > 0 ? p->splits : simt_default_splits(s->U, s->cap);
@@ -178,7 +184,8 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
     a.ring_q = b + c->L.ring_q; a.ring_c = (float *)(b + c->L.ring_c);
     a.q = q; a.k_new = k; a.v_new = v; a.out = out;
     a.s_new = (float *)(b + c->L.s_new); a.F = (float *)(b + c->L.F);
-    a.Fc = c->s.nc > 1 ? (float *)(b + c->L.Fc) : nullptr; a.nc = c->s.nc;
+    a.Fc = c->s.nc > 1 && !c->s.stored ? (float *)(b + c->L.Fc) : nullptr; a.nc = c->s.nc;
+    a.prof = c->s.stored ? (float *)(b + c->L.prof) : nullptr;
     a.part_ml = (float *)(b + c->L.part_ml); a.part_o = (float *)(b + c->L.part_o);
     a.ticket = (int *)(b + c->L.ticket); a.evicted_pos = (int *)(b + c->L.evicted);
     a.st = (DevState *)(b + c->L.state);
@@ -200,6 +207,8 @@ DecodeArgs make_args(const mkv_ctx *c, const void *q, const void *k, const void 
 bool clear_arena(mkv_ctx *c, cudaStream_t stream)
 {
     const size_t kv = (size_t)c->s.U * c->s.cap * c->s.D * c->s.es, rq = (size_t)c->s.U * c->s.R * c->s.G * c->s.D * c->s.es;
+    if (c->s.stored &&
+        cudaMemsetAsync(c->base + c->L.prof, 0, (size_t)c->s.U * c->s.R * c->s.cap * 4, stream) != cudaSuccess) return false;
     return cudaMemsetAsync(c->base + c->L.K, 0, kv, stream) == cudaSuccess &&
            cudaMemsetAsync(c->base + c->L.V, 0, kv, stream) == cudaSuccess &&
            cudaMemsetAsync(c->base + c->L.ring_q, 0, rq, stream) == cudaSuccess;
@@ -218,6 +227,7 @@ DecodeArgs make_args_layer(const mkv_ctx *c, int layer, const void *q, const voi
     a.ring_q = (char *)a.ring_q + u0 * s.R * s.G * s.D * s.es; a.ring_c += u0 * s.R * s.G;
     a.s_new += u0 * s.G * s.cap; a.F += u0 * s.cap;
     if (a.Fc) a.Fc += u0 * s.nc * s.cap;
+    if (a.prof) a.prof += u0 * s.R * s.cap;
     a.part_ml += u0 * s.splits * s.G * 2; a.part_o += u0 * s.splits * s.G * s.D;
     a.ticket += u0; a.evicted_pos += u0;
     a.st = a.st + 1 + layer;
@@ -250,6 +260,13 @@ mkv_status launch_step(mkv_ctx *ctx, int layer, const void *q, const void *k, co
     const mkv_status ls = level_states(ctx, layer < 0 ? 1 : 2, stream);
     if (ls != MKV_OK) return ls;
     const DecodeArgs a = layer < 0 ? make_args(ctx, q, k, v, out) : make_args_layer(ctx, layer, q, k, v, out);
+    // stored-profile mode: a policy step reads its fused scores from the table first (the kernel checks the device
+    // state itself and does nothing on other steps)
+    if (ctx->s.stored && step_scores(ctx->t, ctx->n, ctx->steps, ctx->s.R, ctx->s.C, ctx->s.T)) {
+        const cudaError_t ef = launch_profile_fuse(a, stream);
+        if (ef != cudaSuccess) return fail(ctx, MKV_CUDA, "profile launch failed: %s", cudaGetErrorString(ef));
+        ctx->launches += 1;
+    }
     const cudaError_t e = ctx->kind == kKindTc ? launch_decode_tc(layer < 0 ? ctx->plan : ctx->plan_layer, a, stream)
                                                : launch_decode_simt(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "decode launch failed: %s", cudaGetErrorString(e));
@@ -377,6 +394,12 @@ mkv_status core_prefill(mkv_ctx *ctx, const void *k, const void *v, const void *
     if (e == cudaErrorLaunchTimeout) { cudaGetLastError(); return fail(ctx, MKV_DEVICE_TIMEOUT, "%s: a device-side wait of the prompt phase ran out", where); }
     if (e != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase: %s", cudaGetErrorString(e));
     ctx->n = (prompt_len - Rw > ctx->s.C) ? ctx->s.C + Rw : prompt_len;
+    if (ctx->s.stored) {        // the window rows' profiles over the kept tokens
+        cudaError_t ep = launch_prefill_profile(a, ctx->n, prompt_len, stream);
+        if (ep == cudaSuccess) ep = cudaStreamSynchronize(stream);
+        if (ep != cudaSuccess) return fail(ctx, MKV_CUDA, "prompt phase (profile table): %s", cudaGetErrorString(ep));
+        ctx->launches += 1;
+    }
     ctx->t = prompt_len;
     ctx->steps = 0;
     ctx->next_layer = 0;
@@ -393,6 +416,7 @@ mkv_status core_prefill_ragged(mkv_ctx *ctx, const void *k, const void *v, const
     const Shape &s = ctx->s;
     if (ctx->prefilled) return fail(ctx, MKV_BAD_STATE, "mkv_prefill_ragged: context already holds a sequence%s");
     if (s.T > 1) return fail(ctx, MKV_UNSUPPORTED, "mkv_prefill_ragged: not available with coarse-grained eviction%s");
+    if (s.stored) return fail(ctx, MKV_UNSUPPORTED, "mkv_prefill_ragged: not available with the stored attention profile%s");
     if (s.nc > 1) return fail(ctx, MKV_UNSUPPORTED, "mkv_prefill_ragged: not available with a window of more than 256 ring rows on the tensor-core kernel; create the context with the CUDA-core kernel%s");
     int longest = 0;
     for (int b = 0; b < s.B; ++b) longest = std::max(longest, (int)prompt_len[b]);
@@ -539,6 +563,7 @@ static mkv_params full_layer_params(const mkv_params *p)
     c.max_tokens = 0;
     c.C = p->max_tokens - p->R;
     c.evict_interval = 1;
+    c.profile_mode = MKV_PROFILE_RECOMPUTE;      // those layers keep everything: there is no score to take
     c.workspace = nullptr;
     c.workspace_bytes = 0;
     return c;

@@ -62,6 +62,10 @@ struct DecodeArgs {
     int *row_n;                // [2][B]
     const int *row_shift;      // [B]
     int B, Hkv;                // unit u (of this launch) belongs to batch row (u / Hkv) % B
+    float *prof;               // [U][R][cap]  stored-profile mode (nullptr otherwise): prof[r][k] is the weight, summed
+                               // over the group, that the window token of ring slot r gave to the token in cache slot
+                               // k when it was generated (the attention profile the paper's implementation stores
+                               // beside the KV cache); the fused scores are then read from this table, not recomputed
     int n_hint;                // the host's view of st->n when the launch was enqueued (0: none).  Only used to
                                // prefetch: a stale value (steps replayed from a CUDA graph) costs time, not results
 };
@@ -306,6 +310,16 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     int *pos = a.pos + (size_t)u * a.cap;
     float *F = a.F + (size_t)u * a.cap;
     int e_slot = n, e_pos = -1;
+    // stored-profile mode: the new token's row of the table is written on every step, policy or not
+    float *prof_row = a.prof ? a.prof + ((size_t)u * a.R + (int)(t % a.R)) * a.cap : nullptr;
+    if (prof_row != nullptr && !evict) {
+        const float *sn = a.s_new + (size_t)u * G * a.cap;
+        for (int k = tid; k < n; k += nthr) {
+            float s = 0.f;
+            for (int g = 0; g < G; ++g) s += exp2f(__ldcg(sn + (size_t)g * a.cap + k) - cnew[g]);
+            prof_row[k] = s;
+        }
+    }
     if (evict) {
         const float *sn = a.s_new + (size_t)u * G * a.cap;
         const long long thr = t - shift - a.R;        // positions are the row's own; ring slots follow t
@@ -340,6 +354,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
             for (int b = 0; b < 4; ++b) {
                 const int k = kb + b * nthr;
                 if (k >= n) continue;
+                if (prof_row != nullptr) prof_row[k] = s[b];
                 if ((long long)p[b] <= thr) {
                     const float f = fuse(a.fusion, f0[b], s[b]);
                     F[k] = f;
@@ -395,6 +410,13 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     T *rq = static_cast<T *>(a.ring_q) + ((size_t)u * a.R + rs) * G * D;
     for (int i = tid; i < G * D; i += nthr) stf(rq + i, i < Gq * D ? ldf(q + i) : 0.f);
     if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
+    if (a.prof != nullptr) {
+        // the slot the new token takes: no older window token ever attended to it; the new token's weight on itself
+        float self_w = 0.f;
+        for (int g = 0; g < G; ++g) self_w += exp2f(s_self[g] - cnew[g]);
+        float *col = a.prof + (size_t)u * a.R * a.cap + e_slot;
+        for (int r = tid; r < a.R; r += nthr) col[(size_t)r * a.cap] = r == rs ? self_w : 0.f;
+    }
     if (tid == 0) {
         pos[e_slot] = (int)(t - shift);
         a.evicted_pos[u] = e_pos;

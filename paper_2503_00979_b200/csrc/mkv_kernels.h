@@ -67,6 +67,12 @@ size_t prefill_static_max_floats();
 cudaError_t run_prefill_static(const DecodeArgs &a, bool f32, int D, const void *k, const void *v, const void *q_window,
                                int P, cudaStream_t stream, unsigned long long *launches, int device, int n_states);
 
+// Stored-profile mode (bf16, head_dim 128, tensor-core kernel): the fused scores of a policy step from the profile
+// table into a.F (a no-op on other steps; launched in front of the decode kernel), and the table after the prompt
+// phase (the arena's ring, K rows and positions must be in place; the table must have been cleared).
+cudaError_t launch_profile_fuse(const DecodeArgs &a, cudaStream_t stream);
+cudaError_t launch_prefill_profile(const DecodeArgs &a, int n, long long P, cudaStream_t stream);
+
 // Copies one step state over n_dst others (the whole-stack state and the per-layer states are brought level when
 // a context switches between whole-stack and per-layer calls).
 cudaError_t launch_copy_state(DevState *dst, int n_dst, const DevState *src, cudaStream_t stream, int *rows_dst = nullptr,

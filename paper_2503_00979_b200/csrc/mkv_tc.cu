@@ -385,7 +385,11 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
     // chunk that holds the slot of the new query (the main chunk) does everything a unit does otherwise; the
     // other chunks only score their rows against the unit's keys, into their own slab of a.Fc.  On a step that
     // does not run the policy only the main chunks are walked.
-    const int NCe = MC ? (evict ? geo.nc : 1) : 1;               // chunks walked per unit on this step
+    // Stored-profile mode (a.prof, served by this instantiation whatever the window's size): the fused scores of the
+    // window rows come from the table (written into a.F by a launch before this one), so no chunk is scored here and
+    // only the main chunk, which attends, is walked; the unit's epilogue keeps the table up to date.
+    const bool stored = MC && a.prof != nullptr;
+    const int NCe = MC ? ((evict && !stored) ? geo.nc : 1) : 1;  // chunks walked per unit on this step
     const int c_main = MC ? rs_new / (RGP / G) : 0;
     const int rs_loc = MC ? rs_new - c_main * (RGP / G) : rs_new;  // the new query's slot inside its chunk
     // Every thread of this CTA holds its copy of the step state (the barrier above orders their reads
@@ -651,7 +655,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 for (int g = 0; g < G; ++g) {
                     const float s2 = valid ? __uint_as_float(sv[g]) * a.scale2 : -INFINITY;
                     st_w[g * 32 + lane] = s2;
-                    if (valid && us.evict) s_new[(size_t)g * a.cap + key] = s2;
+                    if (valid && (us.evict || stored)) s_new[(size_t)g * a.cap + key] = s2;
                     const float mn = fmaxf(mrun[g], warp_max(s2));
                     // factor that brings what was accumulated under the old reference to the new one
                     const float f = mn == mrun[g] ? 1.f : ex2f(mrun[g] - mn);
@@ -732,7 +736,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                 // ---- fused scores of this warp's 32 keys over the ring rows (Eq. 4-6): only on steps that run the
                 // policy.  While the cache is still filling, and between two runs of a coarse-grained policy, nothing
                 // is evicted and the accumulator buffer goes back as soon as the new row's logits have been read.
-                if (us.evict) {
+                if (us.evict && !stored) {
                     float F = 0.f;
                     for (int c = 0; c < RGP; c += 32) {
                         uint32_t v[32];
@@ -853,7 +857,7 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                     }
                     group_sync(kEpiBar, kGroupThreads);
                     if (*flag) {
-                        if (us.evict) {
+                        if (us.evict && !stored) {
                             float *F = a.F + (size_t)u * a.cap;
                             const float *Fc = a.Fc + (size_t)u * geo.nc * a.cap;
                             for (int key = etid; key < us.n; key += kGroupThreads) {
@@ -954,7 +958,8 @@ cudaError_t launch_gfn(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 template <int G, int FUSION>
 cudaError_t launch_gf(TcPlan *plan, const DecodeArgs &a, cudaStream_t stream)
 {
-    if (plan->geo.nc > 1) return a.row_n ? cudaErrorInvalidValue : launch_gfn<G, FUSION, kComputeGroups, true, false>(plan, a, stream);
+    if (plan->geo.nc > 1 || a.prof)
+        return a.row_n ? cudaErrorInvalidValue : launch_gfn<G, FUSION, kComputeGroups, true, false>(plan, a, stream);
     return a.row_n ? launch_gfn<G, FUSION, kComputeGroups, false, true>(plan, a, stream)
                    : launch_gfn<G, FUSION, kComputeGroups, false, false>(plan, a, stream);
 }
@@ -1021,7 +1026,7 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned
     const int G = a.G;
     g.nc = a.nc;
     g.rgpad = g.nc > 1 ? chunk_rows(a.Gq, a.R) : pad32(a.R * G);
-    if (g.nc != tc_ring_chunks(a.Gq, a.R) || g.rgpad > 256 || g.rgpad * g.nc < a.R * G || (g.nc > 1 && !a.Fc)) {
+    if (g.nc != tc_ring_chunks(a.Gq, a.R) || g.rgpad > 256 || g.rgpad * g.nc < a.R * G || (g.nc > 1 && !a.Fc && !a.prof)) {
         snprintf(err, err_len, "tensor-core kernel: ring chunk geometry does not match the shape");
         delete p;
         return cudaErrorInvalidValue;
@@ -1050,7 +1055,7 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned
         return cudaErrorInvalidConfiguration;
     }
     g.sk = total_stages >= 7 ? 3 : total_stages >= 5 ? 2 : 1;
-    if (g.nc > 1 && total_stages >= 4) g.sk = 2;      // most items of a chunked window read K only
+    if (g.nc > 1 && !a.prof && total_stages >= 4) g.sk = 2;      // most items of a chunked window read K only
     g.sv = total_stages - g.sk;
     g.smem_bytes = tc_smem_layout(g, G).total + 1024;
     if (!encode_map(&p->tmK, a.K, a.U, a.cap, kTile) || !encode_map(&p->tmV, a.V, a.U, a.cap, kTile) ||

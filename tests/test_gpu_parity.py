@@ -822,3 +822,28 @@ def test_ragged_prompts_degenerate_cases(lens):
     rep = run_parity_ragged(w, lens, steps=w.steps, kernel="auto")
     _report(rep)
     assert rep.kernel == "tc" and rep.evictions > 0
+
+
+# ---- the attention profiles kept as a table beside the cache (the paper's own bookkeeping) instead of recomputed
+@pytest.mark.parametrize("q_heads,kv_heads,R,C,P,fusion", [(8, 2, 16, 150, 260, "sum"),      # evicts from the first step
+                                                           (8, 2, 32, 230, 200, "max"),      # starts in the fill phase
+                                                           (14, 2, 12, 90, 133, "sum"),      # group 7 -> 8
+                                                           (8, 2, 200, 600, 1000, "sum"),    # window 200: 800 ring rows
+                                                           (2, 2, 9, 40, 5, "max")])         # prompt shorter than the window
+def test_stored_profile_mode(q_heads, kv_heads, R, C, P, fusion):
+    w = synth.Workload("stored", 2, 2, q_heads, kv_heads, 128, "bf16", P, 2 * R + 40, C, R, fusion, 900 + R)
+    rep = run_parity(w, steps=w.steps, n_units=8, kernel="auto", check_F_every=5, profile="stored")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+
+
+def test_stored_profile_mode_with_per_layer_calls_and_reset():
+    w = synth.Workload("stored_layer", 3, 1, 8, 2, 128, "bf16", 300, 40, 200, 24, "sum", 951)
+    rep = run_parity(w, steps=w.steps, n_units=6, kernel="auto", per_layer=2, profile="stored")
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions > 0
+    p = binding.mkv_default_params()
+    p.layers, p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.C, p.R = 1, 1, 8, 2, 64, 64, 16       # head_dim 64: CUDA-core kernel only
+    p.profile_mode = binding.PROFILE["stored"]
+    st, h = binding.mkv_create_ex(p)
+    assert st == binding.UNSUPPORTED and h is None
