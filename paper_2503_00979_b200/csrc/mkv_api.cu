@@ -107,8 +107,9 @@ bool resolve(const mkv_params *p, Shape *s, KernelKind *kind)
     if (s->stored && (s->T > 1 || p->norm_mode != MKV_NORM_FROZEN || p->kernel == MKV_KERNEL_SIMT)) return false;
     if (s->T > 64) return false;
     if (p->norm_mode == MKV_NORM_CURRENT && s->T > 1) return false;     // the compaction drops several tokens at once
-    const int nc = tc_ring_chunks(s->G, s->R);
-    const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->R) &&
+    // stored-profile mode: the decode kernel only ever needs the ring rows of the new query, whatever the window's size
+    const int nc = s->stored ? 1 : tc_ring_chunks(s->G, s->R);
+    const bool tc_ok = tc_shape_supported(p->dtype == MKV_DTYPE_F32, s->D, s->G, s->stored ? 1 : s->R) &&
                        (long long)s->U * nc * ((s->cap + 127) / 128) <= (1ll << 30);     // tile indices stay 32-bit
     if (p->kernel == MKV_KERNEL_TC && !tc_ok) return false;
     if (tc_ok && p->kernel != MKV_KERNEL_SIMT) {

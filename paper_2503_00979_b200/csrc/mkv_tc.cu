@@ -1026,7 +1026,11 @@ cudaError_t tc_plan_create(TcPlan **out, const DecodeArgs &a, int grid, unsigned
     const int G = a.G;
     g.nc = a.nc;
     g.rgpad = g.nc > 1 ? chunk_rows(a.Gq, a.R) : pad32(a.R * G);
-    if (g.nc != tc_ring_chunks(a.Gq, a.R) || g.rgpad > 256 || g.rgpad * g.nc < a.R * G || (g.nc > 1 && !a.Fc && !a.prof)) {
+    // stored-profile mode: nothing is scored, so the operand is the 32-row piece of the ring that holds the new
+    // query's slot (the kernel's chunk arithmetic with 32-row chunks, of which only that one is ever walked)
+    if (a.prof) g.rgpad = 32;
+    if (!a.prof &&
+        (g.nc != tc_ring_chunks(a.Gq, a.R) || g.rgpad > 256 || g.rgpad * g.nc < a.R * G || (g.nc > 1 && !a.Fc))) {
         snprintf(err, err_len, "tensor-core kernel: ring chunk geometry does not match the shape");
         delete p;
         return cudaErrorInvalidValue;

@@ -829,7 +829,8 @@ def test_ragged_prompts_degenerate_cases(lens):
                                                            (8, 2, 32, 230, 200, "max"),      # starts in the fill phase
                                                            (14, 2, 12, 90, 133, "sum"),      # group 7 -> 8
                                                            (8, 2, 200, 600, 1000, "sum"),    # window 200: 800 ring rows
-                                                           (2, 2, 9, 40, 5, "max")])         # prompt shorter than the window
+                                                           (2, 2, 9, 40, 5, "max"),          # prompt shorter than the window
+                                                           (8, 2, 700, 900, 1200, "sum")])   # window 700: beyond what recomputation takes
 def test_stored_profile_mode(q_heads, kv_heads, R, C, P, fusion):
     w = synth.Workload("stored", 2, 2, q_heads, kv_heads, 128, "bf16", P, 2 * R + 40, C, R, fusion, 900 + R)
     rep = run_parity(w, steps=w.steps, n_units=8, kernel="auto", check_F_every=5, profile="stored")
