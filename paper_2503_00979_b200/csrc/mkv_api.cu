@@ -261,9 +261,10 @@ mkv_status launch_step(mkv_ctx *ctx, int layer, const void *q, const void *k, co
     const mkv_status ls = level_states(ctx, layer < 0 ? 1 : 2, stream);
     if (ls != MKV_OK) return ls;
     const DecodeArgs a = layer < 0 ? make_args(ctx, q, k, v, out) : make_args_layer(ctx, layer, q, k, v, out);
-    // stored-profile mode: a policy step reads its fused scores from the table first (the kernel checks the device
-    // state itself and does nothing on other steps)
-    if (ctx->s.stored && step_scores(ctx->t, ctx->n, ctx->steps, ctx->s.R, ctx->s.C, ctx->s.T)) {
+    // stored-profile mode: a policy step reads its fused scores from the table first.  Launched on every step: the
+    // kernel decides by the device's step state and returns at once when no policy runs, so that a recorded
+    // sequence of steps stays valid when it is replayed into another phase of the sequence.
+    if (ctx->s.stored) {
         const cudaError_t ef = launch_profile_fuse(a, stream);
         if (ef != cudaSuccess) return fail(ctx, MKV_CUDA, "profile launch failed: %s", cudaGetErrorString(ef));
         ctx->launches += 1;
