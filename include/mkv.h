@@ -50,9 +50,8 @@ typedef enum mkv_status {
 
 typedef enum mkv_fusion { MKV_FUSION_SUM = 0, MKV_FUSION_MAX = 1 } mkv_fusion;   /* Eq. 5, Eq. 6 */
 typedef enum mkv_dtype { MKV_DTYPE_BF16 = 0, MKV_DTYPE_F32 = 1 } mkv_dtype;
-/* which decode kernel to use: AUTO picks the tensor-core kernel when the shape allows it */
-/* How a window row's attention weights enter the fused score (Eq. 4).  FROZEN: as the row assigned them when its
- * token was generated ("the attention weight that w_r assigned").  CURRENT: renormalised over the tokens that are
+/* How a window row's attention weights enter the fused score (Eq. 4).  FROZEN: with the values they had when the
+ * row's token was generated.  CURRENT: renormalised over the tokens that are
  * still cached when the scores are taken (a row never saw tokens newer than itself); not with evict_interval > 1. */
 typedef enum mkv_norm { MKV_NORM_FROZEN = 0, MKV_NORM_CURRENT = 1 } mkv_norm;
 /* where the window tokens' attention profiles come from when the fused scores are taken (Eq. 4-6):
@@ -63,6 +62,9 @@ typedef enum mkv_norm { MKV_NORM_FROZEN = 0, MKV_NORM_CURRENT = 1 } mkv_norm;
  *   for arithmetic; it pays for wide windows.  bf16 / head_dim 128 on the tensor-core kernel only, with per-step
  *   eviction and MKV_NORM_FROZEN; not with mkv_prefill_ragged. */
 typedef enum mkv_profile { MKV_PROFILE_RECOMPUTE = 0, MKV_PROFILE_STORED = 1 } mkv_profile;
+/* which decode kernel to use: AUTO picks the tensor-core kernel when the shape allows it (bf16, head_dim 128, a
+ * window of at most 2048 ring rows R * G', G' the GQA ratio rounded up to a power of two; any window with
+ * MKV_PROFILE_STORED), the CUDA-core kernel otherwise */
 typedef enum mkv_kernel { MKV_KERNEL_AUTO = 0, MKV_KERNEL_SIMT = 1, MKV_KERNEL_TC = 2 } mkv_kernel;
 
 typedef struct mkv_ctx mkv_ctx;
