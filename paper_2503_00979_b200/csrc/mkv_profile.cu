@@ -27,12 +27,12 @@ __global__ void __launch_bounds__(kFT) profile_fuse_kernel(DecodeArgs a)
     const float *p = a.prof + (size_t)u * a.R * a.cap + k;
     float F = 0.f;
     int r = 0;
-    for (; r + 4 <= a.R; r += 4) {          // four rows in flight
-        float w[4];
+    for (; r + 8 <= a.R; r += 8) {          // eight rows in flight
+        float w[8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) w[i] = r + i == rs ? 0.f : __ldcs(p + (size_t)(r + i) * a.cap);
+        for (int i = 0; i < 8; ++i) w[i] = __ldcs(p + (size_t)(r + i) * a.cap);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) F = fuse(a.fusion, F, w[i]);
+        for (int i = 0; i < 8; ++i) F = fuse(a.fusion, F, r + i == rs ? 0.f : w[i]);
     }
     for (; r < a.R; ++r) F = fuse(a.fusion, F, r == rs ? 0.f : __ldcs(p + (size_t)r * a.cap));
     a.F[(size_t)u * a.cap + k] = F;
