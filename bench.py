@@ -47,7 +47,7 @@ NOMINAL_HBM_GBS = 7700.0
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from one ncu
 # capture of a launch of that workload), valid only for the kernel sources it was taken with.
-_TRAFFIC = {"c1": {"bytes": 284.1e6, "sources_sha256": "17674191a2b155fdd107782d84a585c031b50a3ee0ce5982b608d4e675924e51"}}
+_TRAFFIC = {"c1": {"bytes": 284.9e6, "sources_sha256": "5687faec5ff06122cd7ad7a0975de33c1dc8eefe2ac91bbdd3f1f3cf9f928e57"}}
 
 
 def measured_traffic(workload: str):

@@ -233,7 +233,8 @@ __device__ void renormalise_after_eviction(const DecodeArgs &a, int u, int e_slo
 // group size when known at compile time (0: use a.G); it lets the loads of a round be
 // issued together.  Loads are batched so that the whole epilogue costs a handful of L2
 // round trips.
-template <typename T, int D, int GT>
+// PROF: the caller may be serving the stored-profile mode (a.prof); compiled out otherwise.
+template <typename T, int D, int GT, bool PROF = false>
 __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, int active, bool evict, float *sm,
                               int tid, int nthr, int bar_id, int shift = 0)
 {
@@ -311,8 +312,9 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     float *F = a.F + (size_t)u * a.cap;
     int e_slot = n, e_pos = -1;
     // stored-profile mode: the new token's row of the table is written on every step, policy or not
-    float *prof_row = a.prof ? a.prof + ((size_t)u * a.R + (int)(t % a.R)) * a.cap : nullptr;
-    if (prof_row != nullptr && !evict) {
+    float *prof_row = nullptr;
+    if constexpr (PROF) prof_row = a.prof ? a.prof + ((size_t)u * a.R + (int)(t % a.R)) * a.cap : nullptr;
+    if (PROF && prof_row != nullptr && !evict) {
         const float *sn = a.s_new + (size_t)u * G * a.cap;
         for (int k = tid; k < n; k += nthr) {
             float s = 0.f;
@@ -354,7 +356,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
             for (int b = 0; b < 4; ++b) {
                 const int k = kb + b * nthr;
                 if (k >= n) continue;
-                if (prof_row != nullptr) prof_row[k] = s[b];
+                if (PROF && prof_row != nullptr) prof_row[k] = s[b];
                 if ((long long)p[b] <= thr) {
                     const float f = fuse(a.fusion, f0[b], s[b]);
                     F[k] = f;
@@ -410,7 +412,7 @@ __device__ void finalize_unit(const DecodeArgs &a, int u, long long t, int n, in
     T *rq = static_cast<T *>(a.ring_q) + ((size_t)u * a.R + rs) * G * D;
     for (int i = tid; i < G * D; i += nthr) stf(rq + i, i < Gq * D ? ldf(q + i) : 0.f);
     if (tid < G) a.ring_c[((size_t)u * a.R + rs) * G + tid] = cnew[tid];
-    if (a.prof != nullptr) {
+    if (PROF && a.prof != nullptr) {
         // the slot the new token takes: no older window token ever attended to it; the new token's weight on itself
         float self_w = 0.f;
         for (int g = 0; g < G; ++g) self_w += exp2f(s_self[g] - cnew[g]);

@@ -869,8 +869,8 @@ decode_tc_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ C
                         }
                         int idx;
                         const int ncta_main = w.ctas_of_unit(u * NCe + (NCe == 1 ? 0 : c_main), idx);
-                        finalize_unit<__nv_bfloat16, kD, G>(a, u, t, us.n, ncta_main, us.evict, fin_sm, etid, kGroupThreads, kEpiBar,
-                                                            RAGGED ? us.shift : 0);
+                        finalize_unit<__nv_bfloat16, kD, G, true>(a, u, t, us.n, ncta_main, us.evict, fin_sm, etid, kGroupThreads,
+                                                                  kEpiBar, RAGGED ? us.shift : 0);
                     }
                 } else if (ncta == 1) {
                     finalize_fast<G, true>(a, u, t, us.n, 1, us.evict, fin_sm, etid, kEpiBar, o, cml, RAGGED ? us.shift : 0);
