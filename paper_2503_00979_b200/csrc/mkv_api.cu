@@ -276,7 +276,15 @@ mkv_status launch_step(mkv_ctx *ctx, int layer, const void *q, const void *k, co
     const bool ev = step_scores(ctx->t, ctx->n, ctx->steps, ctx->s.R, ctx->s.C, ctx->s.T);
     // coarse-grained eviction: the compaction follows the steps that ran the policy (the kernel itself checks the
     // device state and does nothing if no compaction is pending)
-    if (ctx->s.T > 1 && ev) {
+    // (While the stream is being captured the launch is recorded after every step, so that the recorded sequence
+    // stays valid when it is replayed in another phase of the eviction period.)
+    bool capturing = false;
+    if (ctx->s.T > 1 && !ev) {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        capturing = cudaStreamIsCapturing(stream, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusActive;
+        cudaGetLastError();
+    }
+    if (ctx->s.T > 1 && (ev || capturing)) {
         const cudaError_t e2 = launch_compact(a, ctx->p.dtype == MKV_DTYPE_F32, ctx->s.D, stream);
         if (e2 != cudaSuccess) return fail(ctx, MKV_CUDA, "compaction launch failed: %s", cudaGetErrorString(e2));
         ctx->launches += 1;

@@ -716,9 +716,9 @@ def test_ragged_prefill_rejects_what_it_does_not_support():
 
 
 # ---- the step index lives on the device: steps recorded in a CUDA graph and replayed
-@pytest.mark.parametrize("kernel,dtype,d,profile", [("tc", "bf16", 128, "recompute"), ("simt", "f32", 64, "recompute"),
-                                                    ("tc", "bf16", 128, "stored")])
-def test_steps_replayed_from_a_cuda_graph_equal_direct_calls(kernel, dtype, d, profile):
+@pytest.mark.parametrize("kernel,dtype,d,profile,T", [("tc", "bf16", 128, "recompute", 1), ("simt", "f32", 64, "recompute", 1),
+                                                      ("tc", "bf16", 128, "stored", 1), ("tc", "bf16", 128, "recompute", 3)])
+def test_steps_replayed_from_a_cuda_graph_equal_direct_calls(kernel, dtype, d, profile, T):
     # Four steps are captured once (launches only, on a side stream) and replayed three times with fresh inputs in
     # the same buffers; a second context takes the same twelve steps by direct calls.  Outputs bit for bit, the
     # same retained positions, and the host mirror follows the device state after mkv_sync.  The cache fills
@@ -737,8 +737,9 @@ def test_steps_replayed_from_a_cuda_graph_equal_direct_calls(kernel, dtype, d, p
     vs = vv.permute(3, 0, 1, 2, 4).to(tdt).contiguous()
 
     def fresh():
+        # (T = 3 against four recorded steps: every replay meets the eviction period in another phase)
         mk = binding.MorphKV(w.layers, w.batch, w.n_q_heads, w.n_kv_heads, d, w.C, w.R, w.fusion, dtype, kernel=kernel,
-                             profile=profile)
+                             profile=profile, evict_interval=T)
         mk.prefill(k.to(tdt).contiguous(), v.to(tdt).contiguous(), qw.to(tdt).contiguous())
         mk.sync()
         return mk
