@@ -55,7 +55,7 @@ cudaError_t launch_set_state(DevState *st, int n_states, long long t, int n, cud
 // Tensor-core scoring of the prompt phase (mkv_prefill_tc.cu): two passes over the prompt keys, window-row
 // normalisers into ring_c and fused scores of the older tokens into Fp [nb][P].
 bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P);
-int prefill_tc_splits(int units_in_batch, int P);
+int prefill_tc_splits(int units_in_batch, int P, int window_rows);
 size_t prefill_tc_floats_per_unit(int P, int Rw, int G, int splits);
 cudaError_t run_prefill_scores_tc(const DecodeArgs &a, const void *k, const void *qwin, int P, int ub0, int nb, int splits,
                                   float *Fp, float *part, int *err, unsigned long long *launches, cudaStream_t stream);

@@ -187,26 +187,54 @@ __global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__rest
     int *upos = pos + (size_t)u * cap;
     unsigned long long prefix = 0;
     int remaining = C;
+    static_assert(kPT == 256, "one thread per bucket");
+    constexpr int kSelBatch = 8;                                         // keys per thread in flight
     for (int pass = 7; pass >= 0; --pass) {
-        for (int i = tid; i < 256; i += kPT) hist[i] = 0;
+        hist[tid] = 0;
         __syncthreads();
         const int shift = 8 * pass;
-        for (int j = tid; j < M; j += kPT) {
-            const unsigned long long key = rank_key(__float_as_uint(F[j]), j);
-            if (pass == 7 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
+        for (int c0 = 0; c0 < M; c0 += kPT * kSelBatch) {
+            // the loads of a batch are issued together: a pass is a chain of L2 round trips otherwise
+            unsigned int fb[kSelBatch];
+#pragma unroll
+            for (int i = 0; i < kSelBatch; ++i) {
+                const int j = c0 + i * kPT + tid;
+                fb[i] = j < M ? __float_as_uint(F[j]) : 0u;
+            }
+#pragma unroll
+            for (int i = 0; i < kSelBatch; ++i) {
+                const int j = c0 + i * kPT + tid;
+                unsigned int bin = 256u;                                 // 256: not counted in this pass
+                if (j < M) {
+                    const unsigned long long key = rank_key(fb[i], j);
+                    if (pass == 7 || (key >> (shift + 8)) == prefix) bin = (unsigned)(key >> shift) & 255u;
+                }
+                // one shared-memory atomic per warp and distinct bucket: the high bytes of the keys (sign and
+                // exponent of the score) fall into a few buckets, and 32 atomics on one word would be serialised
+                const unsigned int peers = __match_any_sync(0xffffffffu, bin);
+                if (bin < 256u && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], (unsigned)__popc(peers));
+            }
         }
         __syncthreads();
-        if (tid == 0) {
-            int acc = 0, b = 255;
-            for (; b > 0; --b) {
-                if (acc + (int)hist[b] >= remaining) break;
-                acc += (int)hist[b];
-            }
-            const unsigned long long np = (prefix << 8) | (unsigned long long)b;
+        // the bucket b that holds the `remaining`-th best key: above(b) < remaining <= above(b) + hist[b], with
+        // above(b) the number of keys in higher buckets.  Thread b owns bucket b; exactly one thread qualifies.
+        const int h = (int)hist[tid];
+        int incl = h;                                                    // sum over this warp's buckets >= tid
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_down_sync(0xffffffffu, incl, o);
+            if (lane + o < 32) incl += up;
+        }
+        if (lane == 0) wtot[warp] = incl;
+        __syncthreads();
+        int above = incl - h;
+        for (int w = warp + 1; w < kPT / 32; ++w) above += wtot[w];
+        if (h > 0 && above < remaining && remaining <= above + h) {
+            const unsigned long long np = (prefix << 8) | (unsigned long long)tid;
             // the bucket fills the remaining places exactly: every key in it is kept, so the smallest key with
             // this prefix is the threshold and the finer passes (mostly tie-breaking position bits) are not needed
-            const bool exact = acc + (int)hist[b] == remaining;
-            remaining_s = remaining - acc;
+            const bool exact = above + h == remaining;
+            remaining_s = remaining - above;
             prefix_s = exact ? np << shift : np;
             done_s = exact ? 1 : 0;
         }
@@ -218,17 +246,27 @@ __global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__rest
         if (done) break;
     }
     int base = 0;
-    for (int c0 = 0; c0 < M; c0 += kPT) {
-        const int j = c0 + tid;
-        const bool keep = j < M && rank_key(__float_as_uint(F[j]), j) >= prefix;
-        const unsigned int bal = __ballot_sync(0xffffffffu, keep);
-        if (lane == 0) wtot[warp] = __popc(bal);
-        __syncthreads();
-        int off = base;
-        for (int w = 0; w < warp; ++w) off += wtot[w];
-        if (keep) upos[off + __popc(bal & ((1u << lane) - 1u))] = j;
-        for (int w = 0; w < kPT / 32; ++w) base += wtot[w];
-        __syncthreads();
+    for (int c0 = 0; c0 < M; c0 += kPT * kSelBatch) {
+        unsigned int fb[kSelBatch];
+#pragma unroll
+        for (int i = 0; i < kSelBatch; ++i) {
+            const int j = c0 + i * kPT + tid;
+            fb[i] = j < M ? __float_as_uint(F[j]) : 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < kSelBatch; ++i) {
+            const int j = c0 + i * kPT + tid;
+            if (c0 + i * kPT >= M) break;                                // uniform over the CTA
+            const bool keep = j < M && rank_key(fb[i], j) >= prefix;
+            const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) wtot[warp] = __popc(bal);
+            __syncthreads();
+            int off = base;
+            for (int w = 0; w < warp; ++w) off += wtot[w];
+            if (keep) upos[off + __popc(bal & ((1u << lane) - 1u))] = j;
+            for (int w = 0; w < kPT / 32; ++w) base += wtot[w];
+            __syncthreads();
+        }
     }
     for (int i = tid; i < Rw; i += kPT) upos[C + i] = M + i;
 }
@@ -364,7 +402,7 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
     // (the arena's group must be the padded one: a context that runs the CUDA-core decode kernel keeps G as it is)
     const bool tc = !row && prefill_tc_supported(sizeof(T) == 4, D, a.Gq, R, k, P) && tc_padded_group(a.Gq) == G;
     const int Rws = row ? row->qw_stride : Rw;
-    const int tc_splits = tc ? prefill_tc_splits(U, P) : 0;
+    const int tc_splits = tc ? prefill_tc_splits(U, P, Rw * G) : 0;
     const size_t per_unit = tc ? prefill_tc_floats_per_unit(P, Rw, G, tc_splits) : (size_t)rows * P + P;   // floats
     if (per_unit + 1 > scratch_floats) return cudaErrorInvalidConfiguration;
     size_t ub = (scratch_floats - 1) / per_unit;
@@ -488,7 +526,7 @@ cudaError_t run_prefill(const DecodeArgs &a, bool f32, int D, const void *k, con
 {
     const int Rw = P < a.R ? P : a.R;
     const bool tc = !row && prefill_tc_supported(f32, D, a.Gq, a.R, k, P) && tc_padded_group(a.Gq) == a.G;
-    const size_t per_unit = (tc ? prefill_tc_floats_per_unit(P, Rw, a.G, prefill_tc_splits(a.U, P))
+    const size_t per_unit = (tc ? prefill_tc_floats_per_unit(P, Rw, a.G, prefill_tc_splits(a.U, P, Rw * a.G))
                                 : (size_t)Rw * a.G * P + P) * sizeof(float);
     size_t ub = ((size_t)1 << 30) / per_unit;
     if (ub < 1) ub = 1;

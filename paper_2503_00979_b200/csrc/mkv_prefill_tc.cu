@@ -11,9 +11,11 @@
 //           every thread owns one key, turns its row of logits into weights exp2(s - c_row), sums them over the
 //           group and fuses them over the window; F[k] is written for the candidates (P floats per unit).
 // The selection (radix top-C on (F, position) keys), the gather of the kept rows and the ring set-up stay the
-// kernels of mkv_prefill.cu.  CTA layout: warps 0-3 consume (one TMEM lane quarter each), warp 4 feeds K tiles
-// with TMA into a ring of 32 KB stages, warp 5 issues the MMAs into two TMEM accumulator buffers.  Every wait is
-// bounded; a wait that runs out raises an error word that the host reads after the call.
+// kernels of mkv_prefill.cu.  CTA layout: warps 0-3 and 6-9 are two consumer groups (one TMEM lane quarter per
+// warp); tiles alternate between the groups, so group g always reads accumulator buffer g and keeps its own
+// running (max, sum) per row in pass 1.  Warp 4 feeds K tiles with TMA into a ring of 32 KB stages, warp 5 issues
+// the MMAs into the two TMEM accumulator buffers.  Every wait is bounded; a wait that runs out raises an error
+// word that the host reads after the call.
 #include <stdio.h>
 
 #include "mkv_common.cuh"
@@ -25,12 +27,13 @@ namespace mkv {
 namespace {
 
 constexpr int kPfMaxStages = 3;
-constexpr int kPfThreads = 192;
+constexpr int kPfThreads = 320;
+constexpr int kPfGroups = 2;                 // consumer groups = accumulator buffers
 enum PfWait { kPfKEmpty = 21, kPfKFull, kPfTEmpty, kPfTFull, kPfDrain };
 
 struct PfArgs {
     const __nv_bfloat16 *qwin;   // [U][G][Rw][128]: the window queries of unit u are heads u*G .. u*G+G-1
-    float *part_ml;              // [nb][splits][qrows][2] pass-1 partial (max, sum) per window row, log2 domain
+    float *part_ml;              // [nb][splits * kPfGroups][qrows][2] pass-1 partial (max, sum) per window row, log2 domain
     float *ring_c;               // [U][R][G] arena: normaliser of the row of position p in ring slot p % R
     float *Fp;                   // [nb][P] fused scores of the batch's units
     int *err;                    // error word (0 = none)
@@ -102,11 +105,12 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
         for (int row = tid; row < 256; row += kPfThreads) {
             float nc = -INFINITY;                               // padding rows give weight 0
             if (row < a.rows) {
-                const float *pm = a.part_ml + (size_t)ul * a.splits * QR * 2;
+                const int np = a.splits * kPfGroups;
+                const float *pm = a.part_ml + (size_t)ul * np * QR * 2;
                 float m = -INFINITY;
-                for (int s = 0; s < a.splits; ++s) m = fmaxf(m, pm[((size_t)s * QR + row) * 2]);
+                for (int s = 0; s < np; ++s) m = fmaxf(m, pm[((size_t)s * QR + row) * 2]);
                 float l = 0.f;
-                for (int s = 0; s < a.splits; ++s) {
+                for (int s = 0; s < np; ++s) {
                     const float ms = pm[((size_t)s * QR + row) * 2];
                     if (ms > -INFINITY) l += pm[((size_t)s * QR + row) * 2 + 1] * exp2f(ms - m);
                 }
@@ -203,9 +207,11 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
             __syncwarp();
         }
     } else {
-        // ------------------------------------------------ consumers: one TMEM lane quarter per warp
-        const int lq = warp * 32 + lane;                     // lane of the accumulator this thread reads
-        const uint32_t tlane = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // ------------------------------------------------ consumers: one TMEM lane quarter per warp (a warp reads
+        // the quarter warp % 4), group 0 = warps 0-3 takes the even tiles, group 1 = warps 6-9 the odd ones
+        const int grp = warp < 4 ? 0 : 1;
+        const int lq = (warp & 3) * 32 + lane;               // lane of the accumulator this thread reads
+        const uint32_t tlane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
         if (PASS == 1) {
             // this thread's rows (one per block of 128) and the last key each may see
@@ -216,8 +222,8 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
                 const int row = rb * 128 + lq;
                 lim[rb] = (rb < RB && row < a.rows) ? a.P - a.Rw + row / G : -1;
             }
-            for (int j = 0; j < ntile && ok; ++j) {
-                const int b = j & 1;
+            for (int j = grp; j < ntile && ok; j += kPfGroups) {
+                const int b = grp;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * b, (uint32_t)((j >> 1) & 1), abort_flag, kPfTFull, WL));
                 if (!ok) break;
                 tc_fence_after();
@@ -252,15 +258,15 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
                 __syncwarp();
             }
             if (ok) {
-                float *pm = a.part_ml + ((size_t)ul * a.splits + sp) * QR * 2;
+                float *pm = a.part_ml + (((size_t)ul * a.splits + sp) * kPfGroups + grp) * QR * 2;
 #pragma unroll
                 for (int rb = 0; rb < 2; ++rb)
                     if (rb < RB) { pm[(rb * 128 + lq) * 2] = m[rb]; pm[(rb * 128 + lq) * 2 + 1] = l[rb]; }
             }
         } else {
             float *Fu = a.Fp + (size_t)ul * a.P;
-            for (int j = 0; j < ntile && ok; ++j) {
-                const int b = j & 1;
+            for (int j = grp; j < ntile && ok; j += kPfGroups) {
+                const int b = grp;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * b, (uint32_t)((j >> 1) & 1), abort_flag, kPfTFull, WL));
                 if (!ok) break;
                 tc_fence_after();
@@ -324,22 +330,32 @@ bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P)
     return tc_shape_supported(f32, D, G, R) && tc_ring_chunks(G, R) == 1 && ((uintptr_t)k & 15) == 0 && P >= 1;
 }
 
-int prefill_tc_splits(int units_in_batch, int P)
+int prefill_tc_splits(int units_in_batch, int P, int window_rows)
 {
+    // CTAs per unit along the keys.  A CTA pays a set-up (TMEM, barriers, the window queries into shared memory,
+    // in pass 2 the merge of the partial normalisers) worth about `kSetupTiles` key tiles, and the grid runs in
+    // waves of `slots` resident CTAs: take the split with the fewest tile-times over all waves.
+    constexpr int kSetupTiles = 3;
     const int nt = (P + kTile - 1) / kTile;
-    int s = (8 * 148 + units_in_batch - 1) / units_in_batch;       // about four waves of two CTAs per SM
-    if (s > nt) s = nt;
-    return s < 1 ? 1 : s;
+    const int slots = 148 * (window_rows <= 128 ? 2 : 1);
+    int best = 1;
+    long long best_cost = -1;
+    for (int s = 1; s <= nt && s <= 64; ++s) {
+        const long long waves = ((long long)units_in_batch * s + slots - 1) / slots;
+        const long long cost = waves * ((nt + s - 1) / s + kSetupTiles);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    return best;
 }
 
 size_t prefill_tc_floats_per_unit(int P, int Rw, int G, int splits)
 {
     const int qrows = ((Rw * G + 127) / 128) * 128;
-    return (size_t)P + (size_t)splits * qrows * 2;
+    return (size_t)P + (size_t)splits * kPfGroups * qrows * 2;
 }
 
 // Window-row normalisers into ring_c and fused scores of the prompt's older tokens into Fp [nb][P] for units
-// ub0 .. ub0+nb-1.  `part` holds nb * splits * qrows * 2 floats of scratch, `err` is a zeroed error word.
+// ub0 .. ub0+nb-1.  `part` holds nb * splits * kPfGroups * qrows * 2 floats of scratch, `err` is a zeroed error word.
 cudaError_t run_prefill_scores_tc(const DecodeArgs &a, const void *k, const void *qwin, int P, int ub0, int nb, int splits,
                                   float *Fp, float *part, int *err, unsigned long long *launches, cudaStream_t stream)
 {
