@@ -236,18 +236,26 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
                         tmem_ld32(tlane + (uint32_t)(b * bufcols + rb * 128 + c), v);
                         const int kc = key0 + c;
                         if (kc <= lim[rb]) {                 // else: nothing this row may see in these 32 keys
+                            if (kc + 31 > lim[rb]) {         // the row's causal limit falls inside the chunk
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (kc + i > lim[rb]) v[i] = 0xff800000u;        // -inf: weight 0
+                            }
+                            // the scale is positive, so the maximum is taken on the raw logits and scaled once;
+                            // one FFMA per key then forms s * scale - m
                             float cm = -INFINITY;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const float s2 = kc + i <= lim[rb] ? __uint_as_float(v[i]) * a.scale2 : -INFINITY;
-                                v[i] = __float_as_uint(s2);
-                                cm = fmaxf(cm, s2);
-                            }
+                            for (int i = 0; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(v[i]));
+                            cm *= a.scale2;
                             if (cm > m[rb]) { l[rb] *= ex2f(m[rb] - cm); m[rb] = cm; }
-                            float acc = 0.f;
+                            const float nm = -m[rb];
+                            float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) acc += ex2f(__uint_as_float(v[i]) - m[rb]);
-                            l[rb] += acc;
+                            for (int i = 0; i < 32; i += 2) {
+                                acc0 += ex2f(fmaf(__uint_as_float(v[i]), a.scale2, nm));
+                                acc1 += ex2f(fmaf(__uint_as_float(v[i + 1]), a.scale2, nm));
+                            }
+                            l[rb] += acc0 + acc1;
                         }
                         __syncwarp();                        // the lanes meet again in front of the aligned TMEM load
                     }
