@@ -174,36 +174,37 @@ __global__ void __launch_bounds__(kPT) prefill_fuse_kernel(const float *__restri
 // Top-C of the M = P - Rw older tokens by (F descending, position ascending): an 8-pass
 // radix select finds the C-th best 64-bit rank key, then an order-preserving compaction
 // lists the kept positions, followed by the window positions.
-__global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__restrict__ Fp, int *__restrict__ pos, int ub0,
-                                                             int P, int Rw, int C, int cap)
+constexpr int kSelT = 1024;  // threads of the selection kernel: a pass is a chain of rounds of kSelT keys
+__global__ void __launch_bounds__(kSelT) prefill_select_kernel(const float *__restrict__ Fp, int *__restrict__ pos, int ub0,
+                                                               int P, int Rw, int C, int cap)
 {
     __shared__ unsigned int hist[256];
     __shared__ unsigned long long prefix_s;
     __shared__ int remaining_s, done_s;
-    __shared__ int wtot[kPT / 32];
+    __shared__ int wtot[kSelT / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int u = ub0 + blockIdx.x, M = P - Rw;
     const float *F = Fp + (size_t)blockIdx.x * P;
     int *upos = pos + (size_t)u * cap;
     unsigned long long prefix = 0;
     int remaining = C;
-    static_assert(kPT == 256, "one thread per bucket");
-    constexpr int kSelBatch = 8;                                         // keys per thread in flight
+    constexpr int kSelBatch = 4;                                         // keys per thread in flight
     for (int pass = 7; pass >= 0; --pass) {
-        hist[tid] = 0;
+        if (tid < 256) hist[tid] = 0;
         __syncthreads();
         const int shift = 8 * pass;
-        for (int c0 = 0; c0 < M; c0 += kPT * kSelBatch) {
+        for (int c0 = 0; c0 < M; c0 += kSelT * kSelBatch) {
             // the loads of a batch are issued together: a pass is a chain of L2 round trips otherwise
             unsigned int fb[kSelBatch];
 #pragma unroll
             for (int i = 0; i < kSelBatch; ++i) {
-                const int j = c0 + i * kPT + tid;
+                const int j = c0 + i * kSelT + tid;
                 fb[i] = j < M ? __float_as_uint(F[j]) : 0u;
             }
 #pragma unroll
             for (int i = 0; i < kSelBatch; ++i) {
-                const int j = c0 + i * kPT + tid;
+                if (c0 + i * kSelT >= M) break;                          // uniform over the CTA
+                const int j = c0 + i * kSelT + tid;
                 unsigned int bin = 256u;                                 // 256: not counted in this pass
                 if (j < M) {
                     const unsigned long long key = rank_key(fb[i], j);
@@ -217,26 +218,32 @@ __global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__rest
         }
         __syncthreads();
         // the bucket b that holds the `remaining`-th best key: above(b) < remaining <= above(b) + hist[b], with
-        // above(b) the number of keys in higher buckets.  Thread b owns bucket b; exactly one thread qualifies.
-        const int h = (int)hist[tid];
-        int incl = h;                                                    // sum over this warp's buckets >= tid
+        // above(b) the number of keys in higher buckets.  Thread b < 256 owns bucket b; exactly one qualifies.
+        int h = 0, incl = 0;
+        if (tid < 256) {                                                 // whole warps 0..7
+            h = (int)hist[tid];
+            incl = h;                                                    // sum over this warp's buckets >= tid
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_down_sync(0xffffffffu, incl, o);
-            if (lane + o < 32) incl += up;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_down_sync(0xffffffffu, incl, o);
+                if (lane + o < 32) incl += up;
+            }
+            if (lane == 0) wtot[warp] = incl;
         }
-        if (lane == 0) wtot[warp] = incl;
         __syncthreads();
-        int above = incl - h;
-        for (int w = warp + 1; w < kPT / 32; ++w) above += wtot[w];
-        if (h > 0 && above < remaining && remaining <= above + h) {
-            const unsigned long long np = (prefix << 8) | (unsigned long long)tid;
-            // the bucket fills the remaining places exactly: every key in it is kept, so the smallest key with
-            // this prefix is the threshold and the finer passes (mostly tie-breaking position bits) are not needed
-            const bool exact = above + h == remaining;
-            remaining_s = remaining - above;
-            prefix_s = exact ? np << shift : np;
-            done_s = exact ? 1 : 0;
+        if (tid < 256) {
+            int above = incl - h;
+            for (int w = warp + 1; w < 8; ++w) above += wtot[w];
+            if (h > 0 && above < remaining && remaining <= above + h) {
+                const unsigned long long np = (prefix << 8) | (unsigned long long)tid;
+                // the bucket fills the remaining places exactly: every key in it is kept, so the smallest key with
+                // this prefix is the threshold and the finer passes (mostly tie-breaking position bits) are not
+                // needed
+                const bool exact = above + h == remaining;
+                remaining_s = remaining - above;
+                prefix_s = exact ? np << shift : np;
+                done_s = exact ? 1 : 0;
+            }
         }
         __syncthreads();
         prefix = prefix_s;
@@ -245,30 +252,27 @@ __global__ void __launch_bounds__(kPT) prefill_select_kernel(const float *__rest
         __syncthreads();
         if (done) break;
     }
+    // order-preserving compaction of the kept positions, kSelT keys per round
     int base = 0;
-    for (int c0 = 0; c0 < M; c0 += kPT * kSelBatch) {
-        unsigned int fb[kSelBatch];
+    for (int c0 = 0; c0 < M; c0 += kSelT) {
+        const int j = c0 + tid;
+        const bool keep = j < M && rank_key(__float_as_uint(F[j]), j) >= prefix;
+        const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) wtot[warp] = __popc(bal);
+        __syncthreads();
+        int incl = wtot[lane];                                           // every warp scans the 32 warp totals
 #pragma unroll
-        for (int i = 0; i < kSelBatch; ++i) {
-            const int j = c0 + i * kPT + tid;
-            fb[i] = j < M ? __float_as_uint(F[j]) : 0u;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int dn = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += dn;
         }
-#pragma unroll
-        for (int i = 0; i < kSelBatch; ++i) {
-            const int j = c0 + i * kPT + tid;
-            if (c0 + i * kPT >= M) break;                                // uniform over the CTA
-            const bool keep = j < M && rank_key(fb[i], j) >= prefix;
-            const unsigned int bal = __ballot_sync(0xffffffffu, keep);
-            if (lane == 0) wtot[warp] = __popc(bal);
-            __syncthreads();
-            int off = base;
-            for (int w = 0; w < warp; ++w) off += wtot[w];
-            if (keep) upos[off + __popc(bal & ((1u << lane) - 1u))] = j;
-            for (int w = 0; w < kPT / 32; ++w) base += wtot[w];
-            __syncthreads();
-        }
+        const int before = warp == 0 ? 0 : __shfl_sync(0xffffffffu, incl, warp - 1);
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        if (keep) upos[base + before + __popc(bal & ((1u << lane) - 1u))] = j;
+        base += total;
+        __syncthreads();
     }
-    for (int i = tid; i < Rw; i += kPT) upos[C + i] = M + i;
+    for (int i = tid; i < Rw; i += kSelT) upos[C + i] = M + i;
 }
 
 __global__ void prefill_identity_pos_kernel(int *pos, int U, int n, int cap)
@@ -439,7 +443,7 @@ cudaError_t run_prefill_t(const DecodeArgs &a, const T *k, const T *v, const T *
                     S, a.ring_c, Fp, ub0, P, Rw, a.Gq, G, R, a.fusion, shift);
                 ++*launches;
             }
-            prefill_select_kernel<<<nb, kPT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
+            prefill_select_kernel<<<nb, kSelT, 0, stream>>>(Fp, a.pos, ub0, P, Rw, C, a.cap);
             ++*launches;
         }
     }
