@@ -1,4 +1,5 @@
-// Prompt-phase scoring on the tensor cores (bf16, head_dim 128, GQA group in {1,2,4,8,16}, window rows R*G <= 256).
+// Prompt-phase scoring on the tensor cores (bf16, head_dim 128, GQA group in {1,2,4,8,16}; a window of more than 256
+// rows R*G is scored in pieces of up to 256 rows, one pair of passes per piece, the pieces' scores fused in place).
 //
 // One application of Algorithm 1 to the whole prompt needs, for every older prompt token k, the fused score
 // F[k] = sum_r / max_r of S_r[k], S_r[k] = sum over the GQA group of the causal soft-max weight window row r puts
@@ -40,7 +41,9 @@ struct PfArgs {
     int ub0;                     // first unit of this batch
     int P, Rw, G, R;
     int Gq;                      // real heads per unit in qwin; heads Gq .. G-1 are padding
-    int rows;                    // Rw * G window rows; row = window slot * G + head
+    int rows;                    // window rows of this launch; row = (window slot - i0) * G + head
+    int i0;                      // first window slot of this launch (a wide window is scored piece by piece)
+    int accumulate;              // pass 2: fuse the scores into Fp (a later piece) instead of writing them
     int qrows;                   // rows padded to a multiple of 128 (pass 1: MMA M blocks)
     int rpad;                    // rows padded to a multiple of 32 (pass 2: MMA N)
     int splits;                  // CTAs per unit along the keys
@@ -95,7 +98,7 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
         uint4 v = make_uint4(0, 0, 0, 0);
         if (row < a.rows && row % G < a.Gq) {
             const int i = row / G, g = row % G;
-            v = reinterpret_cast<const uint4 *>(a.qwin + (((size_t)u * a.Gq + g) * a.Rw + i) * kD)[ch];
+            v = reinterpret_cast<const uint4 *>(a.qwin + (((size_t)u * a.Gq + g) * a.Rw + a.i0 + i) * kD)[ch];
         }
         const uint32_t off = (uint32_t)((ch >> 3) * (QR * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4));
         *reinterpret_cast<uint4 *>(smem + off) = v;
@@ -119,7 +122,7 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
                 nc = -c;
                 if (sp == 0) {
                     const int i = row / G, g = row % G;
-                    const int rslot = (a.P - a.Rw + i) % a.R;
+                    const int rslot = (a.P - a.Rw + a.i0 + i) % a.R;
                     a.ring_c[((size_t)u * a.R + rslot) * G + g] = c;
                 }
             }
@@ -220,7 +223,7 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
 #pragma unroll
             for (int rb = 0; rb < 2; ++rb) {
                 const int row = rb * 128 + lq;
-                lim[rb] = (rb < RB && row < a.rows) ? a.P - a.Rw + row / G : -1;
+                lim[rb] = (rb < RB && row < a.rows) ? a.P - a.Rw + a.i0 + row / G : -1;
             }
             for (int j = grp; j < ntile && ok; j += kPfGroups) {
                 const int b = grp;
@@ -289,7 +292,10 @@ prefill_tc_kernel(const __grid_constant__ PfArgs a, const __grid_constant__ CUte
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * b);
                 __syncwarp();
                 const int key = (t0 + j) * kTile + lq;
-                if (key < nkeys) Fu[key] = F;
+                if (key < nkeys) {
+                    if (a.accumulate) F = FUSION == kFusionSum ? Fu[key] + F : fmaxf(Fu[key], F);   // Eq. 5 / 6 over the pieces
+                    Fu[key] = F;
+                }
             }
         }
     }
@@ -335,7 +341,7 @@ cudaError_t launch_pass_any(const PfArgs &a, const CUtensorMap &tm, int nb, int 
 
 bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P)
 {
-    return tc_shape_supported(f32, D, G, R) && tc_ring_chunks(G, R) == 1 && ((uintptr_t)k & 15) == 0 && P >= 1;
+    return tc_shape_supported(f32, D, G, R) && ((uintptr_t)k & 15) == 0 && P >= 1;
 }
 
 int prefill_tc_splits(int units_in_batch, int P, int window_rows)
@@ -345,7 +351,7 @@ int prefill_tc_splits(int units_in_batch, int P, int window_rows)
     // waves of `slots` resident CTAs: take the split with the fewest tile-times over all waves.
     constexpr int kSetupTiles = 3;
     const int nt = (P + kTile - 1) / kTile;
-    const int slots = 148 * (window_rows <= 128 ? 2 : 1);
+    const int slots = 148 * (window_rows <= 128 ? 2 : 1);             // pieces of a wide window: one CTA per SM
     int best = 1;
     long long best_cost = -1;
     for (int s = 1; s <= nt && s <= 64; ++s) {
@@ -358,7 +364,8 @@ int prefill_tc_splits(int units_in_batch, int P, int window_rows)
 
 size_t prefill_tc_floats_per_unit(int P, int Rw, int G, int splits)
 {
-    const int qrows = ((Rw * G + 127) / 128) * 128;
+    const int rows = Rw * G < 256 ? Rw * G : 256;                        // a launch scores at most 256 window rows
+    const int qrows = ((rows + 127) / 128) * 128;
     return (size_t)P + (size_t)splits * kPfGroups * qrows * 2;
 }
 
@@ -373,19 +380,27 @@ cudaError_t run_prefill_scores_tc(const DecodeArgs &a, const void *k, const void
     pa.qwin = static_cast<const __nv_bfloat16 *>(qwin);
     pa.part_ml = part; pa.ring_c = a.ring_c; pa.Fp = Fp; pa.err = err;
     pa.ub0 = ub0; pa.P = P; pa.Rw = P < a.R ? P : a.R; pa.G = a.G; pa.R = a.R; pa.Gq = a.Gq;
-    pa.rows = pa.Rw * a.G;
-    pa.qrows = ((pa.rows + 127) / 128) * 128;
-    pa.rpad = (pa.rows + 31) & ~31;
     pa.splits = splits;
     pa.tmem_cols = 0;
-    pa.stages = pf_stages(pa.qrows);
     pa.scale2 = a.scale2;
     pa.wait_cycles = kWaitCycles;
-    cudaError_t e = launch_pass_any<1>(pa, tm, nb, a.fusion, stream);
-    if (e != cudaSuccess) return e;
-    e = launch_pass_any<2>(pa, tm, nb, a.fusion, stream);
-    *launches += 2;
-    return e;
+    // up to 256 window rows per pair of passes; the rows of a wider window are taken in pieces of whole window
+    // slots, whose normalisers are independent and whose scores fuse associatively (Eq. 5 / 6)
+    const int slots_per_piece = 256 / a.G;
+    for (int i0 = 0; i0 < pa.Rw; i0 += slots_per_piece) {
+        pa.i0 = i0;
+        pa.accumulate = i0 > 0 ? 1 : 0;
+        pa.rows = min(slots_per_piece, pa.Rw - i0) * a.G;
+        pa.qrows = ((pa.rows + 127) / 128) * 128;
+        pa.rpad = (pa.rows + 31) & ~31;
+        pa.stages = pf_stages(pa.qrows);
+        cudaError_t e = launch_pass_any<1>(pa, tm, nb, a.fusion, stream);
+        if (e != cudaSuccess) return e;
+        e = launch_pass_any<2>(pa, tm, nb, a.fusion, stream);
+        *launches += 2;
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace mkv
