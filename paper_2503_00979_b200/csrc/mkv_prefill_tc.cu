@@ -341,7 +341,9 @@ cudaError_t launch_pass_any(const PfArgs &a, const CUtensorMap &tm, int nb, int 
 
 bool prefill_tc_supported(bool f32, int D, int G, int R, const void *k, int P)
 {
-    return tc_shape_supported(f32, D, G, R) && ((uintptr_t)k & 15) == 0 && P >= 1;
+    // any window: the pieces need no more than 256 rows at a time (the decode kernel's own limit on the ring, which
+    // the stored-profile mode lifts, does not apply here)
+    return !f32 && D == kD && G >= 1 && G <= kMaxGroup && R >= 1 && ((uintptr_t)k & 15) == 0 && P >= 1;
 }
 
 int prefill_tc_splits(int units_in_batch, int P, int window_rows)

@@ -438,21 +438,24 @@ def test_long_prompt_selection_against_the_oracle(P, layers, n_units):
     assert rep.kernel == "tc" and rep.evictions == rep.units * 8 and rep.prefill_resyncs <= 1
 
 
-@pytest.mark.parametrize("q_heads,kv_heads,R,pieces", [(8, 2, 200, 4), (14, 2, 40, 2), (8, 2, 32, 1)])
-def test_prompt_phase_of_a_wide_window_scores_on_the_tensor_cores(q_heads, kv_heads, R, pieces):
+@pytest.mark.parametrize("q_heads,kv_heads,R,pieces,profile", [(8, 2, 200, 4, "recompute"), (14, 2, 40, 2, "recompute"),
+                                                                (8, 2, 32, 1, "recompute"), (8, 2, 700, 11, "stored")])
+def test_prompt_phase_of_a_wide_window_scores_on_the_tensor_cores(q_heads, kv_heads, R, pieces, profile):
     # a window of more than 256 rows R * G' is scored in pieces of 256 / G' window slots, one pair of tensor-core
     # passes per piece: the call then launches arena set-up, 2 x pieces scoring passes, the selection, the gather,
-    # the ring copy and the state kernel (the CUDA-core scoring path would launch three scoring kernels instead);
+    # the ring copy and the state kernel (the CUDA-core scoring path would launch two or three scoring kernels instead);
     # that the pieces' scores fuse to the oracle's is what the wide-window parity tests above check
     w = synth.Workload("wide_prompt", 1, 1, q_heads, kv_heads, 128, "bf16", 900, 4, 500, R, "sum", 3)
     st = synth.Stream(w, torch.device("cuda:0"))
     k, v = st.kv(np.arange(w.prompt_len))
     qw = st.q(np.arange(w.prompt_len - R, w.prompt_len))
-    mk = binding.MorphKV(1, 1, q_heads, kv_heads, 128, w.C, R, w.fusion, "bf16")
+    mk = binding.MorphKV(1, 1, q_heads, kv_heads, 128, w.C, R, w.fusion, "bf16", profile=profile)
     assert mk.kernel_name == "tc"
     n0 = mk.launch_count
     mk.prefill(k.bfloat16().contiguous(), v.bfloat16().contiguous(), qw.bfloat16().contiguous())
-    assert mk.launch_count - n0 == 1 + 2 * pieces + 1 + 2 + 1
+    # (a window of 700 keeps the whole 900-token prompt: the position kernel stands in for the selection; the stored
+    # profile adds the launch that fills its table)
+    assert mk.launch_count - n0 == 1 + 2 * pieces + 1 + 2 + 1 + (1 if profile == "stored" else 0)
     mk.close()
 
 
