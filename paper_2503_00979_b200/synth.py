@@ -125,6 +125,8 @@ for _P in (6144, 32768, 131072):
 # the long-response setting with a window of 200 recent tokens inside a 4K budget, on the Llama-3.1-8B-shaped stack:
 # 800 ring rows per unit, more than one tensor-core operand holds
 WORKLOADS["w200"] = Workload("w200", 32, 1, 32, 8, 128, "bf16", 4096, 4096, 3896, 200, "sum", _SEED0 + 6)
+# its prompt phase: a 6144-token prompt compressed into that budget (the 800 window rows are scored in four pieces)
+WORKLOADS["prefill_w200_P6144"] = Workload("prefill_w200_P6144", 32, 1, 32, 8, 128, "bf16", 6144, 8, 3896, 200, "sum", _SEED0 + 7)
 
 
 class Stream:

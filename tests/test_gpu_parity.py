@@ -428,11 +428,12 @@ def test_config1_all_units_prompt_phase_and_first_steps_against_the_oracle():
 
 
 # ---- long prompts into a 2K cache (the long-context setting): the prompt phase on the tensor cores
-@pytest.mark.parametrize("P,layers,n_units", [(6144, 4, 8), (32768, 1, 3)])
-def test_long_prompt_selection_against_the_oracle(P, layers, n_units):
+@pytest.mark.parametrize("name,layers,n_units", [("prefill_P6144", 4, 8), ("prefill_P32768", 1, 3),
+                                                 ("prefill_w200_P6144", 2, 4)])      # window of 200: four pieces
+def test_long_prompt_selection_against_the_oracle(name, layers, n_units):
     # retained set of every checked unit against the oracle's one-shot Algorithm 1 (near-tie rule), kept K/V rows
     # bit for bit, then a few decode steps whose outputs depend on the window rows' normalisers
-    w = synth.WORKLOADS[f"prefill_P{P}"].replace(layers=layers)
+    w = synth.WORKLOADS[name].replace(layers=layers)
     rep = run_parity(w, steps=8, n_units=n_units, chunk=8, check_F_every=8)
     _report(rep)
     assert rep.kernel == "tc" and rep.evictions == rep.units * 8 and rep.prefill_resyncs <= 1
