@@ -379,10 +379,11 @@ def test_full_size_config3_sampled_units_full_cache():
     assert rep.kernel == "tc" and rep.evictions >= 5 * 24
 
 
-@pytest.mark.parametrize("name", ["c4_C512_max", "c4_C8192_sum"])
+@pytest.mark.parametrize("name", [f"c4_C{C}_{f}" for C in (512, 1024, 2048, 4096, 8192) for f in ("sum", "max")])
 def test_full_size_config4_sampled_units(name):
+    # every point of the capacity sweep, both fusions
     w = synth.WORKLOADS[name]
-    steps = 48 if w.C <= 512 else 16
+    steps = 48 if w.C <= 512 else 32 if w.C <= 2048 else 16
     rep = run_parity(w, steps=steps, n_units=6, kernel="auto", check_F_every=8)
     _report(rep)
     assert rep.kernel == "tc" and rep.evictions >= 5 * steps
@@ -404,6 +405,16 @@ def test_full_length_config2_every_generated_step():
     _report(rep)
     assert rep.kernel == "tc" and rep.steps == 4096 and rep.units == 8
     assert rep.evictions == 8 * 4096 and rep.near_tie_resyncs <= 0.002 * rep.evictions + 2
+
+
+@pytest.mark.parametrize("name", [f"c4_C{C}_{f}" for C in (512, 1024, 2048, 4096, 8192) for f in ("sum", "max")])
+def test_full_length_config4_every_generated_step(name):
+    # every point of the capacity sweep over all of its 1024 steps
+    w = synth.WORKLOADS[name]
+    rep = run_parity(w, steps=w.steps, n_units=4, chunk=128, check_F_every=256)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.steps == 1024 and rep.units == 4
+    assert rep.evictions == 4 * 1024 and rep.near_tie_resyncs <= 0.002 * rep.evictions + 2
 
 
 def test_config3_from_its_real_prompt_through_the_fill_into_eviction():
