@@ -318,6 +318,16 @@ def test_windows_of_more_than_256_ring_rows_on_the_tensor_cores(q_heads, kv_head
     assert rep.kernel == "tc" and rep.evictions > 0
 
 
+def test_wide_window_with_a_prompt_shorter_than_the_window():
+    # 150 prompt tokens under a window of 200 (600 window rows: the prompt phase takes them in three pieces and has
+    # no candidates to score); the cache fills for 150 steps, then every step evicts while rows of the prompt are
+    # still inside the window, so the fused scores depend on the normalisers the prompt phase wrote
+    w = synth.Workload("wide_short_prompt", 1, 2, 8, 2, 128, "bf16", 150, 170, 100, 200, "sum", 2024)
+    rep = run_parity(w, steps=w.steps, n_units=4, kernel="auto", check_F_every=5)
+    _report(rep)
+    assert rep.kernel == "tc" and rep.evictions == 4 * 20 and rep.F_compared > 0
+
+
 def test_wide_window_with_per_layer_calls_and_current_normalisation():
     w = synth.Workload("wide_layer", 3, 1, 8, 2, 128, "bf16", 500, 90, 400, 70, "sum", 5)
     rep = run_parity(w, steps=w.steps, n_units=6, kernel="auto", per_layer=1)
